@@ -1,0 +1,92 @@
+/* libmonarch_attn — MonarchAttention forward pass (arXiv 2505.18698) for NVIDIA B200 (sm_100a).
+ *
+ * The method (Sec. 3 of the paper): with N = m*b, find a Monarch matrix M = P^T B whose block
+ * factors L (b x m x m) and R (m x b x b) approximately maximise the softmax variational
+ * objective f(M; Q, K) (Eq. 6) by T rounds of exact alternating maximisation from L = identity
+ * (Eq. 7-10, R before L), then return Y = M V through the two factors (Eq. 4).  The N x N matrix
+ * is never formed.
+ *
+ * Common conventions for every entry point
+ *   - Q, K, V, Y: row-major contiguous [batch][heads][N][d]; row r of a head is block r / b,
+ *     position r % b (text below Eq. 10).  Base addresses 16-byte aligned.  Y has the input
+ *     dtype and must not alias an input.  All buffers are owned by the caller.
+ *   - m = N / b; N must be a multiple of b; T >= 1.
+ *   - softmax scale: multiplies Q (footnote to Eq. 3), i.e. both score tensors, never c_L.
+ *   - Device entry points are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream).  Errors detectable on the host return before anything is enqueued.
+ *   - Return value: an ma_status code.  The library never aborts and never prints.
+ */
+#ifndef MONARCH_ATTN_H_
+#define MONARCH_ATTN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { MA_F32 = 0, MA_F16 = 1, MA_BF16 = 2 } ma_dtype;
+
+typedef enum {
+  MA_OK = 0,
+  MA_ERR_NULL = 1,        /* a required pointer is NULL */
+  MA_ERR_SHAPE = 2,       /* batch, heads, N, d, b <= 0; N % b != 0; T < 1 */
+  MA_ERR_DTYPE = 3,       /* dtype not one of ma_dtype */
+  MA_ERR_UNSUPPORTED = 4, /* the requested path has no kernel for this (b, m, d, dtype) */
+  MA_ERR_ALIGN = 5,       /* a base address is not 16-byte aligned, or Y aliases an input */
+  MA_ERR_WORKSPACE = 6,   /* workspace NULL or smaller than monarch_attn_workspace_bytes() */
+  MA_ERR_CUDA = 7,        /* a CUDA runtime/driver call failed */
+  MA_ERR_TIMEOUT = 8      /* a bounded device-side wait ran out (see monarch_attn_device_status) */
+} ma_status;
+
+/* Which kernels run.  AUTO picks the fastest path that supports the shape. */
+typedef enum {
+  MA_PATH_AUTO = 0,
+  MA_PATH_GENERIC = 1, /* fp32 SIMT kernels, fp32 states; any dtype, any N = m*b that fits smem */
+  MA_PATH_TENSOR = 2   /* tcgen05/TMA kernels, 16-bit states; f16/bf16, d = 64, m = b in {64,128} */
+} ma_path;
+
+/* T-step MonarchAttention forward (Eq. 7-10 then Eq. 4) with scale = 1/sqrt(d).
+ * Q, K, V, Y: DEVICE pointers.  Uses a per-process, per-device workspace that the library grows
+ * on demand (the only allocation it ever makes; call once outside any timed or captured region
+ * to pre-size it).  Not safe to call concurrently from several host threads on one device. */
+int monarch_attn_fwd(const void* Q, const void* K, const void* V, void* Y,
+                     int batch, int heads, int N, int d, int b, int T,
+                     int dtype, void* stream);
+
+/* Bytes of scratch that monarch_attn_fwd_ex needs for this problem on `path`
+ * (states alpha_L, alpha_R, y, c_L, c_R of Sec. 3 'Implementation', plus a status word).
+ * Returns 0 if the arguments are invalid or the path does not support them. */
+size_t monarch_attn_workspace_bytes(int batch, int heads, int N, int d, int b, int T,
+                                    int dtype, int path);
+
+/* As monarch_attn_fwd, with an explicit softmax scale, an explicit path and caller-owned scratch.
+ * workspace: DEVICE pointer, 256-byte aligned, at least monarch_attn_workspace_bytes() long; its
+ * contents are overwritten.  Allocates nothing. */
+int monarch_attn_fwd_ex(const void* Q, const void* K, const void* V, void* Y,
+                        int batch, int heads, int N, int d, int b, int T, int dtype,
+                        float softmax_scale, int path,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* End-to-end variant: Q, K, V, Y are HOST pointers (pinned memory gives asynchronous copies).
+ * Copies Q, K, V to device staging buffers owned by the library, runs monarch_attn_fwd, copies Y
+ * back, all on `stream`; does not synchronise.  Grows the staging buffers on demand. */
+int monarch_attn_fwd_host(const void* Q_host, const void* K_host, const void* V_host, void* Y_host,
+                          int batch, int heads, int N, int d, int b, int T,
+                          int dtype, void* stream);
+
+/* Synchronises `stream` and reads the status word a run left in `workspace` (DEVICE pointer; NULL
+ * means the library's own workspace on the current device): MA_OK, or MA_ERR_TIMEOUT if a bounded
+ * wait inside a kernel gave up (outputs are then undefined). */
+int monarch_attn_device_status(const void* workspace, void* stream);
+
+/* Number of kernel launches the last successful call on this host thread enqueued. */
+int monarch_attn_last_launch_count(void);
+
+/* Static, NUL-terminated description of an ma_status code. */
+const char* monarch_attn_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MONARCH_ATTN_H_ */

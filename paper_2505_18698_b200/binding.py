@@ -1,0 +1,167 @@
+"""ctypes binding of libmonarch_attn.so: argument marshalling only.
+
+Every step of the method runs inside the library's CUDA kernels.  torch is used for device
+memory and streams.  If the shared library has not been built the binding raises; there is no
+CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+import re
+
+import torch
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libmonarch_attn.so")
+HEADER_PATH = os.path.join(os.path.dirname(_PKG_DIR), "include", "monarch_attn.h")
+
+MA_F32, MA_F16, MA_BF16 = 0, 1, 2
+MA_PATH_AUTO, MA_PATH_GENERIC, MA_PATH_TENSOR = 0, 1, 2
+MA_OK = 0
+
+_TORCH_TO_CODE = {torch.float32: MA_F32, torch.float16: MA_F16, torch.bfloat16: MA_BF16}
+_NAME_TO_TORCH = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
+
+_lib = None
+
+
+class MonarchAttnError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"monarch_attn: {what} (status {code})")
+        self.code = code
+
+
+def declared_symbols(header_path: str = HEADER_PATH):
+    """Names of the functions the public header declares."""
+    text = open(header_path).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(monarch_attn_\w+)\s*\(", text)))
+
+
+def load_library(path: str = LIB_PATH):
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(path):
+        raise MonarchAttnError(-1, f"{path} is missing: build it with __graft_entry__.build()")
+    lib = ctypes.CDLL(path)
+    vp, i, sz, f = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_float
+    lib.monarch_attn_fwd.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
+    lib.monarch_attn_fwd.restype = i
+    lib.monarch_attn_workspace_bytes.argtypes = [i, i, i, i, i, i, i, i]
+    lib.monarch_attn_workspace_bytes.restype = sz
+    lib.monarch_attn_fwd_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, sz, vp]
+    lib.monarch_attn_fwd_ex.restype = i
+    lib.monarch_attn_fwd_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
+    lib.monarch_attn_fwd_host.restype = i
+    lib.monarch_attn_device_status.argtypes = [vp, vp]
+    lib.monarch_attn_device_status.restype = i
+    lib.monarch_attn_last_launch_count.argtypes = []
+    lib.monarch_attn_last_launch_count.restype = i
+    lib.monarch_attn_status_string.argtypes = [i]
+    lib.monarch_attn_status_string.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().monarch_attn_status_string(int(code)).decode()
+
+
+def _check(code: int):
+    if code != MA_OK:
+        raise MonarchAttnError(code, status_string(code))
+
+
+def _stream_ptr(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _shape_of(Q, K, V):
+    if Q.dim() != 4:
+        raise ValueError("Q, K, V must be (batch, heads, N, d)")
+    if not (Q.shape == K.shape == V.shape and Q.dtype == K.dtype == V.dtype):
+        raise ValueError("Q, K, V must share shape and dtype")
+    if Q.dtype not in _TORCH_TO_CODE:
+        raise ValueError(f"unsupported dtype {Q.dtype}")
+    for t in (Q, K, V):
+        if not t.is_contiguous():
+            raise ValueError("Q, K, V must be contiguous")
+    return tuple(int(x) for x in Q.shape)
+
+
+def monarch_attn_workspace_bytes(batch, heads, N, d, b, T, dtype, path=MA_PATH_AUTO) -> int:
+    code = _TORCH_TO_CODE[dtype] if isinstance(dtype, torch.dtype) else int(dtype)
+    return int(load_library().monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, path))
+
+
+def monarch_attn_fwd(Q, K, V, b, T, Y=None, stream=None):
+    """Y = MonarchAttention(Q, K, V) with block size b, T steps, scale 1/sqrt(d).
+    Q, K, V: CUDA tensors (batch, heads, N, d)."""
+    lib = load_library()
+    if not Q.is_cuda:
+        raise MonarchAttnError(-2, "monarch_attn_fwd needs CUDA tensors; there is no CPU path")
+    batch, heads, N, d = _shape_of(Q, K, V)
+    if Y is None:
+        Y = torch.empty_like(Q)
+    _check(lib.monarch_attn_fwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                batch, heads, N, d, b, T, _TORCH_TO_CODE[Q.dtype],
+                                _stream_ptr(stream)))
+    return Y
+
+
+def monarch_attn_fwd_ex(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, workspace=None,
+                        Y=None, stream=None):
+    """As monarch_attn_fwd with explicit scale, path and (optionally) caller-owned workspace
+    (a uint8 CUDA tensor).  Returns Y."""
+    lib = load_library()
+    if not Q.is_cuda:
+        raise MonarchAttnError(-2, "monarch_attn_fwd_ex needs CUDA tensors; there is no CPU path")
+    batch, heads, N, d = _shape_of(Q, K, V)
+    code = _TORCH_TO_CODE[Q.dtype]
+    if softmax_scale is None:
+        softmax_scale = 1.0 / math.sqrt(d)
+    if Y is None:
+        Y = torch.empty_like(Q)
+    if workspace is None:
+        need = lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, path)
+        workspace = torch.empty(max(int(need), 256), dtype=torch.uint8, device=Q.device)
+    _check(lib.monarch_attn_fwd_ex(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                   batch, heads, N, d, b, T, code, float(softmax_scale), int(path),
+                                   workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
+    return Y
+
+
+def monarch_attn_fwd_host(Qh, Kh, Vh, Yh, b, T, stream=None):
+    """End-to-end call on HOST tensors (pinned for asynchronous copies): H2D, kernels, D2H on
+    `stream`; returns Yh without synchronising."""
+    lib = load_library()
+    batch, heads, N, d = _shape_of(Qh, Kh, Vh)
+    if Qh.is_cuda or Yh.is_cuda:
+        raise ValueError("monarch_attn_fwd_host takes host tensors")
+    _check(lib.monarch_attn_fwd_host(Qh.data_ptr(), Kh.data_ptr(), Vh.data_ptr(), Yh.data_ptr(),
+                                     batch, heads, N, d, b, T, _TORCH_TO_CODE[Qh.dtype],
+                                     _stream_ptr(stream)))
+    return Yh
+
+
+def monarch_attn_device_status(workspace=None, stream=None) -> int:
+    lib = load_library()
+    ptr = None if workspace is None else workspace.data_ptr()
+    return int(lib.monarch_attn_device_status(ptr, _stream_ptr(stream)))
+
+
+def monarch_attn_last_launch_count() -> int:
+    return int(load_library().monarch_attn_last_launch_count())
+
+
+def torch_dtype(name: str) -> torch.dtype:
+    return _NAME_TO_TORCH[name]
+
+
+def to_device(x_f32_numpy, dtype_name: str, device="cuda"):
+    """float32 numpy array whose values are representable in `dtype_name` -> torch tensor."""
+    return torch.from_numpy(x_f32_numpy).to(device=device, dtype=_NAME_TO_TORCH[dtype_name]).contiguous()

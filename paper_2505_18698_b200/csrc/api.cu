@@ -1,0 +1,306 @@
+// C-ABI boundary of libmonarch_attn: argument validation, workspace layout, path selection and
+// kernel launches.  No torch types; plain device/host pointers and sizes only.
+#include "../../include/monarch_attn.h"
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "generic_kernels.cuh"
+#include "tensor_path.cuh"
+
+namespace ma {
+
+static thread_local int g_last_launches = 0;
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int esize(int dtype) { return dtype == MA_F32 ? 4 : 2; }
+
+struct Problem {
+  int batch, heads, N, d, b, T, dtype, m, BH;
+};
+
+static int validate_shape(int batch, int heads, int N, int d, int b, int T, int dtype, Problem* p) {
+  if (dtype != MA_F32 && dtype != MA_F16 && dtype != MA_BF16) return MA_ERR_DTYPE;
+  if (batch <= 0 || heads <= 0 || N <= 0 || d <= 0 || b <= 0 || T < 1) return MA_ERR_SHAPE;
+  if (N % b != 0) return MA_ERR_SHAPE;
+  if ((long long)batch * heads > 0x7fffffffLL / 2) return MA_ERR_SHAPE;
+  *p = Problem{batch, heads, N, d, b, T, dtype, N / b, batch * heads};
+  return MA_OK;
+}
+
+// ------------------------------------------------------------------ generic path
+constexpr size_t kStatusBytes = 256;
+constexpr size_t kMaxSmem = 227 * 1024;
+
+static bool generic_supported(const Problem& p) {
+  if (p.BH > 65535) return false;   // gridDim.y
+  size_t r = generic::r_step_smem_floats(p.b, p.d, true) * 4;
+  size_t l = generic::l_step_smem_floats(p.m, p.d, false) * 4;
+  size_t lf = generic::l_step_smem_floats(p.m, p.d, true) * 4;
+  return r <= kMaxSmem && l <= kMaxSmem && lf <= kMaxSmem;
+}
+
+struct GenericWs {
+  int* status;
+  float *aL, *aR, *y, *cL, *cR;
+  size_t bytes;
+};
+
+static GenericWs generic_layout(const Problem& p, void* base) {
+  GenericWs w;
+  char* c = (char*)base;
+  size_t off = 0;
+  size_t big = align_up((size_t)p.BH * p.N * p.d * 4, 256);
+  size_t small = align_up((size_t)p.BH * p.N * 4, 256);
+  w.status = (int*)(c + off); off += kStatusBytes;
+  w.aL = (float*)(c + off); off += big;
+  w.aR = (float*)(c + off); off += big;
+  w.y = (float*)(c + off); off += big;
+  w.cL = (float*)(c + off); off += small;
+  w.cR = (float*)(c + off); off += small;
+  w.bytes = off;
+  return w;
+}
+
+template <typename TIn>
+static int launch_generic_t(const Problem& p, const TIn* Q, const TIn* K, const TIn* V, TIn* Y,
+                            float scale, const GenericWs& w, cudaStream_t st) {
+  using namespace generic;
+  int launches = 0;
+  dim3 gr(p.m, p.BH), gl(p.b, p.BH);
+  auto set_smem = [](const void* f, size_t bytes) {
+    return cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  };
+  if (cudaMemsetAsync(w.status, 0, kStatusBytes, st) != cudaSuccess) return MA_ERR_CUDA;
+  for (int t = 1; t <= p.T; ++t) {
+    const bool first = (t == 1), last = (t == p.T);
+    size_t rs = r_step_smem_floats(p.b, p.d, last) * 4;
+#define MA_LAUNCH_R(FIRST, WITHV)                                                              \
+  do {                                                                                         \
+    if (set_smem((const void*)r_step_kernel<TIn, FIRST, WITHV>, rs) != cudaSuccess)            \
+      return MA_ERR_CUDA;                                                                      \
+    r_step_kernel<TIn, FIRST, WITHV><<<gr, kThreads, rs, st>>>(Q, K, V, w.aR, w.cR, w.aL,     \
+                                                                w.cL, w.y, p.N, p.d, p.b, p.m, \
+                                                                scale);                        \
+  } while (0)
+    if (first && last) MA_LAUNCH_R(true, true);
+    else if (first) MA_LAUNCH_R(true, false);
+    else if (last) MA_LAUNCH_R(false, true);
+    else MA_LAUNCH_R(false, false);
+#undef MA_LAUNCH_R
+    ++launches;
+    size_t ls = l_step_smem_floats(p.m, p.d, last) * 4;
+    if (last) {
+      if (set_smem((const void*)l_step_kernel<TIn, true>, ls) != cudaSuccess) return MA_ERR_CUDA;
+      l_step_kernel<TIn, true><<<gl, kThreads, ls, st>>>(Q, w.aL, w.cL, w.y, w.aR, w.cR, Y, p.N,
+                                                         p.d, p.b, p.m, scale);
+    } else {
+      if (set_smem((const void*)l_step_kernel<TIn, false>, ls) != cudaSuccess) return MA_ERR_CUDA;
+      l_step_kernel<TIn, false><<<gl, kThreads, ls, st>>>(Q, w.aL, w.cL, w.y, w.aR, w.cR, Y, p.N,
+                                                          p.d, p.b, p.m, scale);
+    }
+    ++launches;
+  }
+  if (cudaGetLastError() != cudaSuccess) return MA_ERR_CUDA;
+  g_last_launches = launches;
+  return MA_OK;
+}
+
+static int launch_generic(const Problem& p, const void* Q, const void* K, const void* V, void* Y,
+                          float scale, void* ws, cudaStream_t st) {
+  GenericWs w = generic_layout(p, ws);
+  switch (p.dtype) {
+    case MA_F32:
+      return launch_generic_t<float>(p, (const float*)Q, (const float*)K, (const float*)V,
+                                     (float*)Y, scale, w, st);
+    case MA_F16:
+      return launch_generic_t<__half>(p, (const __half*)Q, (const __half*)K, (const __half*)V,
+                                      (__half*)Y, scale, w, st);
+    default:
+      return launch_generic_t<__nv_bfloat16>(p, (const __nv_bfloat16*)Q, (const __nv_bfloat16*)K,
+                                             (const __nv_bfloat16*)V, (__nv_bfloat16*)Y, scale, w,
+                                             st);
+  }
+}
+
+// ------------------------------------------------------------------ path selection
+static int resolve_path(const Problem& p, int path) {
+  if (path == MA_PATH_AUTO) {
+    if (tensor::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TENSOR;
+    if (generic_supported(p)) return MA_PATH_GENERIC;
+    return -1;
+  }
+  if (path == MA_PATH_GENERIC) return generic_supported(p) ? path : -1;
+  if (path == MA_PATH_TENSOR)
+    return tensor::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
+  return -1;
+}
+
+static size_t workspace_bytes_for(const Problem& p, int resolved) {
+  if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
+  if (resolved == MA_PATH_TENSOR) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
+  return 0;
+}
+
+// ------------------------------------------------------------------ library-owned buffers
+constexpr int kMaxDevices = 64;
+struct DeviceBuffers {
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  void* stage = nullptr;   // Q, K, V, Y staging for the host entry point
+  size_t stage_bytes = 0;
+};
+static DeviceBuffers g_dev[kMaxDevices];
+
+static int grow(void** ptr, size_t* have, size_t need) {
+  if (*have >= need) return MA_OK;
+  if (*ptr) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return MA_ERR_CUDA;
+    cudaFree(*ptr);
+    *ptr = nullptr;
+    *have = 0;
+  }
+  size_t sz = align_up(need, (size_t)1 << 20);
+  if (cudaMalloc(ptr, sz) != cudaSuccess) {
+    cudaGetLastError();
+    *ptr = nullptr;
+    return MA_ERR_CUDA;
+  }
+  *have = sz;
+  return MA_OK;
+}
+
+static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Problem& p,
+                  float scale, int resolved, void* ws, size_t ws_bytes, cudaStream_t st) {
+  if (!ws || ws_bytes < workspace_bytes_for(p, resolved)) return MA_ERR_WORKSPACE;
+  if (((uintptr_t)ws & 255) != 0) return MA_ERR_ALIGN;
+  if (resolved == MA_PATH_GENERIC) return launch_generic(p, Q, K, V, Y, scale, ws, st);
+  int launches = 0;
+  int rc = tensor::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.T, p.dtype, scale, ws, st, &launches);
+  if (rc == MA_OK) g_last_launches = launches;
+  return rc;
+}
+
+static int check_ptrs(const void* Q, const void* K, const void* V, void* Y, const Problem& p) {
+  if (!Q || !K || !V || !Y) return MA_ERR_NULL;
+  if ((((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)Y) & 15) != 0) return MA_ERR_ALIGN;
+  size_t bytes = (size_t)p.BH * p.N * p.d * esize(p.dtype);
+  const char* y0 = (const char*)Y;
+  const void* in[3] = {Q, K, V};
+  for (int i = 0; i < 3; ++i) {
+    const char* a = (const char*)in[i];
+    if (y0 < a + bytes && a < y0 + bytes) return MA_ERR_ALIGN;
+  }
+  return MA_OK;
+}
+
+}  // namespace ma
+
+using namespace ma;
+
+extern "C" {
+
+size_t monarch_attn_workspace_bytes(int batch, int heads, int N, int d, int b, int T, int dtype,
+                                    int path) {
+  Problem p;
+  if (validate_shape(batch, heads, N, d, b, T, dtype, &p) != MA_OK) return 0;
+  int r = resolve_path(p, path);
+  if (r < 0) return 0;
+  return workspace_bytes_for(p, r);
+}
+
+int monarch_attn_fwd_ex(const void* Q, const void* K, const void* V, void* Y, int batch, int heads,
+                        int N, int d, int b, int T, int dtype, float softmax_scale, int path,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+  Problem p;
+  int rc = validate_shape(batch, heads, N, d, b, T, dtype, &p);
+  if (rc != MA_OK) return rc;
+  rc = check_ptrs(Q, K, V, Y, p);
+  if (rc != MA_OK) return rc;
+  if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
+  int r = resolve_path(p, path);
+  if (r < 0) return MA_ERR_UNSUPPORTED;
+  return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+int monarch_attn_fwd(const void* Q, const void* K, const void* V, void* Y, int batch, int heads,
+                     int N, int d, int b, int T, int dtype, void* stream) {
+  Problem p;
+  int rc = validate_shape(batch, heads, N, d, b, T, dtype, &p);
+  if (rc != MA_OK) return rc;
+  rc = check_ptrs(Q, K, V, Y, p);
+  if (rc != MA_OK) return rc;
+  int r = resolve_path(p, MA_PATH_AUTO);
+  if (r < 0) return MA_ERR_UNSUPPORTED;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MA_ERR_CUDA;
+  DeviceBuffers& B = g_dev[dev];
+  rc = grow(&B.ws, &B.ws_bytes, workspace_bytes_for(p, r));
+  if (rc != MA_OK) return rc;
+  return fwd_ex(Q, K, V, Y, p, 1.0f / sqrtf((float)d), r, B.ws, B.ws_bytes, (cudaStream_t)stream);
+}
+
+int monarch_attn_fwd_host(const void* Qh, const void* Kh, const void* Vh, void* Yh, int batch,
+                          int heads, int N, int d, int b, int T, int dtype, void* stream) {
+  Problem p;
+  int rc = validate_shape(batch, heads, N, d, b, T, dtype, &p);
+  if (rc != MA_OK) return rc;
+  if (!Qh || !Kh || !Vh || !Yh) return MA_ERR_NULL;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MA_ERR_CUDA;
+  DeviceBuffers& B = g_dev[dev];
+  size_t one = align_up((size_t)p.BH * p.N * p.d * esize(p.dtype), 256);
+  rc = grow(&B.stage, &B.stage_bytes, 4 * one);
+  if (rc != MA_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* s = (char*)B.stage;
+  size_t bytes = (size_t)p.BH * p.N * p.d * esize(p.dtype);
+  if (cudaMemcpyAsync(s, Qh, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(s + one, Kh, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(s + 2 * one, Vh, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return MA_ERR_CUDA;
+  rc = monarch_attn_fwd(s, s + one, s + 2 * one, s + 3 * one, batch, heads, N, d, b, T, dtype,
+                        stream);
+  if (rc != MA_OK) return rc;
+  if (cudaMemcpyAsync(Yh, s + 3 * one, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return MA_ERR_CUDA;
+  return MA_OK;
+}
+
+int monarch_attn_device_status(const void* workspace, void* stream) {
+  const void* ws = workspace;
+  if (!ws) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MA_ERR_CUDA;
+    ws = g_dev[dev].ws;
+    if (!ws) return MA_OK;
+  }
+  int word = 0;
+  if (cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream) !=
+      cudaSuccess)
+    return MA_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MA_ERR_CUDA;
+  return word == 0 ? MA_OK : MA_ERR_TIMEOUT;
+}
+
+int monarch_attn_last_launch_count(void) { return g_last_launches; }
+
+const char* monarch_attn_status_string(int status) {
+  switch (status) {
+    case MA_OK: return "ok";
+    case MA_ERR_NULL: return "a required pointer is NULL";
+    case MA_ERR_SHAPE: return "invalid shape: need batch, heads, N, d, b > 0, N % b == 0, T >= 1";
+    case MA_ERR_DTYPE: return "unknown dtype";
+    case MA_ERR_UNSUPPORTED: return "no kernel on the requested path for this (b, m, d, dtype)";
+    case MA_ERR_ALIGN: return "pointer not aligned, or output aliases an input";
+    case MA_ERR_WORKSPACE: return "workspace missing or too small";
+    case MA_ERR_CUDA: return "a CUDA call failed";
+    case MA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

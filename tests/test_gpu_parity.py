@@ -1,0 +1,178 @@
+"""Parity of the CUDA path (through the C-ABI) with the fp64 oracle on the same seeded inputs.
+
+Metric and bar: max over (batch, head) of ||Y_gpu - Y_ref||_F / ||Y_ref||_F  <= 1e-2 for
+f16/bf16 inputs (fp32 accumulation), <= 1e-5 for fp32 inputs.
+"""
+import numpy as np
+import pytest
+import torch
+
+import __graft_entry__ as entry
+from oracle import monarch_oracle as mo
+from paper_2505_18698_b200 import binding, workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-5, "f16": 1e-2, "bf16": 1e-2}
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    entry.build()
+    return binding.load_library()
+
+
+def rel_err(Y, ref):
+    Y = Y.reshape(-1, *Y.shape[-2:])
+    ref = ref.reshape(-1, *ref.shape[-2:])
+    return max(np.linalg.norm(Y[h] - ref[h]) / max(np.linalg.norm(ref[h]), 1e-300)
+               for h in range(Y.shape[0]))
+
+
+def gpu_forward(Q, K, V, dtype, b, T, path=binding.MA_PATH_AUTO, scale=None, use_ex=True):
+    Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))
+    if use_ex:
+        Yd = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, b, T, softmax_scale=scale, path=path)
+    else:
+        Yd = binding.monarch_attn_fwd(Qd, Kd, Vd, b, T)
+    torch.cuda.synchronize()
+    assert binding.monarch_attn_last_launch_count() >= 2
+    return Yd.float().cpu().numpy().astype(np.float64)
+
+
+def check(batch, heads, N, d, b, T, dtype, rank=0, s=0.0, seed=0, path=binding.MA_PATH_AUTO,
+          scale=None, use_ex=True, tol=None):
+    Q, K, V = wl.make_qkv(batch, heads, N, d, dtype, rank, s, seed)
+    Y = gpu_forward(Q, K, V, dtype, b, T, path, scale, use_ex)
+    ref = mo.monarch_attention(Q, K, V, b, T, scale)
+    assert np.isfinite(Y).all()
+    err = rel_err(Y, ref)
+    assert err <= (tol or TOL[dtype]), (err, batch, heads, N, d, b, T, dtype)
+    return err
+
+
+# ------------------------------------------------------------------ generic path, small shapes
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("N,b,d,T", [
+    (16, 4, 8, 1), (24, 6, 5, 2), (24, 4, 5, 3), (24, 2, 7, 2), (64, 8, 64, 2), (60, 12, 16, 2),
+    (256, 16, 64, 1), (256, 16, 72, 3), (210, 14, 64, 2), (384, 24, 64, 1), (384, 96, 64, 1),
+    (1024, 32, 64, 2), (2048, 32, 64, 2), (6, 6, 4, 2), (6, 1, 4, 2),
+])
+def test_generic_path_small_shapes(N, b, d, T, dtype):
+    check(1, 3, N, d, b, T, dtype, rank=min(4, d), s=1.0, seed=N + b + T,
+          path=binding.MA_PATH_GENERIC)
+
+
+@pytest.mark.parametrize("BH", [(1, 1), (3, 1), (37, 4), (149, 1)])
+def test_generic_path_many_heads(BH):
+    check(BH[0], BH[1], 64, 16, 8, 2, "f32", seed=5, path=binding.MA_PATH_GENERIC)
+
+
+def test_explicit_scale_and_default_entry_point():
+    check(2, 2, 64, 16, 8, 2, "f32", seed=9, scale=0.2, path=binding.MA_PATH_GENERIC)
+    check(2, 2, 64, 16, 8, 2, "f32", seed=9, use_ex=False)
+
+
+# ------------------------------------------------------------------ the five configurations
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5"])
+def test_benchmark_configurations_match_oracle(name):
+    w = wl.WORKLOADS[name]
+    Q, K, V = wl.make_workload_inputs(w)
+    Y = gpu_forward(Q, K, V, w.dtype, w.b, w.T, use_ex=False)     # the launch bench.py times
+    assert np.isfinite(Y).all()
+    ref = mo.monarch_attention(Q, K, V, w.b, w.T)
+    err = rel_err(Y, ref)
+    print(f"{name}: max rel Frobenius error {err:.3e}")
+    assert err <= TOL[w.dtype], (name, err)
+
+
+@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5"])
+def test_generic_path_on_configuration_shapes(name):
+    w = wl.WORKLOADS[name]
+    check(1, 2, w.N, w.d, w.b, w.T, w.dtype, w.rank, w.s, seed=100 + w.seed,
+          path=binding.MA_PATH_GENERIC)
+
+
+# ------------------------------------------------------------------ properties at any size
+@pytest.mark.parametrize("path", [binding.MA_PATH_GENERIC, binding.MA_PATH_AUTO])
+def test_constant_v_and_zero_q(path):
+    for (N, b, dtype) in [(256, 16, "f32"), (4096, 64, "bf16")]:
+        Q, K, V = wl.make_qkv(1, 2, N, 64, dtype, 4, 1.0, seed=3)
+        c = wl.round_to_dtype(np.linspace(-2, 2, 64, dtype=np.float32), dtype)
+        Vc = np.broadcast_to(c, V.shape).copy()
+        Y = gpu_forward(Q, K, Vc, dtype, b, 2, path)
+        assert np.abs(Y - Vc).max() <= (1e-5 if dtype == "f32" else 2e-2)
+        Y = gpu_forward(np.zeros_like(Q), K, V, dtype, b, 2, path)
+        mean = V.astype(np.float64).mean(axis=2, keepdims=True)
+        assert np.abs(Y - mean).max() <= (1e-5 if dtype == "f32" else 1e-2)
+
+
+def test_reruns_are_bit_identical_and_heads_are_independent():
+    for (N, b, dtype, heads) in [(256, 16, "f32", 4), (4096, 64, "bf16", 4)]:
+        Q, K, V = wl.make_qkv(1, heads, N, 64, dtype, 8, 1.5, seed=21)
+        Y1 = gpu_forward(Q, K, V, dtype, b, 2)
+        Y2 = gpu_forward(Q, K, V, dtype, b, 2)
+        assert np.array_equal(Y1, Y2)
+        perm = [2, 0, 3, 1]
+        Y3 = gpu_forward(Q[:, perm], K[:, perm], V[:, perm], dtype, b, 2)
+        assert np.array_equal(Y1[:, perm], Y3)
+
+
+@pytest.mark.parametrize("N,b,dtype", [(256, 16, "f16"), (1024, 32, "bf16"), (4096, 64, "bf16"),
+                                       (16384, 128, "bf16")])
+def test_stress_inputs_stay_finite(N, b, dtype):
+    """Un-normalised rank component (logit std ~ 90) and shared coefficients: not a parity gate."""
+    rng = np.random.Generator(np.random.Philox(77))
+    W = rng.standard_normal((8, 64), dtype=np.float32)
+    C = rng.standard_normal((1, 1, N, 8), dtype=np.float32)
+    Q = wl.round_to_dtype(rng.standard_normal((1, 1, N, 64), dtype=np.float32) + 2.0 * C @ W, dtype)
+    K = wl.round_to_dtype(rng.standard_normal((1, 1, N, 64), dtype=np.float32) + 2.0 * C @ W, dtype)
+    V = wl.round_to_dtype(rng.standard_normal((1, 1, N, 64), dtype=np.float32), dtype)
+    Y = gpu_forward(Q, K, V, dtype, b, 2)
+    assert np.isfinite(Y).all()
+    assert np.abs(Y).max() <= np.abs(V).max() * 1.02      # rows of M are convex weights
+
+
+def test_canaries_around_output_and_workspace():
+    w = wl.WORKLOADS["C4"]
+    Q, K, V = wl.make_qkv(1, 2, w.N, w.d, w.dtype, w.rank, w.s, seed=31)
+    Qd, Kd, Vd = (binding.to_device(x, w.dtype) for x in (Q, K, V))
+    n = Qd.numel()
+    pad = 4096
+    buf = torch.full((n + 2 * pad,), 7.0, dtype=Qd.dtype, device="cuda")
+    Y = buf[pad:pad + n].view_as(Qd)
+    need = binding.monarch_attn_workspace_bytes(1, 2, w.N, w.d, w.b, w.T, Qd.dtype)
+    wsbuf = torch.full((need + 2 * pad,), 0x5A, dtype=torch.uint8, device="cuda")
+    off = (-wsbuf.data_ptr()) % 256 + 256
+    ws = wsbuf[off:off + need]
+    binding.monarch_attn_fwd_ex(Qd, Kd, Vd, w.b, w.T, workspace=ws, Y=Y)
+    torch.cuda.synchronize()
+    assert (buf[:pad] == 7.0).all() and (buf[pad + n:] == 7.0).all()
+    assert (wsbuf[:off] == 0x5A).all() and (wsbuf[off + need:] == 0x5A).all()
+    assert binding.monarch_attn_device_status(ws) == 0
+    ref = mo.monarch_attention(Q, K, V, w.b, w.T)
+    assert rel_err(Y.float().cpu().numpy().astype(np.float64), ref) <= 1e-2
+
+
+def test_host_entry_point_matches_device_entry_point():
+    w = wl.WORKLOADS["C1"]
+    Q, K, V = wl.make_workload_inputs(w)
+    Qh, Kh, Vh = (torch.from_numpy(x).pin_memory() for x in (Q, K, V))
+    Yh = torch.empty_like(Qh).pin_memory()
+    binding.monarch_attn_fwd_host(Qh, Kh, Vh, Yh, w.b, w.T)
+    torch.cuda.synchronize()
+    Yd = binding.monarch_attn_fwd(Qh.cuda(), Kh.cuda(), Vh.cuda(), w.b, w.T)
+    assert torch.equal(Yd.cpu(), Yh)
+
+
+def test_unsupported_and_error_paths_on_device():
+    x = torch.zeros(1, 1, 256, 64, device="cuda")
+    with pytest.raises(binding.MonarchAttnError) as e:
+        binding.monarch_attn_fwd_ex(x, x, x, 16, 1, path=binding.MA_PATH_TENSOR)
+    assert e.value.code == 4
+    with pytest.raises(binding.MonarchAttnError) as e:
+        binding.monarch_attn_fwd(x, x, x, b=16, T=1, Y=x)
+    assert e.value.code == 5
+    with pytest.raises(binding.MonarchAttnError) as e:
+        binding.monarch_attn_fwd(x, x, x, b=15, T=1)
+    assert e.value.code == 2
