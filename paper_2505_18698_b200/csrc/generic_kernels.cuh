@@ -81,7 +81,8 @@ r_step_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
     } else {
       const float* a = aR + head_off + ((size_t)k * b + j) * d;
       for (int v = lane; v < d; v += 32) as[v] = a[v];
-      inv_c = 1.f / cR[(size_t)h * N + (size_t)k * b + j];
+      const float c = cR[(size_t)h * N + (size_t)k * b + j];
+      inv_c = c > 1e-30f ? 1.f / c : 0.f;   // c_R underflow: uniform row (Z_R = 0)
     }
     __syncwarp();
     const float f = scale * inv_c;
