@@ -43,7 +43,10 @@ typedef enum {
 typedef enum {
   MA_PATH_AUTO = 0,
   MA_PATH_GENERIC = 1, /* fp32 SIMT kernels, fp32 states; any dtype, any N = m*b that fits smem */
-  MA_PATH_TENSOR = 2   /* tcgen05/TMA kernels, 16-bit states; f16/bf16, d = 64, m = b in {64,128} */
+  MA_PATH_TENSOR = 2,  /* tcgen05/TMA kernels, 16-bit states; f16/bf16, d = 64, m = b in {64,128}:
+                          one persistent launch for all 2T half-steps */
+  MA_PATH_TENSOR_PHASED = 3, /* the same persistent kernel, one launch per half-step */
+  MA_PATH_TENSOR_BASIC = 4   /* one CTA per tile, one launch per half-step (no pipelining) */
 } ma_path;
 
 /* T-step MonarchAttention forward (Eq. 7-10 then Eq. 4) with scale = 1/sqrt(d).

@@ -10,6 +10,7 @@
 
 #include "generic_kernels.cuh"
 #include "tensor_path.cuh"
+#include "tensor_persistent.cuh"
 
 namespace ma {
 
@@ -134,14 +135,16 @@ static int resolve_path(const Problem& p, int path) {
     return -1;
   }
   if (path == MA_PATH_GENERIC) return generic_supported(p) ? path : -1;
-  if (path == MA_PATH_TENSOR)
+  if (path == MA_PATH_TENSOR || path == MA_PATH_TENSOR_PHASED || path == MA_PATH_TENSOR_BASIC)
     return tensor::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
   return -1;
 }
 
 static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
-  if (resolved == MA_PATH_TENSOR) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
+  if (resolved == MA_PATH_TENSOR_BASIC) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
+  if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_PHASED)
+    return tp::workspace_bytes(p.BH, p.N, p.T);
   return 0;
 }
 
@@ -179,7 +182,12 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   if (((uintptr_t)ws & 255) != 0) return MA_ERR_ALIGN;
   if (resolved == MA_PATH_GENERIC) return launch_generic(p, Q, K, V, Y, scale, ws, st);
   int launches = 0;
-  int rc = tensor::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.T, p.dtype, scale, ws, st, &launches);
+  int rc;
+  if (resolved == MA_PATH_TENSOR_BASIC)
+    rc = tensor::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.T, p.dtype, scale, ws, st, &launches);
+  else
+    rc = tp::launch(Q, K, V, Y, p.BH, p.N, p.b, p.T, p.dtype, scale, ws, st, &launches,
+                    resolved == MA_PATH_TENSOR ? 0 : 1);
   if (rc == MA_OK) g_last_launches = launches;
   return rc;
 }

@@ -1,0 +1,569 @@
+// Persistent, warp-specialised tensor-core kernel: all 2T half-steps of the forward pass in ONE
+// launch.  One CTA per SM walks a static list of 128-row tiles ordered half-step by half-step
+// (R1 of every head, L1 of every head, R2 ...).  A tile of half-step p of head h may start once
+// every tile of half-step p-1 of the same head has been stored; that is tracked with one counter
+// per (half-step, head) in the workspace.  Because the list is ordered and every CTA takes its tiles
+// in increasing order, each dependency points to a tile some resident CTA has already taken, so the
+// (bounded) waits cannot deadlock; with the phase-major order a dependency is almost a whole
+// half-step old when it is needed and the waits are normally free.
+//
+// Warp roles (352 threads):
+//   warp 0      TMA producer: dependency wait, then loads the tile's operands into three rings
+//               (E: operand released after MMA 1, L: operand released after MMA 2, V: V/y tile)
+//   warp 1      MMA issuer: scores S = A.B^T into TMEM (two accumulator stages), then, once the
+//               softmax group has written P to shared memory, the apply MMA into O
+//   warps 2-5   softmax group 0 (tiles 0, 2, 4, ... of this CTA): one thread per score row
+//   warps 6-9   softmax group 1 (tiles 1, 3, 5, ...)
+//   warp 10     store lanes (one per softmax group): TMA-store the staged rows, wait until they are
+//               in global memory, then bump the (half-step, head) counter
+// No role ever waits for another CTA while holding up work of an earlier tile of its own CTA: the
+// MMA issuer polls its two pending jobs (MMA 2 of the oldest tile, MMA 1 of the next) instead of
+// blocking on either, and completion is signalled by the store lanes, not by the softmax groups.
+// A softmax group reads S from TMEM (two passes: row max, then exp/sum), writes P (16-bit,
+// 128-byte swizzled) for MMA 2, later reads O from TMEM, normalises, stages the 16-bit rows in the
+// same buffer and one thread TMA-stores them with the strides that realise the permutation.
+#pragma once
+#include "tensor_path.cuh"
+
+namespace ma {
+namespace tp {
+
+using namespace ma::tensor;
+
+constexpr int kThreads = 352;
+constexpr int kRingE = 3, kRingL = 4, kRingV = 2;
+constexpr int kSlot = kTileBytes;   // 16 KB
+
+struct Lay {
+  static constexpr int E = 0;
+  static constexpr int L = E + kRingE * kSlot;
+  static constexpr int V = L + kRingL * kSlot;
+  static constexpr int P = V + kRingV * kSlot;          // 2 x 32 KB
+  static constexpr int Ones = P + 4 * kSlot;            // 2 KB
+  static constexpr int Vec = Ones + 2048;               // 2 x 128 floats
+  static constexpr int Bars = Vec + 1024;
+  static constexpr int Total = Bars + 256;
+};
+constexpr int kSmem = Lay::Total + 1024;
+
+struct __align__(8) Bars {
+  uint64_t fullE[kRingE], emptyE[kRingE];
+  uint64_t fullL[kRingL], emptyL[kRingL];
+  uint64_t fullV[kRingV], emptyV[kRingV];
+  uint64_t s_ready[2], p_ready[2], o_ready[2], o_free[2], stage_ready[2], stage_free[2];
+  uint32_t tmem_slot;
+  volatile int abort_flag;
+};
+
+struct Params {
+  CUtensorMap tmQ, tmK, tmV, tmAR, tmAL, tmY;    // 2D row views (loads)
+  CUtensorMap tmALs, tmYs;                       // 3D stores of aL / y (rows m apart)
+  CUtensorMap tmQs;                              // 3D strided view of Q (load)
+  CUtensorMap tmARs, tmOut;                      // 3D strided stores of aR / Y
+  float* cL;
+  float* cR;
+  int* status;
+  int* counters;       // [2T][BH] completed tiles
+  int m, BH, T;
+  int tiles_per_head, tiles_per_phase;
+  int g_begin, g_end;  // tile range of this launch
+  int check_deps;
+  float scale;
+};
+
+struct Tile {
+  int p, h, idx0;      // half-step, head, first k (R) or j (L) of the tile
+  bool isR, first, withV, final_;
+};
+__device__ __forceinline__ Tile decode(const Params& P, int g, int kTiles) {
+  Tile t;
+  t.p = g / P.tiles_per_phase;
+  const int local = g - t.p * P.tiles_per_phase;
+  t.h = local / P.tiles_per_head;
+  t.idx0 = (local - t.h * P.tiles_per_head) * kTiles;
+  t.isR = (t.p & 1) == 0;
+  t.first = t.p == 0;
+  t.withV = t.p == 2 * P.T - 2;
+  t.final_ = t.p == 2 * P.T - 1;
+  return t;
+}
+
+// Bounded wait.  A wait that runs out records where in the status word and raises the CTA's abort
+// flag; from then on every wait of the CTA returns at once, so all roles run through their
+// remaining (now meaningless) tiles without blocking, barriers stay matched, and the kernel ends.
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Bars* bars,
+                                              int* status, int where) {
+  const uint32_t addr = smem_u32(bar);
+  const long long t0 = clock64();
+  for (;;) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if (bars->abort_flag) return false;
+    if (clock64() - t0 > kWaitCycles) {
+      report_timeout(status, where);
+      bars->abort_flag = 1;
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void group_barrier(int id) {
+  asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
+}
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void tma_store_commit() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() {
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ float tmem_ld1(uint32_t taddr) {
+  uint32_t r;
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
+  return __uint_as_float(r);
+}
+
+// Bounded wait until every tile of half-step p-1 of head h has been stored.
+__device__ __forceinline__ void wait_dependency(const Params& P, const Tile& t, Bars* bars, int where) {
+  if (!P.check_deps || t.p == 0) return;
+  const int* ctr = P.counters + (t.p - 1) * P.BH + t.h;
+  if (ld_acquire(ctr) >= P.tiles_per_head) return;
+  const long long t0 = clock64();
+  while (ld_acquire(ctr) < P.tiles_per_head) {
+    __nanosleep(64);
+    if (bars->abort_flag) return;
+    if (clock64() - t0 > kWaitCycles) {
+      report_timeout(P.status, where);
+      bars->abort_flag = 1;
+      return;
+    }
+  }
+}
+
+template <typename T, int B>
+__global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_constant__ Params P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  Bars* bars = reinterpret_cast<Bars*>(smem + Lay::Bars);
+  constexpr int kTiles = Geo<B>::kTiles;
+  constexpr int FMT = Fmt<T>::code;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m = P.m;
+
+  if (tid == 0) {
+    for (int i = 0; i < kRingE; ++i) { mbar_init(&bars->fullE[i], 1); mbar_init(&bars->emptyE[i], 1); }
+    for (int i = 0; i < kRingL; ++i) { mbar_init(&bars->fullL[i], 1); mbar_init(&bars->emptyL[i], 1); }
+    for (int i = 0; i < kRingV; ++i) { mbar_init(&bars->fullV[i], 1); mbar_init(&bars->emptyV[i], 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars->s_ready[i], 1);
+      mbar_init(&bars->p_ready[i], 128);
+      mbar_init(&bars->o_ready[i], 1);
+      mbar_init(&bars->o_free[i], 128);
+      mbar_init(&bars->stage_ready[i], 128);
+      mbar_init(&bars->stage_free[i], 1);
+    }
+    bars->abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (tid < 128) {   // tile of ones for the column-sum MMA of the non-final L half-step
+    const uint32_t one2 = pack2<T>(1.f, 1.f);
+    *reinterpret_cast<uint4*>(smem + Lay::Ones + tid * 16) = make_uint4(one2, one2, one2, one2);
+  }
+  if (warp == 0) tmem_alloc(&bars->tmem_slot, 512);
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_slot;
+
+  const int first_g = P.g_begin + blockIdx.x;
+  const int stride_g = gridDim.x;
+  const int n_total = first_g < P.g_end ? (P.g_end - first_g + stride_g - 1) / stride_g : 0;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int nv = 0;
+      for (int n = 0; n < n_total; ++n) {
+        const Tile t = decode(P, first_g + n * stride_g, kTiles);
+        wait_dependency(P, t, bars, 10);
+        asm volatile("fence.proxy.async.global;" ::: "memory");
+        const int eE = n % kRingE, eL = n % kRingL;
+        wait_or_abort(&bars->emptyE[eE], ((n / kRingE) & 1) ^ 1, bars, P.status, 11);
+        wait_or_abort(&bars->emptyL[eL], ((n / kRingL) & 1) ^ 1, bars, P.status, 12);
+        uint8_t* sE = smem + Lay::E + eE * kSlot;
+        uint8_t* sL = smem + Lay::L + eL * kSlot;
+        const bool needV = t.isR ? t.withV : t.final_;
+        uint8_t* sV = nullptr;
+        int eV = 0;
+        if (needV) {
+          eV = nv % kRingV;
+          wait_or_abort(&bars->emptyV[eV], ((nv / kRingV) & 1) ^ 1, bars, P.status, 13);
+          sV = smem + Lay::V + eV * kSlot;
+          ++nv;
+        }
+        mbar_expect_tx(&bars->fullE[eE], kSlot);
+        mbar_expect_tx(&bars->fullL[eL], kSlot);
+        if (needV) mbar_expect_tx(&bars->fullV[eV], kSlot);
+        if (t.isR) {
+          const int row0 = (t.h * m + t.idx0) * B;
+          tma_load_2d(sE, t.first ? &P.tmQ : &P.tmAR, &bars->fullE[eE], 0, row0);
+          tma_load_2d(sL, &P.tmK, &bars->fullL[eL], 0, row0);
+          if (needV) tma_load_2d(sV, &P.tmV, &bars->fullV[eV], 0, row0);
+        } else {
+          const int row0 = (t.h * B + t.idx0) * m;
+          tma_load_2d(sE, &P.tmAL, &bars->fullE[eE], 0, row0);
+#pragma unroll
+          for (int tt = 0; tt < kTiles; ++tt)
+            tma_load_3d(sL + tt * (B * 128), &P.tmQs, &bars->fullL[eL], 0, t.idx0 + tt, t.h * m);
+          if (needV) tma_load_2d(sV, &P.tmY, &bars->fullV[eV], 0, row0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    // Two pending jobs are polled, never waited for: MMA 2 of the oldest unfinished tile (needs P
+    // from its softmax group) and MMA 1 of the next tile (needs its operands, which may depend on
+    // other CTAs).  Blocking on the second would hold up the first and could deadlock the grid.
+    if (lane == 0) {
+      const uint32_t sE0 = smem_u32(smem + Lay::E), sL0 = smem_u32(smem + Lay::L);
+      const uint32_t sV0 = smem_u32(smem + Lay::V), sP0 = smem_u32(smem + Lay::P);
+      const uint32_t sOnes = smem_u32(smem + Lay::Ones);
+      int i1 = 0, i2 = 0, nv = 0;
+      long long t0 = clock64();
+      bool force = false;
+      while (i2 < n_total) {
+        bool did = false;
+        if (i2 < i1) {
+          const Tile t = decode(P, first_g + i2 * stride_g, kTiles);
+          const int a = i2 & 1, q = i2 >> 1, eL = i2 % kRingL;
+          const bool needV = t.isR ? t.withV : t.final_;
+          const int eV = nv % kRingV;
+          if (force || (mbar_test(&bars->p_ready[a], q & 1) && mbar_test(&bars->o_free[a], (q & 1) ^ 1) &&
+                        (!needV || mbar_test(&bars->fullV[eV], (nv / kRingV) & 1)))) {
+            tc_fence_after();
+            const uint32_t sL = sL0 + eL * kSlot, sV = sV0 + eV * kSlot, sP = sP0 + a * 2 * kSlot;
+            const uint32_t tO = tmem + a * 256 + 128;
+            if (t.isR) {
+              // [aL | y] = P [K | V]; the V tile sits (sV - sL) bytes after the K tile
+              issue_apply<B, FMT>(tO, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
+            } else if (t.final_) {
+              issue_apply<B, FMT>(tO, sP, sV, 16, 1);
+            } else {
+              issue_transposed_apply<B, FMT>(tO, sP, sL, sOnes);
+            }
+            umma_commit(&bars->emptyL[eL]);
+            if (needV) { umma_commit(&bars->emptyV[eV]); ++nv; }
+            umma_commit(&bars->o_ready[a]);
+            ++i2;
+            did = true;
+          }
+        }
+        if (i1 < n_total && i1 < i2 + 2) {
+          const int eE = i1 % kRingE, eL = i1 % kRingL, a = i1 & 1;
+          if (force || (mbar_test(&bars->fullE[eE], (i1 / kRingE) & 1) &&
+                        mbar_test(&bars->fullL[eL], (i1 / kRingL) & 1))) {
+            const Tile t = decode(P, first_g + i1 * stride_g, kTiles);
+            tc_fence_after();
+            const uint32_t sE = sE0 + eE * kSlot, sL = sL0 + eL * kSlot;
+            // R: A = aR (E ring), B = K (L ring).  L: A = Qb (L ring), B = aL (E ring).
+            issue_scores<B, FMT>(tmem + a * 256, t.isR ? sE : sL, t.isR ? sL : sE);
+            umma_commit(&bars->emptyE[eE]);
+            umma_commit(&bars->s_ready[a]);
+            ++i1;
+            did = true;
+          }
+        }
+        if (did) {
+          t0 = clock64();
+        } else if (!force) {
+          if (bars->abort_flag) {
+            force = true;
+          } else if (clock64() - t0 > kWaitCycles) {
+            report_timeout(P.status, 20);
+            bars->abort_flag = 1;
+            force = true;
+          }
+        }
+      }
+    }
+  } else if (warp < 10) {
+    // ------------------------------------------------------------------ softmax groups
+    const int w = (warp - 2) >> 2;             // group = accumulator stage
+    const int tw = tid - 64 - w * 128;         // 0..127 inside the group
+    const int sub = warp & 3;                  // TMEM sub-partition this warp may access
+    const int t_row = sub * 32 + lane;         // TMEM lane = score row owned by this thread
+    const int tile = Geo<B>::tile(t_row), r = Geo<B>::row(t_row), srow = tile * B + r;
+    const uint32_t tS = tmem + w * 256 + ((uint32_t)(sub * 32) << 16);
+    const uint32_t tO = tS + 128;
+    uint8_t* sP = smem + Lay::P + w * 2 * kSlot;
+    float* cvec = reinterpret_cast<float*>(smem + Lay::Vec) + w * 128;
+    const int bar_id = 1 + w;
+
+    for (int n = w; n < n_total; n += 2) {
+      const Tile t = decode(P, first_g + n * stride_g, kTiles);
+      const int q = n >> 1;
+      wait_dependency(P, t, bars, 32);         // c_L / c_R of the previous half-step are final
+      float inv_c = 1.f;
+      size_t rrow = 0;
+      if (t.isR) {
+        rrow = (size_t)(t.h * m + t.idx0) * B + srow;       // [h][k][j]
+        if (!t.first) {
+          const float c = __ldcg(P.cR + rrow);
+          inv_c = c > 1e-30f ? 1.f / c : 0.f;
+        }
+      } else {
+        const int tile_e = tw / B, k_e = tw - tile_e * B;     // cL column(s) j0 (+1)
+        cvec[tw] = __ldcg(P.cL + ((size_t)t.h * m + k_e) * B + t.idx0 + tile_e) * kLog2e;
+      }
+      wait_or_abort(&bars->s_ready[w], q & 1, bars, P.status, 30);
+      if (!t.isR) group_barrier(bar_id);       // publish cvec
+      tc_fence_after();
+
+      float mx = -INFINITY, sum = 0.f, sz = 0.f, f, inv_s;
+      if (t.isR) {
+        f = P.scale * inv_c * kLog2e;
+#pragma unroll
+        for (int c = 0; c < B / 32; ++c) {
+          float s[32];
+          tmem_ld32(tS + 32 * c, s);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, s[i]);
+        }
+        const float off = -mx * f;
+        // P and the store staging share a buffer: the previous tile's rows must have been read
+        wait_or_abort(&bars->stage_free[w], (q & 1) ^ 1, bars, P.status, 33);
+#pragma unroll
+        for (int c = 0; c < B / 32; ++c) {
+          float s[32];
+          tmem_ld32(tS + 32 * c, s);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float p = fast_exp2(fmaf(s[i], f, off));
+            sz = fmaf(p, s[i], sz);
+            sum += p;
+            s[i] = p;
+          }
+          store_row32<T>(sP, srow, 32 * c, s, 1.f);
+        }
+        inv_s = 1.f / sum;
+      } else {
+        f = P.scale * kLog2e;
+        const float* cv = cvec + tile * B;
+#pragma unroll
+        for (int c = 0; c < B / 32; ++c) {
+          float s[32];
+          tmem_ld32(tS + 32 * c, s);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaf(s[i], f, -cv[32 * c + i]));
+        }
+        if (t.final_) {
+          wait_or_abort(&bars->stage_free[w], (q & 1) ^ 1, bars, P.status, 33);
+#pragma unroll
+          for (int c = 0; c < B / 32; ++c) {
+            float s[32];
+            tmem_ld32(tS + 32 * c, s);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              s[i] = fast_exp2(fmaf(s[i], f, -cv[32 * c + i]) - mx);
+              sum += s[i];
+            }
+            store_row32<T>(sP, srow, 32 * c, s, 1.f);
+          }
+          inv_s = 1.f / sum;
+        } else {
+          // P must be normalised before MMA 2 (it contracts over rows): one more pass
+#pragma unroll
+          for (int c = 0; c < B / 32; ++c) {
+            float s[32];
+            tmem_ld32(tS + 32 * c, s);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sum += fast_exp2(fmaf(s[i], f, -cv[32 * c + i]) - mx);
+          }
+          inv_s = 1.f / sum;
+          wait_or_abort(&bars->stage_free[w], (q & 1) ^ 1, bars, P.status, 33);
+#pragma unroll
+          for (int c = 0; c < B / 32; ++c) {
+            float s[32];
+            tmem_ld32(tS + 32 * c, s);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) s[i] = fast_exp2(fmaf(s[i], f, -cv[32 * c + i]) - mx);
+            store_row32<T>(sP, srow, 32 * c, s, inv_s);
+          }
+        }
+      }
+      fence_proxy_async();
+      tc_fence_before();
+      mbar_arrive(&bars->p_ready[w]);
+      if (t.isR) P.cL[rrow] = kLn2 * (f * (sz * inv_s - mx) - fast_log2(sum));
+
+      wait_or_abort(&bars->o_ready[w], q & 1, bars, P.status, 31);
+      tc_fence_after();
+      const int ncol = t.isR ? (t.withV ? 128 : 64) : 64;
+      const float mul = (t.isR || t.final_) ? inv_s : 1.f;
+      for (int c = 0; c < ncol / 32; ++c) {
+        float o[32];
+        tmem_ld32(tO + 32 * c, o);
+        tmem_ld_wait();
+        store_row32<T>(sP, srow, 32 * c, o, mul);
+      }
+      if (!t.isR && !t.final_) {
+        const float c1 = tmem_ld1(tO + 64);
+        tmem_ld_wait();
+        P.cR[((size_t)t.h * m + r) * B + t.idx0 + tile] = c1;
+      }
+      tc_fence_before();
+      mbar_arrive(&bars->o_free[w]);
+      fence_proxy_async();
+      mbar_arrive(&bars->stage_ready[w]);
+    }
+  } else {
+    // ------------------------------------------------------------------ store lanes
+    if (lane < 2) {
+      const int w = lane;
+      const uint8_t* sP = smem + Lay::P + w * 2 * kSlot;
+      for (int n = w; n < n_total; n += 2) {
+        const Tile t = decode(P, first_g + n * stride_g, kTiles);
+        const int q = n >> 1;
+        wait_or_abort(&bars->stage_ready[w], q & 1, bars, P.status, 40);
+#pragma unroll
+        for (int tt = 0; tt < kTiles; ++tt) {
+          const uint8_t* src = sP + tt * (B * 128);
+          if (t.isR) {
+            tma_store_3d(&P.tmALs, src, 0, t.idx0 + tt, t.h * B);
+            if (t.withV) tma_store_3d(&P.tmYs, src + kSlot, 0, t.idx0 + tt, t.h * B);
+          } else {
+            tma_store_3d(t.final_ ? &P.tmOut : &P.tmARs, src, 0, t.idx0 + tt, t.h * m);
+          }
+        }
+        tma_store_commit();
+        tma_store_wait_read();
+        mbar_arrive(&bars->stage_free[w]);
+        tma_store_wait_all();                 // rows (and the group's c_L / c_R) are in global memory
+        asm volatile("fence.proxy.async.global;" ::: "memory");
+        __threadfence();
+        atomicAdd(P.counters + t.p * P.BH + t.h, 1);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (bars->abort_flag) {
+    // give copies still in flight time to land before shared and tensor memory are released
+    const long long t0 = clock64();
+    while (clock64() - t0 < 200000) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+// ------------------------------------------------------------------------------------ host side
+inline size_t counters_bytes(int BH, int T) {
+  return ((size_t)2 * T * BH * sizeof(int) + 255) / 256 * 256;
+}
+inline size_t workspace_bytes(int BH, int N, int T) {
+  return ws_layout(nullptr, BH, N).bytes + counters_bytes(BH, T);
+}
+
+template <typename T, int B>
+inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int T_steps,
+                    int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode) {
+  const Ws w = ws_layout(ws, BH, N);
+  int* counters = (int*)((char*)ws + w.bytes);
+  const int m = N / B;
+  const uint64_t rows = (uint64_t)BH * N;
+  Params P;
+  bool ok = make_map_rows(&P.tmQ, dtype, (void*)Q, rows) && make_map_rows(&P.tmK, dtype, (void*)K, rows) &&
+            make_map_rows(&P.tmV, dtype, (void*)V, rows) && make_map_rows(&P.tmAR, dtype, w.aR, rows) &&
+            make_map_rows(&P.tmAL, dtype, w.aL, rows) && make_map_rows(&P.tmY, dtype, w.y, rows) &&
+            make_map_strided(&P.tmALs, dtype, w.aL, m, (uint64_t)BH * B, B) &&
+            make_map_strided(&P.tmYs, dtype, w.y, m, (uint64_t)BH * B, B) &&
+            make_map_strided(&P.tmQs, dtype, (void*)Q, B, (uint64_t)BH * m, B) &&
+            make_map_strided(&P.tmARs, dtype, w.aR, B, (uint64_t)BH * m, B) &&
+            make_map_strided(&P.tmOut, dtype, Y, B, (uint64_t)BH * m, B);
+  if (!ok) return 7;
+  P.cL = w.cL; P.cR = w.cR; P.status = w.status; P.counters = counters;
+  P.m = m; P.BH = BH; P.T = T_steps;
+  P.tiles_per_head = m / Geo<B>::kTiles;
+  P.tiles_per_phase = BH * P.tiles_per_head;
+  P.scale = scale;
+  if (cudaMemsetAsync(ws, 0, kWsStatusBytes, st) != cudaSuccess) return 7;
+  if (cudaMemsetAsync(counters, 0, counters_bytes(BH, T_steps), st) != cudaSuccess) return 7;
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 7;
+  }
+  const void* fn = (const void*)monarch_persistent<T, B>;
+  if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
+    return 7;
+  const int total = 2 * T_steps * P.tiles_per_phase;
+  int n = 0;
+  if (mode == 0) {          // one launch, dependencies tracked by counters
+    P.g_begin = 0; P.g_end = total; P.check_deps = 1;
+    const int grid = total < num_sms ? total : num_sms;
+    monarch_persistent<T, B><<<grid, kThreads, kSmem, st>>>(P);
+    n = 1;
+  } else {                  // one launch per half-step (stream order is the dependency)
+    P.check_deps = 0;
+    for (int p = 0; p < 2 * T_steps; ++p) {
+      P.g_begin = p * P.tiles_per_phase; P.g_end = P.g_begin + P.tiles_per_phase;
+      const int grid = P.tiles_per_phase < num_sms ? P.tiles_per_phase : num_sms;
+      monarch_persistent<T, B><<<grid, kThreads, kSmem, st>>>(P);
+      ++n;
+    }
+  }
+  if (cudaGetLastError() != cudaSuccess) return 7;
+  *launches = n;
+  return 0;
+}
+
+inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int b, int T,
+                  int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode) {
+  if (dtype == 1) {
+    if (b == 128) return launch_t<__half, 128>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode);
+    return launch_t<__half, 64>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode);
+  }
+  if (b == 128)
+    return launch_t<__nv_bfloat16, 128>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode);
+  return launch_t<__nv_bfloat16, 64>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode);
+}
+
+}  // namespace tp
+}  // namespace ma

@@ -36,7 +36,7 @@ def gpu_forward(Q, K, V, dtype, b, T, path=binding.MA_PATH_AUTO, scale=None, use
     else:
         Yd = binding.monarch_attn_fwd(Qd, Kd, Vd, b, T)
     torch.cuda.synchronize()
-    assert binding.monarch_attn_last_launch_count() >= 2
+    assert binding.monarch_attn_last_launch_count() >= 1
     return Yd.float().cpu().numpy().astype(np.float64)
 
 
@@ -91,6 +91,46 @@ def test_generic_path_on_configuration_shapes(name):
     w = wl.WORKLOADS[name]
     check(1, 2, w.N, w.d, w.b, w.T, w.dtype, w.rank, w.s, seed=100 + w.seed,
           path=binding.MA_PATH_GENERIC)
+
+
+# ------------------------------------------------------------------ tensor-core paths
+TENSOR_PATHS = [binding.MA_PATH_TENSOR, binding.MA_PATH_TENSOR_PHASED, binding.MA_PATH_TENSOR_BASIC]
+
+
+@pytest.mark.parametrize("path", TENSOR_PATHS)
+@pytest.mark.parametrize("N,b,T,dtype,batch,heads", [
+    (4096, 64, 1, "bf16", 1, 1), (4096, 64, 2, "f16", 1, 3), (4096, 64, 3, "bf16", 2, 2),
+    (16384, 128, 1, "f16", 1, 1), (16384, 128, 2, "bf16", 1, 3), (16384, 128, 3, "bf16", 1, 2),
+    (4096, 64, 2, "bf16", 1, 7),       # 224 tiles per half-step: ragged tail over 148 CTAs
+])
+def test_tensor_paths_match_oracle(N, b, T, dtype, batch, heads, path):
+    check(batch, heads, N, 64, b, T, dtype, rank=16, s=1.5, seed=N + T + heads, path=path)
+
+
+def test_tensor_paths_agree_bit_for_bit_between_launch_modes():
+    """One persistent launch with dependency counters computes exactly what one launch per
+    half-step computes (same kernel, same tile order inside a half-step)."""
+    Q, K, V = wl.make_qkv(1, 5, 4096, 64, "bf16", 16, 1.5, seed=41)
+    a = gpu_forward(Q, K, V, "bf16", 64, 3, binding.MA_PATH_TENSOR)
+    b_ = gpu_forward(Q, K, V, "bf16", 64, 3, binding.MA_PATH_TENSOR_PHASED)
+    assert np.array_equal(a, b_)
+
+
+def test_persistent_kernel_repeated_calls_share_workspace():
+    """Counters and status are re-armed by every call."""
+    w = wl.WORKLOADS["C5"]
+    Q, K, V = wl.make_qkv(1, 2, w.N, w.d, w.dtype, w.rank, w.s, seed=51)
+    Qd, Kd, Vd = (binding.to_device(x, w.dtype) for x in (Q, K, V))
+    need = binding.monarch_attn_workspace_bytes(1, 2, w.N, w.d, w.b, w.T, Qd.dtype)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    outs = []
+    for _ in range(3):
+        outs.append(binding.monarch_attn_fwd_ex(Qd, Kd, Vd, w.b, w.T, workspace=ws).clone())
+    torch.cuda.synchronize()
+    assert binding.monarch_attn_device_status(ws) == 0
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+    ref = mo.monarch_attention(Q, K, V, w.b, w.T)
+    assert rel_err(outs[0].float().cpu().numpy().astype(np.float64), ref) <= 1e-2
 
 
 # ------------------------------------------------------------------ properties at any size
