@@ -86,6 +86,14 @@ int monarch_attn_device_status(const void* workspace, void* stream);
 /* Number of kernel launches the last successful call on this host thread enqueued. */
 int monarch_attn_last_launch_count(void);
 
+/* Profiling aid for the persistent tensor path.  With a DEVICE buffer of at least 4*64*8 int64
+ * set, CTAs 0-3 of later MA_PATH_TENSOR / MA_PATH_TENSOR_PHASED launches write SM-clock stamps
+ * [cta][tile][event] for their first 64 tiles; events: 0 operands requested, 1 score MMA issued,
+ * 2 softmax group sees the scores, 3 P written, 4 apply MMA issued, 5 softmax group sees O,
+ * 6 rows staged, 7 rows stored and signalled.  NULL switches it off (the default).  Process-wide;
+ * the buffer stays owned by the caller. */
+int monarch_attn_set_trace_buffer(void* device_buffer, size_t bytes);
+
 /* Static, NUL-terminated description of an ma_status code. */
 const char* monarch_attn_status_string(int status);
 

@@ -60,6 +60,8 @@ def load_library(path: str = LIB_PATH):
     lib.monarch_attn_device_status.restype = i
     lib.monarch_attn_last_launch_count.argtypes = []
     lib.monarch_attn_last_launch_count.restype = i
+    lib.monarch_attn_set_trace_buffer.argtypes = [vp, sz]
+    lib.monarch_attn_set_trace_buffer.restype = i
     lib.monarch_attn_status_string.argtypes = [i]
     lib.monarch_attn_status_string.restype = ctypes.c_char_p
     _lib = lib
@@ -156,6 +158,15 @@ def monarch_attn_device_status(workspace=None, stream=None) -> int:
 
 def monarch_attn_last_launch_count() -> int:
     return int(load_library().monarch_attn_last_launch_count())
+
+
+def monarch_attn_set_trace_buffer(buf=None):
+    """buf: int64 CUDA tensor with >= 4*64*8 elements, or None to switch tracing off."""
+    lib = load_library()
+    if buf is None:
+        _check(lib.monarch_attn_set_trace_buffer(None, 0))
+    else:
+        _check(lib.monarch_attn_set_trace_buffer(buf.data_ptr(), buf.numel() * buf.element_size()))
 
 
 def torch_dtype(name: str) -> torch.dtype:

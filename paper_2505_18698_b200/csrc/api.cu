@@ -296,6 +296,12 @@ int monarch_attn_device_status(const void* workspace, void* stream) {
 
 int monarch_attn_last_launch_count(void) { return g_last_launches; }
 
+int monarch_attn_set_trace_buffer(void* device_buffer, size_t bytes) {
+  if (device_buffer != nullptr && bytes < (size_t)4 * 64 * 8 * sizeof(long long)) return MA_ERR_WORKSPACE;
+  tp::trace_buffer() = (long long*)device_buffer;
+  return MA_OK;
+}
+
 const char* monarch_attn_status_string(int status) {
   switch (status) {
     case MA_OK: return "ok";

@@ -128,6 +128,31 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t 
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// Same with the accumulate flag known at compile time (no predicate register to set up).
+template <bool ACC>
+__device__ __forceinline__ void umma_c(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                       uint32_t idesc) {
+  if (ACC)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 1, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc)
+        : "memory");
+  else
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc)
+        : "memory");
+}
+// One lane of a fully active warp (lets the compiler keep MMA operands in uniform registers).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
                    smem_u32(bar))
@@ -199,6 +224,37 @@ template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, fl
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// Packed fp32 pairs (sm_100 f32x2 instructions: one issue slot for two lanes of work).
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "mov.b64 rc, {%6, %7};\n\tfma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+  return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+__device__ __forceinline__ float2 fmul2(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 // Writes 32 consecutive columns [col0, col0+32) of row `srow` of a [chunks][128][64] 16-bit tile
 // with 128-byte swizzled rows (the layout TMA produces and the MMA descriptors describe).
 template <typename T>
@@ -206,13 +262,33 @@ __device__ __forceinline__ void store_row32(uint8_t* tile, int srow, int col0, c
                                             float mul) {
   uint8_t* base = tile + (col0 >> 6) * kTileBytes + srow * 128;
   const int c0 = (col0 & 63) >> 3;
+  const float2 m2 = make_float2(mul, mul);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const float2 a = fmul2(make_float2(v[8 * c + 0], v[8 * c + 1]), m2);
+    const float2 b = fmul2(make_float2(v[8 * c + 2], v[8 * c + 3]), m2);
+    const float2 cc = fmul2(make_float2(v[8 * c + 4], v[8 * c + 5]), m2);
+    const float2 d = fmul2(make_float2(v[8 * c + 6], v[8 * c + 7]), m2);
+    uint4 q;
+    q.x = pack2<T>(a.x, a.y);
+    q.y = pack2<T>(b.x, b.y);
+    q.z = pack2<T>(cc.x, cc.y);
+    q.w = pack2<T>(d.x, d.y);
+    *reinterpret_cast<uint4*>(base + (((c0 + c) ^ (srow & 7)) << 4)) = q;
+  }
+}
+// Same without scaling.
+template <typename T>
+__device__ __forceinline__ void store_row32(uint8_t* tile, int srow, int col0, const float* v) {
+  uint8_t* base = tile + (col0 >> 6) * kTileBytes + srow * 128;
+  const int c0 = (col0 & 63) >> 3;
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     uint4 q;
-    q.x = pack2<T>(v[8 * c + 0] * mul, v[8 * c + 1] * mul);
-    q.y = pack2<T>(v[8 * c + 2] * mul, v[8 * c + 3] * mul);
-    q.z = pack2<T>(v[8 * c + 4] * mul, v[8 * c + 5] * mul);
-    q.w = pack2<T>(v[8 * c + 6] * mul, v[8 * c + 7] * mul);
+    q.x = pack2<T>(v[8 * c + 0], v[8 * c + 1]);
+    q.y = pack2<T>(v[8 * c + 2], v[8 * c + 3]);
+    q.z = pack2<T>(v[8 * c + 4], v[8 * c + 5]);
+    q.w = pack2<T>(v[8 * c + 6], v[8 * c + 7]);
     *reinterpret_cast<uint4*>(base + (((c0 + c) ^ (srow & 7)) << 4)) = q;
   }
 }
@@ -245,8 +321,10 @@ __device__ __forceinline__ void issue_scores(uint32_t tmem_s, uint32_t sA, uint3
     const uint64_t da = smem_desc(sA + t * (B * 128), 16, 1024);
     const uint64_t db = smem_desc(sB + t * (B * 128), 16, 1024);
 #pragma unroll
-    for (int ks = 0; ks < kD / 16; ++ks)
-      umma(tmem_s + ((uint32_t)(t * 16) << 16), da + 2 * ks, db + 2 * ks, idesc, ks > 0);
+    for (int ks = 0; ks < kD / 16; ++ks) {
+      if (ks == 0) umma_c<false>(tmem_s + ((uint32_t)(t * 16) << 16), da, db, idesc);
+      else umma_c<true>(tmem_s + ((uint32_t)(t * 16) << 16), da + 2 * ks, db + 2 * ks, idesc);
+    }
   }
 }
 
@@ -262,8 +340,12 @@ __device__ __forceinline__ void issue_apply(uint32_t tmem_o, uint32_t sP, uint32
     for (int ks = 0; ks < B / 16; ++ks) {
       const uint32_t pa = sP + (ks >> 2) * kTileBytes + t * (B * 128) + (ks & 3) * 32;
       const uint32_t xb = sX0 + t * (B * 128) + ks * 2048;
-      umma(tmem_o + ((uint32_t)(t * 16) << 16), smem_desc(pa, 16, 1024),
-           smem_desc(xb, x_chunk_stride, 1024), idesc, ks > 0);
+      if (ks == 0)
+        umma_c<false>(tmem_o + ((uint32_t)(t * 16) << 16), smem_desc(pa, 16, 1024),
+                      smem_desc(xb, x_chunk_stride, 1024), idesc);
+      else
+        umma_c<true>(tmem_o + ((uint32_t)(t * 16) << 16), smem_desc(pa, 16, 1024),
+                     smem_desc(xb, x_chunk_stride, 1024), idesc);
     }
   }
 }
@@ -283,8 +365,13 @@ __device__ __forceinline__ void issue_transposed_apply(uint32_t tmem_o, uint32_t
     for (int ks = 0; ks < B / 16; ++ks) {
       const uint64_t da = smem_desc(sP + t * (B * 128) + ks * 2048, kTileBytes, 1024);
       const uint64_t db = smem_desc(sX + t * (B * 128) + ks * 2048, 16, 1024);
-      umma(d, da, db, idesc, ks > 0);
-      umma(d + 64, da, ones, idesc1, ks > 0);
+      if (ks == 0) {
+        umma_c<false>(d, da, db, idesc);
+        umma_c<false>(d + 64, da, ones, idesc1);
+      } else {
+        umma_c<true>(d, da, db, idesc);
+        umma_c<true>(d + 64, da, ones, idesc1);
+      }
     }
   }
 }
@@ -392,7 +479,7 @@ r_step_tc(const __grid_constant__ CUtensorMap tmA,      // aR (or Q when FIRST):
     }
 #pragma unroll
     for (int c = 0; c < B / 32; ++c)
-      store_row32<T>(smem + SmemLayout::P, srow, 32 * c, s + 32 * c, 1.f);
+      store_row32<T>(smem + SmemLayout::P, srow, 32 * c, s + 32 * c);
     const float inv_s = 1.f / sum;
     cL[(size_t)row0 + srow] = kLn2 * (sz * inv_s - mx - fast_log2(sum));
     fence_proxy_async();

@@ -7,15 +7,17 @@
 // (bounded) waits cannot deadlock; with the phase-major order a dependency is almost a whole
 // half-step old when it is needed and the waits are normally free.
 //
-// Warp roles (352 threads):
-//   warp 0      TMA producer: dependency wait, then loads the tile's operands into three rings
+// Warp roles (384 threads):
+//   warp 0      TMA producer (one thread, polling, never blocking): checks the tile's dependency
+//               counter (fetched one tile ahead) and loads its operands into three rings
 //               (E: operand released after MMA 1, L: operand released after MMA 2, V: V/y tile)
 //   warp 1      MMA issuer: scores S = A.B^T into TMEM (two accumulator stages), then, once the
 //               softmax group has written P to shared memory, the apply MMA into O
 //   warps 2-5   softmax group 0 (tiles 0, 2, 4, ... of this CTA): one thread per score row
 //   warps 6-9   softmax group 1 (tiles 1, 3, 5, ...)
-//   warp 10     store lanes (one per softmax group): TMA-store the staged rows, wait until they are
-//               in global memory, then bump the (half-step, head) counter
+//   warps 10,11 store threads (one per softmax group, in warps of their own because a suspended
+//               mbarrier wait suspends the whole warp): TMA-store the staged rows, wait until
+//               they are in global memory, then bump the (half-step, head) counter
 // No role ever waits for another CTA while holding up work of an earlier tile of its own CTA: the
 // MMA issuer polls its two pending jobs (MMA 2 of the oldest tile, MMA 1 of the next) instead of
 // blocking on either, and completion is signalled by the store lanes, not by the softmax groups.
@@ -30,8 +32,8 @@ namespace tp {
 
 using namespace ma::tensor;
 
-constexpr int kThreads = 352;
-constexpr int kRingE = 3, kRingL = 4, kRingV = 2;
+constexpr int kThreads = 384;
+constexpr int kRingE = 2, kRingL = 4, kRingV = 3;
 constexpr int kSlot = kTileBytes;   // 16 KB
 
 struct Lay {
@@ -40,8 +42,8 @@ struct Lay {
   static constexpr int V = L + kRingL * kSlot;
   static constexpr int P = V + kRingV * kSlot;          // 2 x 32 KB
   static constexpr int Ones = P + 4 * kSlot;            // 2 KB
-  static constexpr int Vec = Ones + 2048;               // 2 x 128 floats
-  static constexpr int Bars = Vec + 1024;
+  static constexpr int Vec = Ones + 2048;               // kRingL x 128 floats (c_R / c_L)
+  static constexpr int Bars = Vec + kRingL * 512;
   static constexpr int Total = Bars + 256;
 };
 constexpr int kSmem = Lay::Total + 1024;
@@ -64,6 +66,7 @@ struct Params {
   float* cR;
   int* status;
   int* counters;       // [2T][BH] completed tiles
+  long long* trace;    // optional: clock64 stamps [4 CTAs][64 tiles][8 events] (profiling aid)
   int m, BH, T;
   int tiles_per_head, tiles_per_phase;
   int g_begin, g_end;  // tile range of this launch
@@ -75,18 +78,33 @@ struct Tile {
   int p, h, idx0;      // half-step, head, first k (R) or j (L) of the tile
   bool isR, first, withV, final_;
 };
-__device__ __forceinline__ Tile decode(const Params& P, int g, int kTiles) {
-  Tile t;
-  t.p = g / P.tiles_per_phase;
-  const int local = g - t.p * P.tiles_per_phase;
-  t.h = local / P.tiles_per_head;
-  t.idx0 = (local - t.h * P.tiles_per_head) * kTiles;
-  t.isR = (t.p & 1) == 0;
-  t.first = t.p == 0;
-  t.withV = t.p == 2 * P.T - 2;
-  t.final_ = t.p == 2 * P.T - 1;
-  return t;
-}
+// Walks the tiles g0, g0 + step, g0 + 2 step, ... of one role without integer divisions
+// (tiles_per_head is a power of two on this path).
+struct TileIter {
+  int p, local, step, tpp, tph_shift, tph_mask, kTiles, lastR;
+  __device__ __forceinline__ TileIter(const Params& P, int g0, int step_, int kTiles_)
+      : step(step_), tpp(P.tiles_per_phase), kTiles(kTiles_), lastR(2 * P.T - 2) {
+    p = g0 / tpp;
+    local = g0 - p * tpp;
+    tph_shift = 31 - __clz(P.tiles_per_head);
+    tph_mask = P.tiles_per_head - 1;
+  }
+  __device__ __forceinline__ Tile get() const {
+    Tile t;
+    t.p = p;
+    t.h = local >> tph_shift;
+    t.idx0 = (local & tph_mask) * kTiles;
+    t.isR = (p & 1) == 0;
+    t.first = p == 0;
+    t.withV = p == lastR;
+    t.final_ = p == lastR + 1;
+    return t;
+  }
+  __device__ __forceinline__ void next() {
+    local += step;
+    while (local >= tpp) { local -= tpp; ++p; }
+  }
+};
 
 // Bounded wait.  A wait that runs out records where in the status word and raises the CTA's abort
 // flag; from then on every wait of the CTA returns at once, so all roles run through their
@@ -124,6 +142,11 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
       : "memory");
   return done != 0;
 }
+// Profiling aid: CTAs 0-3 stamp eight pipeline events of their first 64 tiles.
+__device__ __forceinline__ void stamp(const Params& P, int n, int ev) {
+  if (P.trace != nullptr && blockIdx.x < 4 && n < 64)
+    P.trace[((size_t)blockIdx.x * 64 + n) * 8 + ev] = clock64();
+}
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -144,27 +167,19 @@ __device__ __forceinline__ void tma_store_wait_read() {
 __device__ __forceinline__ void tma_store_wait_all() {
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
+// 1-D bulk copy global -> shared (16-byte aligned, size a multiple of 16), completes on `bar`.
+__device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_t bytes,
+                                             uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst)),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
 __device__ __forceinline__ float tmem_ld1(uint32_t taddr) {
   uint32_t r;
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
   return __uint_as_float(r);
-}
-
-// Bounded wait until every tile of half-step p-1 of head h has been stored.
-__device__ __forceinline__ void wait_dependency(const Params& P, const Tile& t, Bars* bars, int where) {
-  if (!P.check_deps || t.p == 0) return;
-  const int* ctr = P.counters + (t.p - 1) * P.BH + t.h;
-  if (ld_acquire(ctr) >= P.tiles_per_head) return;
-  const long long t0 = clock64();
-  while (ld_acquire(ctr) < P.tiles_per_head) {
-    __nanosleep(64);
-    if (bars->abort_flag) return;
-    if (clock64() - t0 > kWaitCycles) {
-      report_timeout(P.status, where);
-      bars->abort_flag = 1;
-      return;
-    }
-  }
 }
 
 template <typename T, int B>
@@ -211,40 +226,84 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int nv = 0;
-      for (int n = 0; n < n_total; ++n) {
-        const Tile t = decode(P, first_g + n * stride_g, kTiles);
-        wait_dependency(P, t, bars, 10);
-        asm volatile("fence.proxy.async.global;" ::: "memory");
-        const int eE = n % kRingE, eL = n % kRingL;
-        wait_or_abort(&bars->emptyE[eE], ((n / kRingE) & 1) ^ 1, bars, P.status, 11);
-        wait_or_abort(&bars->emptyL[eL], ((n / kRingL) & 1) ^ 1, bars, P.status, 12);
-        uint8_t* sE = smem + Lay::E + eE * kSlot;
-        uint8_t* sL = smem + Lay::L + eL * kSlot;
-        const bool needV = t.isR ? t.withV : t.final_;
-        uint8_t* sV = nullptr;
-        int eV = 0;
-        if (needV) {
-          eV = nv % kRingV;
-          wait_or_abort(&bars->emptyV[eV], ((nv / kRingV) & 1) ^ 1, bars, P.status, 13);
-          sV = smem + Lay::V + eV * kSlot;
-          ++nv;
-        }
-        mbar_expect_tx(&bars->fullE[eE], kSlot);
-        mbar_expect_tx(&bars->fullL[eL], kSlot);
-        if (needV) mbar_expect_tx(&bars->fullV[eV], kSlot);
-        if (t.isR) {
-          const int row0 = (t.h * m + t.idx0) * B;
-          tma_load_2d(sE, t.first ? &P.tmQ : &P.tmAR, &bars->fullE[eE], 0, row0);
-          tma_load_2d(sL, &P.tmK, &bars->fullL[eL], 0, row0);
-          if (needV) tma_load_2d(sV, &P.tmV, &bars->fullV[eV], 0, row0);
-        } else {
-          const int row0 = (t.h * B + t.idx0) * m;
-          tma_load_2d(sE, &P.tmAL, &bars->fullE[eE], 0, row0);
+      const bool deps = P.check_deps != 0;
+      auto counter_of = [&](const Tile& t) { return P.counters + (t.p - 1) * P.BH + t.h; };
+      auto needs_v = [&](const Tile& t) { return t.isR ? t.withV : t.final_; };
+      int nE = 0, nVt = 0, nv = 0;                 // next tile for E/L, next tile to scan for V
+      TileIter itE(P, first_g, stride_g, kTiles), itV(P, first_g, stride_g, kTiles);
+      while (nVt < n_total && !needs_v(itV.get())) { ++nVt; itV.next(); }
+      // dependency counters are read one step ahead so their latency is off the critical path
+      int ctrE = 0, ctrV = 0;
+      if (deps && nE < n_total && itE.get().p > 0) ctrE = ld_acquire(counter_of(itE.get()));
+      if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
+      long long t0 = clock64();
+      bool force = false;
+      while (nE < n_total || nVt < n_total) {
+        bool did = false;
+        if (nE < n_total) {
+          const Tile t = itE.get();
+          const int eE = nE % kRingE, eL = nE % kRingL;
+          bool ok = force || !deps || t.p == 0 || ctrE >= P.tiles_per_head;
+          if (!ok) { ctrE = ld_acquire(counter_of(t)); ok = ctrE >= P.tiles_per_head; }
+          if (ok && (force || (mbar_test(&bars->emptyE[eE], ((nE / kRingE) & 1) ^ 1) &&
+                               mbar_test(&bars->emptyL[eL], ((nE / kRingL) & 1) ^ 1)))) {
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            uint8_t* sE = smem + Lay::E + eE * kSlot;
+            uint8_t* sL = smem + Lay::L + eL * kSlot;
+            // c_R rows [k0 .. k0+kTiles) (R, not first) or c_L rows [j0 .. j0+kTiles) (L): 128 floats
+            const bool needC = !t.first;
+            float* sC = reinterpret_cast<float*>(smem + Lay::Vec) + eL * 128;
+            mbar_expect_tx(&bars->fullE[eE], kSlot);
+            mbar_expect_tx(&bars->fullL[eL], kSlot + (needC ? 512 : 0));
+            if (t.isR) {
+              const int row0 = (t.h * m + t.idx0) * B;
+              if (needC) bulk_load_1d(sC, P.cR + row0, 512, &bars->fullL[eL]);
+              tma_load_2d(sE, t.first ? &P.tmQ : &P.tmAR, &bars->fullE[eE], 0, row0);
+              tma_load_2d(sL, &P.tmK, &bars->fullL[eL], 0, row0);
+            } else {
+              const int row0 = (t.h * B + t.idx0) * m;
+              bulk_load_1d(sC, P.cL + row0, 512, &bars->fullL[eL]);
+              tma_load_2d(sE, &P.tmAL, &bars->fullE[eE], 0, row0);
 #pragma unroll
-          for (int tt = 0; tt < kTiles; ++tt)
-            tma_load_3d(sL + tt * (B * 128), &P.tmQs, &bars->fullL[eL], 0, t.idx0 + tt, t.h * m);
-          if (needV) tma_load_2d(sV, &P.tmY, &bars->fullV[eV], 0, row0);
+              for (int tt = 0; tt < kTiles; ++tt)
+                tma_load_3d(sL + tt * (B * 128), &P.tmQs, &bars->fullL[eL], 0, t.idx0 + tt, t.h * m);
+            }
+            stamp(P, nE, 0);
+            ++nE;
+            itE.next();
+            if (deps && nE < n_total && itE.get().p > 0) ctrE = ld_acquire(counter_of(itE.get()));
+            did = true;
+          }
+        }
+        if (nVt < n_total) {
+          // the V (last R half-step) or y (last L half-step) tile is needed only by MMA 2
+          const Tile t = itV.get();
+          const int eV = nv % kRingV;
+          bool ok = force || !deps || t.p == 0 || ctrV >= P.tiles_per_head;
+          if (!ok) { ctrV = ld_acquire(counter_of(t)); ok = ctrV >= P.tiles_per_head; }
+          if (ok && (force || mbar_test(&bars->emptyV[eV], ((nv / kRingV) & 1) ^ 1))) {
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            uint8_t* sV = smem + Lay::V + eV * kSlot;
+            mbar_expect_tx(&bars->fullV[eV], kSlot);
+            if (t.isR) tma_load_2d(sV, &P.tmV, &bars->fullV[eV], 0, (t.h * m + t.idx0) * B);
+            else tma_load_2d(sV, &P.tmY, &bars->fullV[eV], 0, (t.h * B + t.idx0) * m);
+            ++nv;
+            do { ++nVt; itV.next(); } while (nVt < n_total && !needs_v(itV.get()));
+            if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
+            did = true;
+          }
+        }
+        if (did) {
+          t0 = clock64();
+        } else if (!force) {
+          if (bars->abort_flag) {
+            force = true;
+          } else if (clock64() - t0 > kWaitCycles) {
+            report_timeout(P.status, 10);
+            bars->abort_flag = 1;
+            force = true;
+          }
+          __nanosleep(32);
         }
       }
     }
@@ -253,17 +312,18 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
     // Two pending jobs are polled, never waited for: MMA 2 of the oldest unfinished tile (needs P
     // from its softmax group) and MMA 1 of the next tile (needs its operands, which may depend on
     // other CTAs).  Blocking on the second would hold up the first and could deadlock the grid.
-    if (lane == 0) {
+    if (elect_one()) {
       const uint32_t sE0 = smem_u32(smem + Lay::E), sL0 = smem_u32(smem + Lay::L);
       const uint32_t sV0 = smem_u32(smem + Lay::V), sP0 = smem_u32(smem + Lay::P);
       const uint32_t sOnes = smem_u32(smem + Lay::Ones);
       int i1 = 0, i2 = 0, nv = 0;
+      TileIter it1(P, first_g, stride_g, kTiles), it2(P, first_g, stride_g, kTiles);
       long long t0 = clock64();
       bool force = false;
       while (i2 < n_total) {
         bool did = false;
         if (i2 < i1) {
-          const Tile t = decode(P, first_g + i2 * stride_g, kTiles);
+          const Tile t = it2.get();
           const int a = i2 & 1, q = i2 >> 1, eL = i2 % kRingL;
           const bool needV = t.isR ? t.withV : t.final_;
           const int eV = nv % kRingV;
@@ -283,7 +343,9 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             umma_commit(&bars->emptyL[eL]);
             if (needV) { umma_commit(&bars->emptyV[eV]); ++nv; }
             umma_commit(&bars->o_ready[a]);
+            stamp(P, i2, 4);
             ++i2;
+            it2.next();
             did = true;
           }
         }
@@ -291,14 +353,16 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
           const int eE = i1 % kRingE, eL = i1 % kRingL, a = i1 & 1;
           if (force || (mbar_test(&bars->fullE[eE], (i1 / kRingE) & 1) &&
                         mbar_test(&bars->fullL[eL], (i1 / kRingL) & 1))) {
-            const Tile t = decode(P, first_g + i1 * stride_g, kTiles);
+            const Tile t = it1.get();
             tc_fence_after();
             const uint32_t sE = sE0 + eE * kSlot, sL = sL0 + eL * kSlot;
             // R: A = aR (E ring), B = K (L ring).  L: A = Qb (L ring), B = aL (E ring).
             issue_scores<B, FMT>(tmem + a * 256, t.isR ? sE : sL, t.isR ? sL : sE);
             umma_commit(&bars->emptyE[eE]);
             umma_commit(&bars->s_ready[a]);
+            stamp(P, i1, 1);
             ++i1;
+            it1.next();
             did = true;
           }
         }
@@ -312,152 +376,201 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             bars->abort_flag = 1;
             force = true;
           }
+          __nanosleep(20);
         }
       }
     }
   } else if (warp < 10) {
     // ------------------------------------------------------------------ softmax groups
     const int w = (warp - 2) >> 2;             // group = accumulator stage
-    const int tw = tid - 64 - w * 128;         // 0..127 inside the group
     const int sub = warp & 3;                  // TMEM sub-partition this warp may access
     const int t_row = sub * 32 + lane;         // TMEM lane = score row owned by this thread
     const int tile = Geo<B>::tile(t_row), r = Geo<B>::row(t_row), srow = tile * B + r;
     const uint32_t tS = tmem + w * 256 + ((uint32_t)(sub * 32) << 16);
     const uint32_t tO = tS + 128;
     uint8_t* sP = smem + Lay::P + w * 2 * kSlot;
-    float* cvec = reinterpret_cast<float*>(smem + Lay::Vec) + w * 128;
-    const int bar_id = 1 + w;
 
-    for (int n = w; n < n_total; n += 2) {
-      const Tile t = decode(P, first_g + n * stride_g, kTiles);
-      const int q = n >> 1;
-      wait_dependency(P, t, bars, 32);         // c_L / c_R of the previous half-step are final
-      float inv_c = 1.f;
-      size_t rrow = 0;
+    TileIter it(P, first_g + w * stride_g, 2 * stride_g, kTiles);
+    for (int n = w; n < n_total; n += 2, it.next()) {
+      const Tile t = it.get();
+      const int q = n >> 1, eL = n % kRingL;
+      const float* cv = reinterpret_cast<const float*>(smem + Lay::Vec) + eL * 128;
+      // operands (and the c-vector that travels with them) have landed; S is in tensor memory
+      wait_or_abort(&bars->fullL[eL], (n / kRingL) & 1, bars, P.status, 34);
+      wait_or_abort(&bars->s_ready[w], q & 1, bars, P.status, 30);
+      tc_fence_after();
+      if (lane == 0 && sub == 0) stamp(P, n, 2);
+
+      // The row is walked in 32-column chunks read from tensor memory, the next chunk being
+      // fetched while the current one is processed, so that a row never has to sit in registers.
+      // Arithmetic runs on packed fp32 pairs; exponentials are ex2 with log2(e) folded in.
+      constexpr int NC = B / 32;
+      float buf[32];
+      float f, inv_s, mx, sum, sz = 0.f;
+      size_t crow = 0;
+      float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      float2 a2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      const float* cvt = cv + tile * B;        // L: -c_L[j, :] in log2 units
       if (t.isR) {
-        rrow = (size_t)(t.h * m + t.idx0) * B + srow;       // [h][k][j]
+        // Z_R = scale * S / c_R (Eq. 7); c_L = sum R log R (Eq. 10)
+        float inv_c = 1.f;
         if (!t.first) {
-          const float c = __ldcg(P.cR + rrow);
+          const float c = cv[srow];
           inv_c = c > 1e-30f ? 1.f / c : 0.f;
         }
-      } else {
-        const int tile_e = tw / B, k_e = tw - tile_e * B;     // cL column(s) j0 (+1)
-        cvec[tw] = __ldcg(P.cL + ((size_t)t.h * m + k_e) * B + t.idx0 + tile_e) * kLog2e;
-      }
-      wait_or_abort(&bars->s_ready[w], q & 1, bars, P.status, 30);
-      if (!t.isR) group_barrier(bar_id);       // publish cvec
-      tc_fence_after();
-
-      float mx = -INFINITY, sum = 0.f, sz = 0.f, f, inv_s;
-      if (t.isR) {
         f = P.scale * inv_c * kLog2e;
+        crow = ((size_t)t.h * B + r) * m + t.idx0 + tile;      // c_L is stored [h][j][k]
 #pragma unroll
-        for (int c = 0; c < B / 32; ++c) {
-          float s[32];
-          tmem_ld32(tS + 32 * c, s);
+        for (int c = 0; c < NC; ++c) {
+          tmem_ld32(tS + 32 * c, buf);
           tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, s[i]);
+          for (int i = 0; i < 16; ++i)
+            m4[i & 3] = max3(m4[i & 3], buf[2 * i], buf[2 * i + 1]);
         }
-        const float off = -mx * f;
+        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        const float2 f2 = make_float2(f, f), off2 = make_float2(-mx * f, -mx * f);
+        float2 z2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
         // P and the store staging share a buffer: the previous tile's rows must have been read
         wait_or_abort(&bars->stage_free[w], (q & 1) ^ 1, bars, P.status, 33);
+        if (lane == 0 && sub == 0) stamp(P, n, 7);
 #pragma unroll
-        for (int c = 0; c < B / 32; ++c) {
-          float s[32];
-          tmem_ld32(tS + 32 * c, s);
+        for (int c = 0; c < NC; ++c) {
+          tmem_ld32(tS + 32 * c, buf);
           tmem_ld_wait();
+          float* s = buf;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float p = fast_exp2(fmaf(s[i], f, off));
-            sz = fmaf(p, s[i], sz);
-            sum += p;
-            s[i] = p;
+          for (int i = 0; i < 16; ++i) {
+            const float2 sv = make_float2(s[2 * i], s[2 * i + 1]);
+            const float2 zz = ffma2(sv, f2, off2);
+            const float2 pp = make_float2(fast_exp2(zz.x), fast_exp2(zz.y));
+            z2[i & 1] = ffma2(pp, sv, z2[i & 1]);
+            a2[i & 1] = fadd2(a2[i & 1], pp);
+            s[2 * i] = pp.x;
+            s[2 * i + 1] = pp.y;
           }
-          store_row32<T>(sP, srow, 32 * c, s, 1.f);
+          store_row32<T>(sP, srow, 32 * c, s);
         }
+        sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
+        sz = (z2[0].x + z2[0].y) + (z2[1].x + z2[1].y);
         inv_s = 1.f / sum;
       } else {
+        // Z_L = scale * S' - c_L (Eq. 8), softmax over k = along the row
         f = P.scale * kLog2e;
-        const float* cv = cvec + tile * B;
+        const float2 f2 = make_float2(f, f);
 #pragma unroll
-        for (int c = 0; c < B / 32; ++c) {
-          float s[32];
-          tmem_ld32(tS + 32 * c, s);
+        for (int c = 0; c < NC; ++c) {
+          tmem_ld32(tS + 32 * c, buf);
           tmem_ld_wait();
+          const float4* cv4 = reinterpret_cast<const float4*>(cvt + 32 * c);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaf(s[i], f, -cv[32 * c + i]));
+          for (int i = 0; i < 8; ++i) {
+            const float4 cc = cv4[i];
+            const float2 za = ffma2(make_float2(buf[4 * i], buf[4 * i + 1]), f2,
+                                    make_float2(cc.x, cc.y));
+            const float2 zb = ffma2(make_float2(buf[4 * i + 2], buf[4 * i + 3]), f2,
+                                    make_float2(cc.z, cc.w));
+            m4[0] = max3(m4[0], za.x, za.y);
+            m4[1] = max3(m4[1], zb.x, zb.y);
+          }
+        }
+        mx = fmaxf(m4[0], m4[1]);
+        const float2 nmx2 = make_float2(-mx, -mx);
+        if (!t.final_) {
+          // MMA 2 of this half-step contracts over rows, so P must be normalised before it is
+          // written: one pass for the row sum, one to write P / sum.
+#pragma unroll
+          for (int c = 0; c < NC; ++c) {
+            tmem_ld32(tS + 32 * c, buf);
+          tmem_ld_wait();
+            const float4* cv4 = reinterpret_cast<const float4*>(cvt + 32 * c);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float4 cc = cv4[i];
+              float2 za = ffma2(make_float2(buf[4 * i], buf[4 * i + 1]), f2,
+                                make_float2(cc.x, cc.y));
+              float2 zb = ffma2(make_float2(buf[4 * i + 2], buf[4 * i + 3]), f2,
+                                make_float2(cc.z, cc.w));
+              za = fadd2(za, nmx2);
+              zb = fadd2(zb, nmx2);
+              a2[0] = fadd2(a2[0], make_float2(fast_exp2(za.x), fast_exp2(za.y)));
+              a2[1] = fadd2(a2[1], make_float2(fast_exp2(zb.x), fast_exp2(zb.y)));
+            }
+          }
+          sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
+          inv_s = 1.f / sum;
+          a2[0] = a2[1] = make_float2(0.f, 0.f);
+        }
+        wait_or_abort(&bars->stage_free[w], (q & 1) ^ 1, bars, P.status, 33);
+        if (lane == 0 && sub == 0) stamp(P, n, 7);
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          tmem_ld32(tS + 32 * c, buf);
+          tmem_ld_wait();
+          float* s = buf;
+          const float4* cv4 = reinterpret_cast<const float4*>(cvt + 32 * c);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float4 cc = cv4[i];
+            float2 za = ffma2(make_float2(s[4 * i], s[4 * i + 1]), f2, make_float2(cc.x, cc.y));
+            float2 zb = ffma2(make_float2(s[4 * i + 2], s[4 * i + 3]), f2, make_float2(cc.z, cc.w));
+            za = fadd2(za, nmx2);
+            zb = fadd2(zb, nmx2);
+            const float2 pa = make_float2(fast_exp2(za.x), fast_exp2(za.y));
+            const float2 pb = make_float2(fast_exp2(zb.x), fast_exp2(zb.y));
+            a2[0] = fadd2(a2[0], pa);
+            a2[1] = fadd2(a2[1], pb);
+            s[4 * i] = pa.x;
+            s[4 * i + 1] = pa.y;
+            s[4 * i + 2] = pb.x;
+            s[4 * i + 3] = pb.y;
+          }
+          if (t.final_) store_row32<T>(sP, srow, 32 * c, s);
+          else store_row32<T>(sP, srow, 32 * c, s, inv_s);
         }
         if (t.final_) {
-          wait_or_abort(&bars->stage_free[w], (q & 1) ^ 1, bars, P.status, 33);
-#pragma unroll
-          for (int c = 0; c < B / 32; ++c) {
-            float s[32];
-            tmem_ld32(tS + 32 * c, s);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              s[i] = fast_exp2(fmaf(s[i], f, -cv[32 * c + i]) - mx);
-              sum += s[i];
-            }
-            store_row32<T>(sP, srow, 32 * c, s, 1.f);
-          }
+          sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
           inv_s = 1.f / sum;
-        } else {
-          // P must be normalised before MMA 2 (it contracts over rows): one more pass
-#pragma unroll
-          for (int c = 0; c < B / 32; ++c) {
-            float s[32];
-            tmem_ld32(tS + 32 * c, s);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) sum += fast_exp2(fmaf(s[i], f, -cv[32 * c + i]) - mx);
-          }
-          inv_s = 1.f / sum;
-          wait_or_abort(&bars->stage_free[w], (q & 1) ^ 1, bars, P.status, 33);
-#pragma unroll
-          for (int c = 0; c < B / 32; ++c) {
-            float s[32];
-            tmem_ld32(tS + 32 * c, s);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) s[i] = fast_exp2(fmaf(s[i], f, -cv[32 * c + i]) - mx);
-            store_row32<T>(sP, srow, 32 * c, s, inv_s);
-          }
         }
       }
       fence_proxy_async();
       tc_fence_before();
       mbar_arrive(&bars->p_ready[w]);
-      if (t.isR) P.cL[rrow] = kLn2 * (f * (sz * inv_s - mx) - fast_log2(sum));
+      if (lane == 0 && sub == 0) stamp(P, n, 3);
+      // -c_L in log2 units, ready to be the addend of the next L half-step's logits
+      if (t.isR) P.cL[crow] = fast_log2(sum) - f * (sz * inv_s - mx);
 
       wait_or_abort(&bars->o_ready[w], q & 1, bars, P.status, 31);
       tc_fence_after();
-      const int ncol = t.isR ? (t.withV ? 128 : 64) : 64;
-      const float mul = (t.isR || t.final_) ? inv_s : 1.f;
-      for (int c = 0; c < ncol / 32; ++c) {
-        float o[32];
-        tmem_ld32(tO + 32 * c, o);
-        tmem_ld_wait();
-        store_row32<T>(sP, srow, 32 * c, o, mul);
-      }
-      if (!t.isR && !t.final_) {
-        const float c1 = tmem_ld1(tO + 64);
-        tmem_ld_wait();
-        P.cR[((size_t)t.h * m + r) * B + t.idx0 + tile] = c1;
+      if (lane == 0 && sub == 0) stamp(P, n, 5);
+      const int nco = (t.isR && t.withV) ? 4 : 2;            // 32-column chunks of O
+      const bool scaled = t.isR || t.final_;
+      float c1 = 0.f;
+      if (!t.isR && !t.final_) c1 = tmem_ld1(tO + 64);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        if (c < nco) {
+          tmem_ld32(tO + 32 * c, buf);
+          tmem_ld_wait();
+          if (scaled) store_row32<T>(sP, srow, 32 * c, buf, inv_s);
+          else store_row32<T>(sP, srow, 32 * c, buf);
+        }
       }
       tc_fence_before();
       mbar_arrive(&bars->o_free[w]);
+      if (!t.isR && !t.final_) P.cR[((size_t)t.h * m + r) * B + t.idx0 + tile] = c1;
       fence_proxy_async();
       mbar_arrive(&bars->stage_ready[w]);
+      if (lane == 0 && sub == 0) stamp(P, n, 6);
     }
   } else {
-    // ------------------------------------------------------------------ store lanes
-    if (lane < 2) {
-      const int w = lane;
+    // ------------------------------------------------------------------ store threads
+    if (lane == 0) {
+      const int w = warp - 10;
       const uint8_t* sP = smem + Lay::P + w * 2 * kSlot;
-      for (int n = w; n < n_total; n += 2) {
-        const Tile t = decode(P, first_g + n * stride_g, kTiles);
+      TileIter it(P, first_g + w * stride_g, 2 * stride_g, kTiles);
+      for (int n = w; n < n_total; n += 2, it.next()) {
+        const Tile t = it.get();
         const int q = n >> 1;
         wait_or_abort(&bars->stage_ready[w], q & 1, bars, P.status, 40);
 #pragma unroll
@@ -493,6 +606,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
 }
 
 // ------------------------------------------------------------------------------------ host side
+inline long long*& trace_buffer() {
+  static long long* p = nullptr;
+  return p;
+}
 inline size_t counters_bytes(int BH, int T) {
   return ((size_t)2 * T * BH * sizeof(int) + 255) / 256 * 256;
 }
@@ -518,6 +635,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
             make_map_strided(&P.tmOut, dtype, Y, B, (uint64_t)BH * m, B);
   if (!ok) return 7;
   P.cL = w.cL; P.cR = w.cR; P.status = w.status; P.counters = counters;
+  P.trace = trace_buffer();
   P.m = m; P.BH = BH; P.T = T_steps;
   P.tiles_per_head = m / Geo<B>::kTiles;
   P.tiles_per_phase = BH * P.tiles_per_head;
