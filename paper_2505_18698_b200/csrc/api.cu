@@ -153,6 +153,7 @@ constexpr int kMaxDevices = 64;
 struct DeviceBuffers {
   void* ws = nullptr;
   size_t ws_bytes = 0;
+  long long armed_key = -1;   // problem whose status block / counters the workspace is armed for
   void* stage = nullptr;   // Q, K, V, Y staging for the host entry point
   size_t stage_bytes = 0;
 };
@@ -177,7 +178,8 @@ static int grow(void** ptr, size_t* have, size_t need) {
 }
 
 static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Problem& p,
-                  float scale, int resolved, void* ws, size_t ws_bytes, cudaStream_t st) {
+                  float scale, int resolved, void* ws, size_t ws_bytes, cudaStream_t st,
+                  bool ws_armed = false) {
   if (!ws || ws_bytes < workspace_bytes_for(p, resolved)) return MA_ERR_WORKSPACE;
   if (((uintptr_t)ws & 255) != 0) return MA_ERR_ALIGN;
   if (resolved == MA_PATH_GENERIC) return launch_generic(p, Q, K, V, Y, scale, ws, st);
@@ -187,7 +189,7 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
     rc = tensor::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.T, p.dtype, scale, ws, st, &launches);
   else
     rc = tp::launch(Q, K, V, Y, p.BH, p.N, p.b, p.T, p.dtype, scale, ws, st, &launches,
-                    resolved == MA_PATH_TENSOR ? 0 : 1);
+                    resolved == MA_PATH_TENSOR ? 0 : 1, ws_armed);
   if (rc == MA_OK) g_last_launches = launches;
   return rc;
 }
@@ -246,9 +248,17 @@ int monarch_attn_fwd(const void* Q, const void* K, const void* V, void* Y, int b
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MA_ERR_CUDA;
   DeviceBuffers& B = g_dev[dev];
+  const size_t had = B.ws_bytes;
   rc = grow(&B.ws, &B.ws_bytes, workspace_bytes_for(p, r));
   if (rc != MA_OK) return rc;
-  return fwd_ex(Q, K, V, Y, p, 1.0f / sqrtf((float)d), r, B.ws, B.ws_bytes, (cudaStream_t)stream);
+  // The persistent kernel leaves its status block and counters zeroed, so the library's own
+  // workspace is cleared only when the problem (hence the layout) changes.
+  const long long key = ((long long)r << 56) ^ ((long long)p.T << 48) ^ ((long long)p.BH << 24) ^ p.N;
+  const bool armed = (r == MA_PATH_TENSOR) && had == B.ws_bytes && B.armed_key == key;
+  rc = fwd_ex(Q, K, V, Y, p, 1.0f / sqrtf((float)d), r, B.ws, B.ws_bytes, (cudaStream_t)stream,
+              armed);
+  B.armed_key = (rc == MA_OK && r == MA_PATH_TENSOR) ? key : -1;
+  return rc;
 }
 
 int monarch_attn_fwd_host(const void* Qh, const void* Kh, const void* Vh, void* Yh, int batch,
@@ -291,6 +301,10 @@ int monarch_attn_device_status(const void* workspace, void* stream) {
       cudaSuccess)
     return MA_ERR_CUDA;
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MA_ERR_CUDA;
+  if (word != 0 && !workspace) {   // an aborted run leaves counters behind: clear on the next call
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) g_dev[dev].armed_key = -1;
+  }
   return word == 0 ? MA_OK : MA_ERR_TIMEOUT;
 }
 

@@ -224,6 +224,14 @@ template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, fl
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
+template <typename T> __device__ __forceinline__ float2 unpack2(uint32_t u);
+template <> __device__ __forceinline__ float2 unpack2<__half>(uint32_t u) {
+  return __half22float2(*reinterpret_cast<__half2*>(&u));
+}
+template <> __device__ __forceinline__ float2 unpack2<__nv_bfloat16>(uint32_t u) {
+  return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+}
+
 // Packed fp32 pairs (sm_100 f32x2 instructions: one issue slot for two lanes of work).
 __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
   float2 d;
@@ -248,6 +256,31 @@ __device__ __forceinline__ float2 fmul2(float2 a, float2 b) {
       : "=f"(d.x), "=f"(d.y)
       : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
   return d;
+}
+// 2^x for a pair of non-positive arguments on the FMA and integer pipes (the special-function
+// pipe, 16 results per clock per SM, is the busiest pipe of the softmax): round-to-nearest split
+// x = n + r, |r| <= 1/2, cubic minimax polynomial for 2^r (max relative error 7.5e-5, well below
+// 16-bit rounding), n added to the exponent field.  Arguments below -125 give ~2^-125.
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+  x.x = fmaxf(x.x, -125.f);
+  x.y = fmaxf(x.y, -125.f);
+  const float2 magic = make_float2(12582912.f, 12582912.f);      // 1.5 * 2^23
+  const float2 t = fadd2(x, magic);                               // low mantissa bits hold n
+  const float2 n = fadd2(t, make_float2(-12582912.f, -12582912.f));
+  const float2 r = ffma2(n, make_float2(-1.f, -1.f), x);
+  float2 p = ffma2(r, make_float2(0.05517167f, 0.05517167f), make_float2(0.24261112f, 0.24261112f));
+  p = ffma2(p, r, make_float2(0.69326099f, 0.69326099f));
+  p = ffma2(p, r, make_float2(0.99992807f, 0.99992807f));
+  p.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+  p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+  return p;
+}
+// Pair i of a chunk: one pair in kPolyEvery takes the polynomial, the others ex2.approx
+// (i is a compile-time constant after unrolling).
+constexpr int kPolyEvery = 4;
+__device__ __forceinline__ float2 exp2_pair(float2 z, int i) {
+  if (i % kPolyEvery == kPolyEvery - 1) return exp2_poly2(z);
+  return make_float2(fast_exp2(z.x), fast_exp2(z.y));
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;

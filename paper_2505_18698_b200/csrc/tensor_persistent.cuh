@@ -71,6 +71,7 @@ struct Params {
   int tiles_per_head, tiles_per_phase;
   int g_begin, g_end;  // tile range of this launch
   int check_deps;
+  int n_counters;      // 2T * BH
   float scale;
 };
 
@@ -395,8 +396,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       const Tile t = it.get();
       const int q = n >> 1, eL = n % kRingL;
       const float* cv = reinterpret_cast<const float*>(smem + Lay::Vec) + eL * 128;
-      // operands (and the c-vector that travels with them) have landed; S is in tensor memory
-      wait_or_abort(&bars->fullL[eL], (n / kRingL) & 1, bars, P.status, 34);
+      // S is in tensor memory; the c-vector travelled with MMA 1's operands, whose arrival the MMA
+      // thread observed before it issued (and committed) the MMA this barrier reports
       wait_or_abort(&bars->s_ready[w], q & 1, bars, P.status, 30);
       tc_fence_after();
       if (lane == 0 && sub == 0) stamp(P, n, 2);
@@ -443,7 +444,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
           for (int i = 0; i < 16; ++i) {
             const float2 sv = make_float2(s[2 * i], s[2 * i + 1]);
             const float2 zz = ffma2(sv, f2, off2);
-            const float2 pp = make_float2(fast_exp2(zz.x), fast_exp2(zz.y));
+            const float2 pp = exp2_pair(zz, i);
             z2[i & 1] = ffma2(pp, sv, z2[i & 1]);
             a2[i & 1] = fadd2(a2[i & 1], pp);
             s[2 * i] = pp.x;
@@ -476,31 +477,6 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
         }
         mx = fmaxf(m4[0], m4[1]);
         const float2 nmx2 = make_float2(-mx, -mx);
-        if (!t.final_) {
-          // MMA 2 of this half-step contracts over rows, so P must be normalised before it is
-          // written: one pass for the row sum, one to write P / sum.
-#pragma unroll
-          for (int c = 0; c < NC; ++c) {
-            tmem_ld32(tS + 32 * c, buf);
-          tmem_ld_wait();
-            const float4* cv4 = reinterpret_cast<const float4*>(cvt + 32 * c);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const float4 cc = cv4[i];
-              float2 za = ffma2(make_float2(buf[4 * i], buf[4 * i + 1]), f2,
-                                make_float2(cc.x, cc.y));
-              float2 zb = ffma2(make_float2(buf[4 * i + 2], buf[4 * i + 3]), f2,
-                                make_float2(cc.z, cc.w));
-              za = fadd2(za, nmx2);
-              zb = fadd2(zb, nmx2);
-              a2[0] = fadd2(a2[0], make_float2(fast_exp2(za.x), fast_exp2(za.y)));
-              a2[1] = fadd2(a2[1], make_float2(fast_exp2(zb.x), fast_exp2(zb.y)));
-            }
-          }
-          sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
-          inv_s = 1.f / sum;
-          a2[0] = a2[1] = make_float2(0.f, 0.f);
-        }
         wait_or_abort(&bars->stage_free[w], (q & 1) ^ 1, bars, P.status, 33);
         if (lane == 0 && sub == 0) stamp(P, n, 7);
 #pragma unroll
@@ -516,8 +492,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             float2 zb = ffma2(make_float2(s[4 * i + 2], s[4 * i + 3]), f2, make_float2(cc.z, cc.w));
             za = fadd2(za, nmx2);
             zb = fadd2(zb, nmx2);
-            const float2 pa = make_float2(fast_exp2(za.x), fast_exp2(za.y));
-            const float2 pb = make_float2(fast_exp2(zb.x), fast_exp2(zb.y));
+            const float2 pa = exp2_pair(za, 2 * i);
+            const float2 pb = exp2_pair(zb, 2 * i + 1);
             a2[0] = fadd2(a2[0], pa);
             a2[1] = fadd2(a2[1], pb);
             s[4 * i] = pa.x;
@@ -525,12 +501,28 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             s[4 * i + 2] = pb.x;
             s[4 * i + 3] = pb.y;
           }
-          if (t.final_) store_row32<T>(sP, srow, 32 * c, s);
-          else store_row32<T>(sP, srow, 32 * c, s, inv_s);
+          store_row32<T>(sP, srow, 32 * c, s);
         }
-        if (t.final_) {
-          sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
-          inv_s = 1.f / sum;
+        sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
+        inv_s = 1.f / sum;
+        if (!t.final_) {
+          // MMA 2 of this half-step contracts over rows, so P must be normalised before the MMA
+          // reads it: the thread re-reads its own row, rescales it in fp32 and writes it back
+          // (no other thread touches the row in between).
+          const float2 is2 = make_float2(inv_s, inv_s);
+#pragma unroll 2
+          for (int c8 = 0; c8 < B / 8; ++c8) {       // 8 columns = one 16-byte chunk
+            uint4* ptr = reinterpret_cast<uint4*>(sP + (c8 >> 3) * kTileBytes + srow * 128 +
+                                                  (((c8 & 7) ^ (srow & 7)) << 4));
+            uint4 qv = *ptr;
+            uint32_t* qp = reinterpret_cast<uint32_t*>(&qv);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 v = fmul2(unpack2<T>(qp[e]), is2);
+              qp[e] = pack2<T>(v.x, v.y);
+            }
+            *ptr = qv;
+          }
         }
       }
       fence_proxy_async();
@@ -603,6 +595,15 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
     __syncthreads();
   }
   if (warp == 0) tmem_dealloc(tmem, 512);
+  // The last CTA to finish re-arms the dependency counters (every CTA has done its last counter
+  // read by now), so that a caller who keeps the workspace need not clear it between calls.
+  if (tid == 0) {
+    __threadfence();
+    if (atomicAdd(P.status + 1, 1) == (int)gridDim.x - 1) {
+      for (int i = 0; i < P.n_counters; ++i) P.counters[i] = 0;
+      P.status[1] = 0;
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -619,7 +620,8 @@ inline size_t workspace_bytes(int BH, int N, int T) {
 
 template <typename T, int B>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int T_steps,
-                    int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode) {
+                    int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
+                    bool ws_armed) {
   const Ws w = ws_layout(ws, BH, N);
   int* counters = (int*)((char*)ws + w.bytes);
   const int m = N / B;
@@ -640,8 +642,11 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   P.tiles_per_head = m / Geo<B>::kTiles;
   P.tiles_per_phase = BH * P.tiles_per_head;
   P.scale = scale;
-  if (cudaMemsetAsync(ws, 0, kWsStatusBytes, st) != cudaSuccess) return 7;
-  if (cudaMemsetAsync(counters, 0, counters_bytes(BH, T_steps), st) != cudaSuccess) return 7;
+  P.n_counters = 2 * T_steps * BH;
+  if (!ws_armed) {   // status block and counters start at zero; the kernel leaves them that way
+    if (cudaMemsetAsync(ws, 0, kWsStatusBytes, st) != cudaSuccess) return 7;
+    if (cudaMemsetAsync(counters, 0, counters_bytes(BH, T_steps), st) != cudaSuccess) return 7;
+  }
   static int num_sms = 0;
   if (num_sms == 0) {
     int dev = 0;
@@ -673,14 +678,15 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
 }
 
 inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int b, int T,
-                  int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode) {
+                  int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
+                  bool ws_armed) {
   if (dtype == 1) {
-    if (b == 128) return launch_t<__half, 128>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode);
-    return launch_t<__half, 64>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode);
+    if (b == 128) return launch_t<__half, 128>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed);
+    return launch_t<__half, 64>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed);
   }
   if (b == 128)
-    return launch_t<__nv_bfloat16, 128>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode);
-  return launch_t<__nv_bfloat16, 64>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode);
+    return launch_t<__nv_bfloat16, 128>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed);
+  return launch_t<__nv_bfloat16, 64>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed);
 }
 
 }  // namespace tp
