@@ -97,6 +97,32 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* tm, ui
       "l"((uint64_t)tm), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
+// L2 eviction-priority policies for data that is touched once.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* tm, uint64_t* bar,
+                                                 int x, int y, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4}], [%2], %5;" ::"r"(smem_u32(dst)),
+      "l"((uint64_t)tm), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_3d_hint(const CUtensorMap* tm, const void* src, int x,
+                                                  int y, int z, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4}], "
+      "[%1], %5;" ::"l"((uint64_t)tm),
+      "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z), "l"(policy)
+      : "memory");
+}
+// Drops a 128-byte line from L2 without writing it back (its contents become undefined).
+__device__ __forceinline__ void discard_line(const void* p) {
+  asm volatile("discard.global.L2 [%0], 128;" ::"l"(p) : "memory");
+}
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, const void* src, int x, int y,
                                              int z) {
   asm volatile(
@@ -363,14 +389,18 @@ __device__ __forceinline__ void issue_scores(uint32_t tmem_s, uint32_t sA, uint3
 
 // Issues MMA 2 with A = P (K-major, [rows][B] in 64-column chunks) and B = [X0 | X1] read MN-major
 // from [B rows][64] tiles (N = 64 * nb).  D[row, :] = sum_c P[row, c] X[c, :].
-template <int B, int FMT>
+// PART: 0 = all k-steps, 1 = first half of the P columns only, 2 = second half only (so that the
+// first half can run while the softmax is still producing the second).
+template <int B, int FMT, int PART = 0>
 __device__ __forceinline__ void issue_apply(uint32_t tmem_o, uint32_t sP, uint32_t sX0,
                                             uint32_t x_chunk_stride, int nb) {
   const uint32_t idesc = instr_desc(B, 64 * nb, FMT, 0, 1);
+  constexpr int KS = B / 16;
+  constexpr int ks0 = PART == 2 ? KS / 2 : 0, ks1 = PART == 1 ? KS / 2 : KS;
 #pragma unroll
   for (int t = 0; t < Geo<B>::kTiles; ++t) {
 #pragma unroll
-    for (int ks = 0; ks < B / 16; ++ks) {
+    for (int ks = ks0; ks < ks1; ++ks) {
       const uint32_t pa = sP + (ks >> 2) * kTileBytes + t * (B * 128) + (ks & 3) * 32;
       const uint32_t xb = sX0 + t * (B * 128) + ks * 2048;
       if (ks == 0)

@@ -52,7 +52,7 @@ struct __align__(8) Bars {
   uint64_t fullE[kRingE], emptyE[kRingE];
   uint64_t fullL[kRingL], emptyL[kRingL];
   uint64_t fullV[kRingV], emptyV[kRingV];
-  uint64_t s_ready[2], p_ready[2], o_ready[2], o_free[2], stage_ready[2], stage_free[2];
+  uint64_t s_ready[2], p_half[2], p_ready[2], o_ready[2], o_free[2], stage_ready[2], stage_free[2];
   uint32_t tmem_slot;
   volatile int abort_flag;
 };
@@ -64,6 +64,7 @@ struct Params {
   CUtensorMap tmARs, tmOut;                      // 3D strided stores of aR / Y
   float* cL;
   float* cR;
+  uint8_t *aL, *aR, *y;  // state arrays (for L2 discards once a tile has been consumed)
   int* status;
   int* counters;       // [2T][BH] completed tiles
   long long* trace;    // optional: clock64 stamps [4 CTAs][64 tiles][8 events] (profiling aid)
@@ -199,6 +200,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
     for (int i = 0; i < kRingV; ++i) { mbar_init(&bars->fullV[i], 1); mbar_init(&bars->emptyV[i], 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars->s_ready[i], 1);
+      mbar_init(&bars->p_half[i], 128);
       mbar_init(&bars->p_ready[i], 128);
       mbar_init(&bars->o_ready[i], 1);
       mbar_init(&bars->o_free[i], 128);
@@ -234,6 +236,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       TileIter itE(P, first_g, stride_g, kTiles), itV(P, first_g, stride_g, kTiles);
       while (nVt < n_total && !needs_v(itV.get())) { ++nVt; itV.next(); }
       // dependency counters are read one step ahead so their latency is off the critical path
+      const uint64_t pol_first = policy_evict_first();
       int ctrE = 0, ctrV = 0;
       if (deps && nE < n_total && itE.get().p > 0) ctrE = ld_acquire(counter_of(itE.get()));
       if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
@@ -286,7 +289,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             asm volatile("fence.proxy.async.global;" ::: "memory");
             uint8_t* sV = smem + Lay::V + eV * kSlot;
             mbar_expect_tx(&bars->fullV[eV], kSlot);
-            if (t.isR) tma_load_2d(sV, &P.tmV, &bars->fullV[eV], 0, (t.h * m + t.idx0) * B);
+            if (t.isR) tma_load_2d_hint(sV, &P.tmV, &bars->fullV[eV], 0, (t.h * m + t.idx0) * B, pol_first);
             else tma_load_2d(sV, &P.tmY, &bars->fullV[eV], 0, (t.h * B + t.idx0) * m);
             ++nv;
             do { ++nVt; itV.next(); } while (nVt < n_total && !needs_v(itV.get()));
@@ -318,6 +321,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       const uint32_t sV0 = smem_u32(smem + Lay::V), sP0 = smem_u32(smem + Lay::P);
       const uint32_t sOnes = smem_u32(smem + Lay::Ones);
       int i1 = 0, i2 = 0, nv = 0;
+      bool half_done = false;
       TileIter it1(P, first_g, stride_g, kTiles), it2(P, first_g, stride_g, kTiles);
       long long t0 = clock64();
       bool force = false;
@@ -328,16 +332,28 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
           const int a = i2 & 1, q = i2 >> 1, eL = i2 % kRingL;
           const bool needV = t.isR ? t.withV : t.final_;
           const int eV = nv % kRingV;
-          if (force || (mbar_test(&bars->p_ready[a], q & 1) && mbar_test(&bars->o_free[a], (q & 1) ^ 1) &&
-                        (!needV || mbar_test(&bars->fullV[eV], (nv / kRingV) & 1)))) {
+          const bool split = t.isR || t.final_;     // P arrives in two column halves
+          const uint32_t sL = sL0 + eL * kSlot, sV = sV0 + eV * kSlot, sP = sP0 + a * 2 * kSlot;
+          const uint32_t tO = tmem + a * 256 + 128;
+          if (split && !half_done &&
+              (force || (mbar_test(&bars->p_half[a], q & 1) && mbar_test(&bars->o_free[a], (q & 1) ^ 1) &&
+                         (!needV || mbar_test(&bars->fullV[eV], (nv / kRingV) & 1))))) {
+            // first half of the P columns is in shared memory: start MMA 2 under the softmax
             tc_fence_after();
-            const uint32_t sL = sL0 + eL * kSlot, sV = sV0 + eV * kSlot, sP = sP0 + a * 2 * kSlot;
-            const uint32_t tO = tmem + a * 256 + 128;
+            if (t.isR) issue_apply<B, FMT, 1>(tO, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
+            else issue_apply<B, FMT, 1>(tO, sP, sV, 16, 1);
+            half_done = true;
+            did = true;
+          }
+          if ((half_done || !split) &&
+              (force || (mbar_test(&bars->p_ready[a], q & 1) &&
+                         (split || mbar_test(&bars->o_free[a], (q & 1) ^ 1))))) {
+            tc_fence_after();
             if (t.isR) {
               // [aL | y] = P [K | V]; the V tile sits (sV - sL) bytes after the K tile
-              issue_apply<B, FMT>(tO, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
+              issue_apply<B, FMT, 2>(tO, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
             } else if (t.final_) {
-              issue_apply<B, FMT>(tO, sP, sV, 16, 1);
+              issue_apply<B, FMT, 2>(tO, sP, sV, 16, 1);
             } else {
               issue_transposed_apply<B, FMT>(tO, sP, sL, sOnes);
             }
@@ -347,6 +363,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             stamp(P, i2, 4);
             ++i2;
             it2.next();
+            half_done = false;
             did = true;
           }
         }
@@ -401,6 +418,14 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       wait_or_abort(&bars->s_ready[w], q & 1, bars, P.status, 30);
       tc_fence_after();
       if (lane == 0 && sub == 0) stamp(P, n, 2);
+      // MMA 1 has consumed the state tile (alpha_R rows of an R half-step, alpha_L rows of an L
+      // half-step): every such tile is read exactly once, so its lines are dropped from L2 instead
+      // of being written back to HBM later.
+      if (t.isR) {
+        if (!t.first) discard_line(P.aR + ((size_t)(t.h * m + t.idx0) * B + t_row) * 128);
+      } else {
+        discard_line(P.aL + ((size_t)(t.h * B + t.idx0) * m + t_row) * 128);
+      }
 
       // The row is walked in 32-column chunks read from tensor memory, the next chunk being
       // fetched while the current one is processed, so that a row never has to sit in registers.
@@ -451,6 +476,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             s[2 * i + 1] = pp.y;
           }
           store_row32<T>(sP, srow, 32 * c, s);
+          if (c == NC / 2 - 1) {    // first half of the row's P is written: MMA 2 may start on it
+            fence_proxy_async();
+            mbar_arrive(&bars->p_half[w]);
+          }
         }
         sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
         sz = (z2[0].x + z2[0].y) + (z2[1].x + z2[1].y);
@@ -502,6 +531,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             s[4 * i + 3] = pb.y;
           }
           store_row32<T>(sP, srow, 32 * c, s);
+          if (c == NC / 2 - 1 && t.final_) {    // first half of the row's P is written: MMA 2 may start on it
+            fence_proxy_async();
+            mbar_arrive(&bars->p_half[w]);
+          }
         }
         sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
         inv_s = 1.f / sum;
@@ -510,7 +543,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
           // reads it: the thread re-reads its own row, rescales it in fp32 and writes it back
           // (no other thread touches the row in between).
           const float2 is2 = make_float2(inv_s, inv_s);
-#pragma unroll 2
+#pragma unroll
           for (int c8 = 0; c8 < B / 8; ++c8) {       // 8 columns = one 16-byte chunk
             uint4* ptr = reinterpret_cast<uint4*>(sP + (c8 >> 3) * kTileBytes + srow * 128 +
                                                   (((c8 & 7) ^ (srow & 7)) << 4));
@@ -527,6 +560,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       }
       fence_proxy_async();
       tc_fence_before();
+      if (!t.isR && !t.final_) mbar_arrive(&bars->p_half[w]);   // keeps the barrier's phase in step
       mbar_arrive(&bars->p_ready[w]);
       if (lane == 0 && sub == 0) stamp(P, n, 3);
       // -c_L in log2 units, ready to be the addend of the next L half-step's logits
@@ -535,6 +569,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       wait_or_abort(&bars->o_ready[w], q & 1, bars, P.status, 31);
       tc_fence_after();
       if (lane == 0 && sub == 0) stamp(P, n, 5);
+      if (t.final_) discard_line(P.y + ((size_t)(t.h * B + t.idx0) * m + t_row) * 128);   // y: read once
       const int nco = (t.isR && t.withV) ? 4 : 2;            // 32-column chunks of O
       const bool scaled = t.isR || t.final_;
       float c1 = 0.f;
@@ -560,6 +595,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
     if (lane == 0) {
       const int w = warp - 10;
       const uint8_t* sP = smem + Lay::P + w * 2 * kSlot;
+      const uint64_t pol_first = policy_evict_first();
       TileIter it(P, first_g + w * stride_g, 2 * stride_g, kTiles);
       for (int n = w; n < n_total; n += 2, it.next()) {
         const Tile t = it.get();
@@ -572,7 +608,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             tma_store_3d(&P.tmALs, src, 0, t.idx0 + tt, t.h * B);
             if (t.withV) tma_store_3d(&P.tmYs, src + kSlot, 0, t.idx0 + tt, t.h * B);
           } else {
-            tma_store_3d(t.final_ ? &P.tmOut : &P.tmARs, src, 0, t.idx0 + tt, t.h * m);
+            if (t.final_) tma_store_3d_hint(&P.tmOut, src, 0, t.idx0 + tt, t.h * m, pol_first);
+            else tma_store_3d(&P.tmARs, src, 0, t.idx0 + tt, t.h * m);
           }
         }
         tma_store_commit();
@@ -636,6 +673,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
             make_map_strided(&P.tmARs, dtype, w.aR, B, (uint64_t)BH * m, B) &&
             make_map_strided(&P.tmOut, dtype, Y, B, (uint64_t)BH * m, B);
   if (!ok) return 7;
+  P.aL = (uint8_t*)w.aL; P.aR = (uint8_t*)w.aR; P.y = (uint8_t*)w.y;
   P.cL = w.cL; P.cR = w.cR; P.status = w.status; P.counters = counters;
   P.trace = trace_buffer();
   P.m = m; P.BH = BH; P.T = T_steps;
