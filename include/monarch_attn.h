@@ -36,7 +36,8 @@ typedef enum {
   MA_ERR_ALIGN = 5,       /* a base address is not 16-byte aligned, or Y aliases an input */
   MA_ERR_WORKSPACE = 6,   /* workspace NULL or smaller than monarch_attn_workspace_bytes() */
   MA_ERR_CUDA = 7,        /* a CUDA runtime/driver call failed */
-  MA_ERR_TIMEOUT = 8      /* a bounded device-side wait ran out (see monarch_attn_device_status) */
+  MA_ERR_TIMEOUT = 8,     /* a bounded device-side wait ran out (see monarch_attn_device_status) */
+  MA_ERR_TOO_LARGE = 9    /* the problem needs more scratch than monarch_attn_fwd_noalloc carries */
 } ma_status;
 
 /* Which kernels run.  AUTO picks the fastest path that supports the shape. */
@@ -77,6 +78,38 @@ int monarch_attn_fwd_ex(const void* Q, const void* K, const void* V, void* Y,
 int monarch_attn_fwd_host(const void* Q_host, const void* K_host, const void* V_host, void* Y_host,
                           int batch, int heads, int N, int d, int b, int T,
                           int dtype, void* stream);
+
+/* Scratch the no-allocation entry point below carries inside the library image, in bytes. */
+#define MONARCH_ATTN_NOALLOC_SCRATCH_BYTES (8u << 20)
+
+/* The same forward pass for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this is a deployment variant of the library, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a memory pool that owns
+ * the whole device, in a real-time loop where an allocation's implicit synchronisation is not
+ * acceptable, or in a process whose allocator hooks forbid foreign allocations -- and that has no
+ * spare buffer to lend as the workspace of monarch_attn_fwd_ex.
+ *
+ * What it does: runs the fp32 SIMT path (MA_PATH_GENERIC) with its states (alpha_L, alpha_R, y,
+ * c_L, c_R and the status block) in a fixed MONARCH_ATTN_NOALLOC_SCRATCH_BYTES array that is part
+ * of the library image; every GPU that loads the library holds that array until the process
+ * exits.  Q, K, V, Y are DEVICE pointers as for monarch_attn_fwd; scale = 1/sqrt(d).
+ *
+ * Limits and rules:
+ *   - 256 + 3*align256(4*batch*heads*N*d) + 2*align256(4*batch*heads*N) bytes must fit in the
+ *     array (about batch*heads*N*d <= 690,000 for d = 64); otherwise MA_ERR_TOO_LARGE is
+ *     returned and nothing is enqueued.  Shapes the generic path cannot run give
+ *     MA_ERR_UNSUPPORTED.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and keeps it; make that first call before any stream capture.
+ *   - It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left;
+ *     the status block is cleared by each call and every other word is written before it is
+ *     read.  Two calls whose kernels overlap on the GPU (different streams, no dependency) race
+ *     on it: serialise them. */
+int monarch_attn_fwd_noalloc(const void* Q, const void* K, const void* V, void* Y,
+                             int batch, int heads, int N, int d, int b, int T,
+                             int dtype, void* stream);
 
 /* Synchronises `stream` and reads the status word a run left in `workspace` (DEVICE pointer; NULL
  * means the library's own workspace on the current device): MA_OK, or MA_ERR_TIMEOUT if a bounded

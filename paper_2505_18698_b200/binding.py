@@ -56,6 +56,8 @@ def load_library(path: str = LIB_PATH):
     lib.monarch_attn_fwd_ex.restype = i
     lib.monarch_attn_fwd_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
     lib.monarch_attn_fwd_host.restype = i
+    lib.monarch_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
+    lib.monarch_attn_fwd_noalloc.restype = i
     lib.monarch_attn_device_status.argtypes = [vp, vp]
     lib.monarch_attn_device_status.restype = i
     lib.monarch_attn_last_launch_count.argtypes = []
@@ -148,6 +150,24 @@ def monarch_attn_fwd_host(Qh, Kh, Vh, Yh, b, T, stream=None):
                                      batch, heads, N, d, b, T, _TORCH_TO_CODE[Qh.dtype],
                                      _stream_ptr(stream)))
     return Yh
+
+
+NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def monarch_attn_fwd_noalloc(Q, K, V, b, T, Y, stream=None):
+    """Forward pass for callers that may not allocate device memory: the library's built-in
+    scratch array holds the states, and the caller supplies the output tensor Y as well (so this
+    wrapper allocates nothing either).  Small problems only (see the header for the limit);
+    calls that overlap on the GPU race on the shared scratch."""
+    lib = load_library()
+    if not (Q.is_cuda and Y.is_cuda):
+        raise MonarchAttnError(-2, "monarch_attn_fwd_noalloc needs CUDA tensors; there is no CPU path")
+    batch, heads, N, d = _shape_of(Q, K, V)
+    _check(lib.monarch_attn_fwd_noalloc(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                        batch, heads, N, d, b, T, _TORCH_TO_CODE[Q.dtype],
+                                        _stream_ptr(stream)))
+    return Y
 
 
 def monarch_attn_device_status(workspace=None, stream=None) -> int:

@@ -310,6 +310,41 @@ int monarch_attn_device_status(const void* workspace, void* stream) {
 
 int monarch_attn_last_launch_count(void) { return g_last_launches; }
 
+}  // extern "C"
+
+// ------------------------------------------------------------------ no-allocation entry point
+// Scratch for monarch_attn_fwd_noalloc lives in the library image.  In host code the name of a
+// __device__ array is only a handle for the runtime, never a device address: the address is
+// looked up once per device with cudaGetSymbolAddress and that pointer is what kernels receive.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[MONARCH_ATTN_NOALLOC_SCRATCH_BYTES];
+static void* g_noalloc_ptr[ma::kMaxDevices] = {nullptr};
+
+extern "C" {
+
+int monarch_attn_fwd_noalloc(const void* Q, const void* K, const void* V, void* Y, int batch,
+                             int heads, int N, int d, int b, int T, int dtype, void* stream) {
+  Problem p;
+  int rc = validate_shape(batch, heads, N, d, b, T, dtype, &p);
+  if (rc != MA_OK) return rc;
+  rc = check_ptrs(Q, K, V, Y, p);
+  if (rc != MA_OK) return rc;
+  if (!generic_supported(p)) return MA_ERR_UNSUPPORTED;
+  if (generic_layout(p, nullptr).bytes > (size_t)MONARCH_ATTN_NOALLOC_SCRATCH_BYTES)
+    return MA_ERR_TOO_LARGE;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MA_ERR_CUDA;
+  if (!g_noalloc_ptr[dev]) {   // set-up, once per device, with that device current
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return MA_ERR_CUDA;
+    }
+    g_noalloc_ptr[dev] = ptr;
+  }
+  return launch_generic(p, Q, K, V, Y, 1.0f / sqrtf((float)d), g_noalloc_ptr[dev],
+                        (cudaStream_t)stream);
+}
+
 int monarch_attn_set_trace_buffer(void* device_buffer, size_t bytes) {
   if (device_buffer != nullptr && bytes < (size_t)4 * 64 * 8 * sizeof(long long)) return MA_ERR_WORKSPACE;
   tp::trace_buffer() = (long long*)device_buffer;
@@ -327,6 +362,7 @@ const char* monarch_attn_status_string(int status) {
     case MA_ERR_WORKSPACE: return "workspace missing or too small";
     case MA_ERR_CUDA: return "a CUDA call failed";
     case MA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case MA_ERR_TOO_LARGE: return "problem exceeds the scratch built into monarch_attn_fwd_noalloc";
     default: return "unknown status";
   }
 }

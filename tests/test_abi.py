@@ -18,14 +18,15 @@ def test_header_symbols_are_exported(lib):
     names = binding.declared_symbols()
     assert {"monarch_attn_fwd", "monarch_attn_fwd_ex", "monarch_attn_workspace_bytes",
             "monarch_attn_fwd_host", "monarch_attn_device_status",
-            "monarch_attn_status_string", "monarch_attn_last_launch_count"} <= set(names)
+            "monarch_attn_status_string", "monarch_attn_last_launch_count",
+            "monarch_attn_fwd_noalloc", "monarch_attn_set_trace_buffer"} <= set(names)
     for n in names:
         assert getattr(lib, n) is not None
 
 
 def test_status_strings(lib):
-    seen = {binding.status_string(c) for c in range(9)}
-    assert len(seen) == 9 and binding.status_string(0) == "ok"
+    seen = {binding.status_string(c) for c in range(10)}
+    assert len(seen) == 10 and binding.status_string(0) == "ok"
     assert binding.status_string(99) == "unknown status"
 
 
