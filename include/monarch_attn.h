@@ -47,7 +47,9 @@ typedef enum {
   MA_PATH_TENSOR = 2,  /* tcgen05/TMA kernels, 16-bit states; f16/bf16, d = 64, m = b in {64,128}:
                           one persistent launch for all 2T half-steps */
   MA_PATH_TENSOR_PHASED = 3, /* the same persistent kernel, one launch per half-step */
-  MA_PATH_TENSOR_BASIC = 4   /* one CTA per tile, one launch per half-step (no pipelining) */
+  MA_PATH_TENSOR_BASIC = 4,  /* one CTA per tile, one launch per half-step (no pipelining) */
+  MA_PATH_FUSED = 5    /* one CTA per (batch, head), everything in shared memory, one launch:
+                          f16/bf16, N = 256, m = b = 16, d = 64 */
 } ma_path;
 
 /* T-step MonarchAttention forward (Eq. 7-10 then Eq. 4) with scale = 1/sqrt(d).

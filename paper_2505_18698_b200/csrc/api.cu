@@ -11,6 +11,7 @@
 #include "generic_kernels.cuh"
 #include "tensor_path.cuh"
 #include "tensor_persistent.cuh"
+#include "fused_n256.cuh"
 
 namespace ma {
 
@@ -130,11 +131,13 @@ static int launch_generic(const Problem& p, const void* Q, const void* K, const 
 // ------------------------------------------------------------------ path selection
 static int resolve_path(const Problem& p, int path) {
   if (path == MA_PATH_AUTO) {
+    if (fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_FUSED;
     if (tensor::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TENSOR;
     if (generic_supported(p)) return MA_PATH_GENERIC;
     return -1;
   }
   if (path == MA_PATH_GENERIC) return generic_supported(p) ? path : -1;
+  if (path == MA_PATH_FUSED) return fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
   if (path == MA_PATH_TENSOR || path == MA_PATH_TENSOR_PHASED || path == MA_PATH_TENSOR_BASIC)
     return tensor::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
   return -1;
@@ -142,6 +145,7 @@ static int resolve_path(const Problem& p, int path) {
 
 static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
+  if (resolved == MA_PATH_FUSED) return kStatusBytes;   // no states leave the chip
   if (resolved == MA_PATH_TENSOR_BASIC) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
   if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_PHASED)
     return tp::workspace_bytes(p.BH, p.N, p.T);
@@ -183,6 +187,11 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   if (!ws || ws_bytes < workspace_bytes_for(p, resolved)) return MA_ERR_WORKSPACE;
   if (((uintptr_t)ws & 255) != 0) return MA_ERR_ALIGN;
   if (resolved == MA_PATH_GENERIC) return launch_generic(p, Q, K, V, Y, scale, ws, st);
+  if (resolved == MA_PATH_FUSED) {
+    int rc = fused::launch(Q, K, V, Y, p.BH, p.T, p.dtype, scale, st);
+    if (rc == MA_OK) g_last_launches = 1;
+    return rc;
+  }
   int launches = 0;
   int rc;
   if (resolved == MA_PATH_TENSOR_BASIC)
