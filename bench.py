@@ -208,18 +208,24 @@ def time_e2e(w, steps, warmup, torch, binding, dist=None):
     return e0.elapsed_time(e1) / steps, 3 * nbytes, nbytes
 
 
+# DRAM bytes of ONE launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
+# ncu; see the summaries under profiles/ named for each kernel and workload).
+NCU_TRAFFIC_BYTES = {"C5": 191.4e6 + 44.4e6}
+
+
 def roofline(w, ms, peaks, which):
     t_hbm = w.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9)
     t_tc = w.algorithmic_flops() / (peaks["bf16_tflops_sustained"] * 1e12) if w.dtype != "f32" else 0.0
     if t_tc > t_hbm:
         ach = w.algorithmic_flops() / (ms * 1e-3) / 1e12
         return {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
-                "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None,
-                "of": which + " (sustained)", "scope": "whole step (all kernels of one call)"}
+                "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
+                "traffic": NCU_TRAFFIC_BYTES.get(w.name), "of": which + " (sustained)",
+                "scope": "one launch = one step (the tensor path is a single persistent kernel)"}
     ach = w.algorithmic_bytes() / (ms * 1e-3) / 1e9
     return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": ach / peaks["hbm_gbs"], "traffic": None, "of": which,
-            "scope": "whole step (all kernels of one call)"}
+            "frac": ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(w.name), "of": which,
+            "scope": "one step (one launch on the tensor and fused paths, 2T on the generic path)"}
 
 
 def sdpa_ms(w, torch, sets, iters=5):
@@ -265,14 +271,13 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2505_18698_b200 import distributed as D
+    rank, local, world = D.env_world()
     torch.cuda.set_device(local)
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl")
+        D.init("nccl")
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     peaks, which = load_peaks()
 
@@ -280,16 +285,9 @@ def main():
     sampler.start()
     res = time_config(w, steps, warmup, torch, binding, dist=dist)
     clocks = sampler.stop()
-    ms = res["total_ms"] / steps
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = D.max_over_ranks(res["total_ms"] / steps, device="cuda")
     e2e_ms, h2d, d2h = time_e2e(w, max(3, min(steps, 20)), 3, torch, binding, dist)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = D.max_over_ranks(e2e_ms, device="cuda")
 
     line = {
         "metric": METRIC, "value": world * w.tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,

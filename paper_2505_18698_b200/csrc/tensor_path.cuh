@@ -231,9 +231,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
 }
 // Instruction descriptor of tcgen05.mma kind::f16: fp32 accumulate, A/B format (0 f16, 1 bf16),
 // A/B major-ness (0 K-major, 1 MN-major), N >> 3, M >> 4.
-__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int fmt, int a_mn, int b_mn) {
-  return (1u << 4) | ((uint32_t)fmt << 7) | ((uint32_t)fmt << 10) | ((uint32_t)a_mn << 15) |
+__host__ __device__ constexpr uint32_t instr_desc2(int M, int N, int fmt_a, int fmt_b, int a_mn,
+                                                   int b_mn) {
+  return (1u << 4) | ((uint32_t)fmt_a << 7) | ((uint32_t)fmt_b << 10) | ((uint32_t)a_mn << 15) |
          ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int fmt, int a_mn, int b_mn) {
+  return instr_desc2(M, N, fmt, fmt, a_mn, b_mn);
 }
 
 template <typename T> struct Fmt;
@@ -372,9 +376,10 @@ template <int B> struct Geo {
 };
 
 // Issues MMA 1 (scores): both operands K-major [rows][64] tiles, K = d = 64 in four steps.
-template <int B, int FMT>
+// FA / FB: element format of the A / B operand (0 f16, 1 bf16); the two may differ.
+template <int B, int FA, int FB = FA>
 __device__ __forceinline__ void issue_scores(uint32_t tmem_s, uint32_t sA, uint32_t sB) {
-  constexpr uint32_t idesc = instr_desc(B, B, FMT, 0, 0);
+  constexpr uint32_t idesc = instr_desc2(B, B, FA, FB, 0, 0);
 #pragma unroll
   for (int t = 0; t < Geo<B>::kTiles; ++t) {
     const uint64_t da = smem_desc(sA + t * (B * 128), 16, 1024);
@@ -391,10 +396,10 @@ __device__ __forceinline__ void issue_scores(uint32_t tmem_s, uint32_t sA, uint3
 // from [B rows][64] tiles (N = 64 * nb).  D[row, :] = sum_c P[row, c] X[c, :].
 // PART: 0 = all k-steps, 1 = first half of the P columns only, 2 = second half only (so that the
 // first half can run while the softmax is still producing the second).
-template <int B, int FMT, int PART = 0>
+template <int B, int FA, int PART = 0, int FB = FA>
 __device__ __forceinline__ void issue_apply(uint32_t tmem_o, uint32_t sP, uint32_t sX0,
                                             uint32_t x_chunk_stride, int nb) {
-  const uint32_t idesc = instr_desc(B, 64 * nb, FMT, 0, 1);
+  const uint32_t idesc = instr_desc2(B, 64 * nb, FA, FB, 0, 1);
   constexpr int KS = B / 16;
   constexpr int ks0 = PART == 2 ? KS / 2 : 0, ks1 = PART == 1 ? KS / 2 : KS;
 #pragma unroll
@@ -415,11 +420,11 @@ __device__ __forceinline__ void issue_apply(uint32_t tmem_o, uint32_t sP, uint32
 
 // Issues MMA 2 of the non-final L half-step: contraction over the ROW index of P.
 //   D[c, 0:64] = sum_row P[row, c] X[row, :],  D[c, 64:80] = sum_row P[row, c]  (tile of ones)
-template <int B, int FMT>
+template <int B, int FA, int FB = FA>
 __device__ __forceinline__ void issue_transposed_apply(uint32_t tmem_o, uint32_t sP, uint32_t sX,
                                                        uint32_t sOnes) {
-  constexpr uint32_t idesc = instr_desc(B, 64, FMT, 1, 1);
-  constexpr uint32_t idesc1 = instr_desc(B, 16, FMT, 1, 0);
+  constexpr uint32_t idesc = instr_desc2(B, 64, FA, FB, 1, 1);
+  constexpr uint32_t idesc1 = instr_desc2(B, 16, FA, FA, 1, 0);   // ones tile has A's format
   const uint64_t ones = smem_desc(sOnes, 16, 1024);
 #pragma unroll
   for (int t = 0; t < Geo<B>::kTiles; ++t) {

@@ -184,13 +184,22 @@ __device__ __forceinline__ float tmem_ld1(uint32_t taddr) {
   return __uint_as_float(r);
 }
 
-template <typename T, int B>
+// B  = rows of one MMA tile (64 or 128); SB = the method's block size b = m (SB divides B).
+// With SB < B an MMA tile holds B / SB independent blocks on its diagonal: a score row only owns
+// the SB columns of its own block, the other columns of P are written as zeros, and the MMAs run
+// unchanged (b = 32 on M = 64 tiles wastes half the tensor work but none of the exponentials).
+template <typename T, int B, int SB>
 __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_constant__ Params P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   Bars* bars = reinterpret_cast<Bars*>(smem + Lay::Bars);
-  constexpr int kTiles = Geo<B>::kTiles;
-  constexpr int FMT = Fmt<T>::code;
+  constexpr int kBlocks = kRows / SB;         // blocks (k of an R tile, j of an L tile) per CTA
+  constexpr int NSUB = B / SB;                // blocks per MMA tile
+  // P and the states alpha_L, alpha_R, y have the inputs' type: kind::f16 needs A and B in the
+  // SAME 16-bit format on this hardware (an f16 operand against a bf16 one is an illegal
+  // instruction, although the instruction descriptor has a format field for each).
+  typedef T S;
+  constexpr int FT = Fmt<T>::code, FS = Fmt<S>::code;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int m = P.m;
 
@@ -212,7 +221,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
     fence_proxy_async();
   }
   if (tid < 128) {   // tile of ones for the column-sum MMA of the non-final L half-step
-    const uint32_t one2 = pack2<T>(1.f, 1.f);
+    const uint32_t one2 = pack2<S>(1.f, 1.f);
     *reinterpret_cast<uint4*>(smem + Lay::Ones + tid * 16) = make_uint4(one2, one2, one2, one2);
   }
   if (warp == 0) tmem_alloc(&bars->tmem_slot, 512);
@@ -233,7 +242,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       auto counter_of = [&](const Tile& t) { return P.counters + (t.p - 1) * P.BH + t.h; };
       auto needs_v = [&](const Tile& t) { return t.isR ? t.withV : t.final_; };
       int nE = 0, nVt = 0, nv = 0;                 // next tile for E/L, next tile to scan for V
-      TileIter itE(P, first_g, stride_g, kTiles), itV(P, first_g, stride_g, kTiles);
+      TileIter itE(P, first_g, stride_g, kBlocks), itV(P, first_g, stride_g, kBlocks);
       while (nVt < n_total && !needs_v(itV.get())) { ++nVt; itV.next(); }
       // dependency counters are read one step ahead so their latency is off the critical path
       const uint64_t pol_first = policy_evict_first();
@@ -260,17 +269,17 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             mbar_expect_tx(&bars->fullE[eE], kSlot);
             mbar_expect_tx(&bars->fullL[eL], kSlot + (needC ? 512 : 0));
             if (t.isR) {
-              const int row0 = (t.h * m + t.idx0) * B;
+              const int row0 = (t.h * m + t.idx0) * SB;
               if (needC) bulk_load_1d(sC, P.cR + row0, 512, &bars->fullL[eL]);
               tma_load_2d(sE, t.first ? &P.tmQ : &P.tmAR, &bars->fullE[eE], 0, row0);
               tma_load_2d(sL, &P.tmK, &bars->fullL[eL], 0, row0);
             } else {
-              const int row0 = (t.h * B + t.idx0) * m;
+              const int row0 = (t.h * SB + t.idx0) * m;
               bulk_load_1d(sC, P.cL + row0, 512, &bars->fullL[eL]);
               tma_load_2d(sE, &P.tmAL, &bars->fullE[eE], 0, row0);
 #pragma unroll
-              for (int tt = 0; tt < kTiles; ++tt)
-                tma_load_3d(sL + tt * (B * 128), &P.tmQs, &bars->fullL[eL], 0, t.idx0 + tt, t.h * m);
+              for (int tt = 0; tt < kBlocks; ++tt)
+                tma_load_3d(sL + tt * (SB * 128), &P.tmQs, &bars->fullL[eL], 0, t.idx0 + tt, t.h * m);
             }
             stamp(P, nE, 0);
             ++nE;
@@ -289,8 +298,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             asm volatile("fence.proxy.async.global;" ::: "memory");
             uint8_t* sV = smem + Lay::V + eV * kSlot;
             mbar_expect_tx(&bars->fullV[eV], kSlot);
-            if (t.isR) tma_load_2d_hint(sV, &P.tmV, &bars->fullV[eV], 0, (t.h * m + t.idx0) * B, pol_first);
-            else tma_load_2d(sV, &P.tmY, &bars->fullV[eV], 0, (t.h * B + t.idx0) * m);
+            if (t.isR) tma_load_2d_hint(sV, &P.tmV, &bars->fullV[eV], 0, (t.h * m + t.idx0) * SB, pol_first);
+            else tma_load_2d(sV, &P.tmY, &bars->fullV[eV], 0, (t.h * SB + t.idx0) * m);
             ++nv;
             do { ++nVt; itV.next(); } while (nVt < n_total && !needs_v(itV.get()));
             if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
@@ -322,7 +331,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       const uint32_t sOnes = smem_u32(smem + Lay::Ones);
       int i1 = 0, i2 = 0, nv = 0;
       bool half_done = false;
-      TileIter it1(P, first_g, stride_g, kTiles), it2(P, first_g, stride_g, kTiles);
+      TileIter it1(P, first_g, stride_g, kBlocks), it2(P, first_g, stride_g, kBlocks);
       long long t0 = clock64();
       bool force = false;
       while (i2 < n_total) {
@@ -340,8 +349,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
                          (!needV || mbar_test(&bars->fullV[eV], (nv / kRingV) & 1))))) {
             // first half of the P columns is in shared memory: start MMA 2 under the softmax
             tc_fence_after();
-            if (t.isR) issue_apply<B, FMT, 1>(tO, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
-            else issue_apply<B, FMT, 1>(tO, sP, sV, 16, 1);
+            if (t.isR) issue_apply<B, FS, 1, FT>(tO, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
+            else issue_apply<B, FS, 1, FS>(tO, sP, sV, 16, 1);
             half_done = true;
             did = true;
           }
@@ -351,11 +360,11 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             tc_fence_after();
             if (t.isR) {
               // [aL | y] = P [K | V]; the V tile sits (sV - sL) bytes after the K tile
-              issue_apply<B, FMT, 2>(tO, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
+              issue_apply<B, FS, 2, FT>(tO, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
             } else if (t.final_) {
-              issue_apply<B, FMT, 2>(tO, sP, sV, 16, 1);
+              issue_apply<B, FS, 2, FS>(tO, sP, sV, 16, 1);
             } else {
-              issue_transposed_apply<B, FMT>(tO, sP, sL, sOnes);
+              issue_transposed_apply<B, FS, FT>(tO, sP, sL, sOnes);
             }
             umma_commit(&bars->emptyL[eL]);
             if (needV) { umma_commit(&bars->emptyV[eV]); ++nv; }
@@ -375,7 +384,12 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             tc_fence_after();
             const uint32_t sE = sE0 + eE * kSlot, sL = sL0 + eL * kSlot;
             // R: A = aR (E ring), B = K (L ring).  L: A = Qb (L ring), B = aL (E ring).
-            issue_scores<B, FMT>(tmem + a * 256, t.isR ? sE : sL, t.isR ? sL : sE);
+            if (t.isR) {
+              if (t.first) issue_scores<B, FT, FT>(tmem + a * 256, sE, sL);   // A = Q
+              else issue_scores<B, FS, FT>(tmem + a * 256, sE, sL);           // A = alpha_R
+            } else {
+              issue_scores<B, FT, FS>(tmem + a * 256, sL, sE);                // A = Qb, B = alpha_L
+            }
             umma_commit(&bars->emptyE[eE]);
             umma_commit(&bars->s_ready[a]);
             stamp(P, i1, 1);
@@ -404,11 +418,13 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
     const int sub = warp & 3;                  // TMEM sub-partition this warp may access
     const int t_row = sub * 32 + lane;         // TMEM lane = score row owned by this thread
     const int tile = Geo<B>::tile(t_row), r = Geo<B>::row(t_row), srow = tile * B + r;
+    const int sb = r / SB, rb = r - sb * SB;     // block inside the MMA tile, row inside the block
+    const int blk = tile * NSUB + sb;            // block inside the CTA's 128 rows
     const uint32_t tS = tmem + w * 256 + ((uint32_t)(sub * 32) << 16);
     const uint32_t tO = tS + 128;
     uint8_t* sP = smem + Lay::P + w * 2 * kSlot;
 
-    TileIter it(P, first_g + w * stride_g, 2 * stride_g, kTiles);
+    TileIter it(P, first_g + w * stride_g, 2 * stride_g, kBlocks);
     for (int n = w; n < n_total; n += 2, it.next()) {
       const Tile t = it.get();
       const int q = n >> 1, eL = n % kRingL;
@@ -422,21 +438,23 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       // half-step): every such tile is read exactly once, so its lines are dropped from L2 instead
       // of being written back to HBM later.
       if (t.isR) {
-        if (!t.first) discard_line(P.aR + ((size_t)(t.h * m + t.idx0) * B + t_row) * 128);
+        if (!t.first) discard_line(P.aR + ((size_t)(t.h * m + t.idx0) * SB + t_row) * 128);
       } else {
-        discard_line(P.aL + ((size_t)(t.h * B + t.idx0) * m + t_row) * 128);
+        discard_line(P.aL + ((size_t)(t.h * SB + t.idx0) * m + t_row) * 128);
       }
 
       // The row is walked in 32-column chunks read from tensor memory, the next chunk being
       // fetched while the current one is processed, so that a row never has to sit in registers.
       // Arithmetic runs on packed fp32 pairs; exponentials are ex2 with log2(e) folded in.
       constexpr int NC = B / 32;
+      // chunk c holds columns of this row's own block (always, when a block fills the MMA tile)
+      auto mine = [&](int c) { return SB == B || (32 * c) / SB == sb; };
       float buf[32];
       float f, inv_s, mx, sum, sz = 0.f;
       size_t crow = 0;
       float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
       float2 a2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-      const float* cvt = cv + tile * B;        // L: -c_L[j, :] in log2 units
+      const float* cvt = cv + blk * SB;        // L: -c_L[j, :] in log2 units for this row's block
       if (t.isR) {
         // Z_R = scale * S / c_R (Eq. 7); c_L = sum R log R (Eq. 10)
         float inv_c = 1.f;
@@ -445,9 +463,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
           inv_c = c > 1e-30f ? 1.f / c : 0.f;
         }
         f = P.scale * inv_c * kLog2e;
-        crow = ((size_t)t.h * B + r) * m + t.idx0 + tile;      // c_L is stored [h][j][k]
+        crow = ((size_t)t.h * SB + rb) * m + t.idx0 + blk;     // c_L is stored [h][j][k]
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
+          if (!mine(c)) continue;
           tmem_ld32(tS + 32 * c, buf);
           tmem_ld_wait();
 #pragma unroll
@@ -462,9 +481,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
         if (lane == 0 && sub == 0) stamp(P, n, 7);
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
+          float* s = buf;
+          if (mine(c)) {
           tmem_ld32(tS + 32 * c, buf);
           tmem_ld_wait();
-          float* s = buf;
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const float2 sv = make_float2(s[2 * i], s[2 * i + 1]);
@@ -475,7 +495,11 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             s[2 * i] = pp.x;
             s[2 * i + 1] = pp.y;
           }
-          store_row32<T>(sP, srow, 32 * c, s);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) s[i] = 0.f;
+          }
+          store_row32<S>(sP, srow, 32 * c, s);
           if (c == NC / 2 - 1) {    // first half of the row's P is written: MMA 2 may start on it
             fence_proxy_async();
             mbar_arrive(&bars->p_half[w]);
@@ -490,9 +514,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
         const float2 f2 = make_float2(f, f);
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
+          if (!mine(c)) continue;
           tmem_ld32(tS + 32 * c, buf);
           tmem_ld_wait();
-          const float4* cv4 = reinterpret_cast<const float4*>(cvt + 32 * c);
+          const float4* cv4 = reinterpret_cast<const float4*>(cvt + 32 * c - sb * SB);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const float4 cc = cv4[i];
@@ -510,10 +535,11 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
         if (lane == 0 && sub == 0) stamp(P, n, 7);
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
+          float* s = buf;
+          if (mine(c)) {
           tmem_ld32(tS + 32 * c, buf);
           tmem_ld_wait();
-          float* s = buf;
-          const float4* cv4 = reinterpret_cast<const float4*>(cvt + 32 * c);
+          const float4* cv4 = reinterpret_cast<const float4*>(cvt + 32 * c - sb * SB);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const float4 cc = cv4[i];
@@ -530,7 +556,11 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             s[4 * i + 2] = pb.x;
             s[4 * i + 3] = pb.y;
           }
-          store_row32<T>(sP, srow, 32 * c, s);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) s[i] = 0.f;
+          }
+          store_row32<S>(sP, srow, 32 * c, s);
           if (c == NC / 2 - 1 && t.final_) {    // first half of the row's P is written: MMA 2 may start on it
             fence_proxy_async();
             mbar_arrive(&bars->p_half[w]);
@@ -551,8 +581,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
             uint32_t* qp = reinterpret_cast<uint32_t*>(&qv);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const float2 v = fmul2(unpack2<T>(qp[e]), is2);
-              qp[e] = pack2<T>(v.x, v.y);
+              const float2 v = fmul2(unpack2<S>(qp[e]), is2);
+              qp[e] = pack2<S>(v.x, v.y);
             }
             *ptr = qv;
           }
@@ -569,7 +599,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       wait_or_abort(&bars->o_ready[w], q & 1, bars, P.status, 31);
       tc_fence_after();
       if (lane == 0 && sub == 0) stamp(P, n, 5);
-      if (t.final_) discard_line(P.y + ((size_t)(t.h * B + t.idx0) * m + t_row) * 128);   // y: read once
+      if (t.final_) discard_line(P.y + ((size_t)(t.h * SB + t.idx0) * m + t_row) * 128);   // y: read once
       const int nco = (t.isR && t.withV) ? 4 : 2;            // 32-column chunks of O
       const bool scaled = t.isR || t.final_;
       float c1 = 0.f;
@@ -579,13 +609,14 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
         if (c < nco) {
           tmem_ld32(tO + 32 * c, buf);
           tmem_ld_wait();
-          if (scaled) store_row32<T>(sP, srow, 32 * c, buf, inv_s);
-          else store_row32<T>(sP, srow, 32 * c, buf);
+          if (t.final_) store_row32<T>(sP, srow, 32 * c, buf, inv_s);       // Y: the caller's type
+          else if (scaled) store_row32<S>(sP, srow, 32 * c, buf, inv_s);
+          else store_row32<S>(sP, srow, 32 * c, buf);
         }
       }
       tc_fence_before();
       mbar_arrive(&bars->o_free[w]);
-      if (!t.isR && !t.final_) P.cR[((size_t)t.h * m + r) * B + t.idx0 + tile] = c1;
+      if (!t.isR && !t.final_) P.cR[((size_t)t.h * m + rb) * SB + t.idx0 + blk] = c1;
       fence_proxy_async();
       mbar_arrive(&bars->stage_ready[w]);
       if (lane == 0 && sub == 0) stamp(P, n, 6);
@@ -596,17 +627,17 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       const int w = warp - 10;
       const uint8_t* sP = smem + Lay::P + w * 2 * kSlot;
       const uint64_t pol_first = policy_evict_first();
-      TileIter it(P, first_g + w * stride_g, 2 * stride_g, kTiles);
+      TileIter it(P, first_g + w * stride_g, 2 * stride_g, kBlocks);
       for (int n = w; n < n_total; n += 2, it.next()) {
         const Tile t = it.get();
         const int q = n >> 1;
         wait_or_abort(&bars->stage_ready[w], q & 1, bars, P.status, 40);
 #pragma unroll
-        for (int tt = 0; tt < kTiles; ++tt) {
-          const uint8_t* src = sP + tt * (B * 128);
+        for (int tt = 0; tt < kBlocks; ++tt) {
+          const uint8_t* src = sP + tt * (SB * 128);
           if (t.isR) {
-            tma_store_3d(&P.tmALs, src, 0, t.idx0 + tt, t.h * B);
-            if (t.withV) tma_store_3d(&P.tmYs, src + kSlot, 0, t.idx0 + tt, t.h * B);
+            tma_store_3d(&P.tmALs, src, 0, t.idx0 + tt, t.h * SB);
+            if (t.withV) tma_store_3d(&P.tmYs, src + kSlot, 0, t.idx0 + tt, t.h * SB);
           } else {
             if (t.final_) tma_store_3d_hint(&P.tmOut, src, 0, t.idx0 + tt, t.h * m, pol_first);
             else tma_store_3d(&P.tmARs, src, 0, t.idx0 + tt, t.h * m);
@@ -648,6 +679,14 @@ inline long long*& trace_buffer() {
   static long long* p = nullptr;
   return p;
 }
+// f16/bf16, d = 64, m = b in {32, 64, 128} (b = 32 runs on 64-row MMA tiles, two blocks per tile).
+inline bool supported(int N, int d, int b, int m, int dtype, int BH) {
+  if (dtype != 1 && dtype != 2) return false;
+  if (d != kD || b != m) return false;
+  if (b != 32 && b != 64 && b != 128) return false;
+  if ((long long)BH * N >= (1LL << 31)) return false;
+  return true;
+}
 inline size_t counters_bytes(int BH, int T) {
   return ((size_t)2 * T * BH * sizeof(int) + 255) / 256 * 256;
 }
@@ -655,29 +694,29 @@ inline size_t workspace_bytes(int BH, int N, int T) {
   return ws_layout(nullptr, BH, N).bytes + counters_bytes(BH, T);
 }
 
-template <typename T, int B>
+template <typename T, int B, int SB>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int T_steps,
                     int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
                     bool ws_armed) {
   const Ws w = ws_layout(ws, BH, N);
   int* counters = (int*)((char*)ws + w.bytes);
-  const int m = N / B;
+  const int m = N / SB;            // = SB on this path
   const uint64_t rows = (uint64_t)BH * N;
   Params P;
   bool ok = make_map_rows(&P.tmQ, dtype, (void*)Q, rows) && make_map_rows(&P.tmK, dtype, (void*)K, rows) &&
             make_map_rows(&P.tmV, dtype, (void*)V, rows) && make_map_rows(&P.tmAR, dtype, w.aR, rows) &&
             make_map_rows(&P.tmAL, dtype, w.aL, rows) && make_map_rows(&P.tmY, dtype, w.y, rows) &&
-            make_map_strided(&P.tmALs, dtype, w.aL, m, (uint64_t)BH * B, B) &&
-            make_map_strided(&P.tmYs, dtype, w.y, m, (uint64_t)BH * B, B) &&
-            make_map_strided(&P.tmQs, dtype, (void*)Q, B, (uint64_t)BH * m, B) &&
-            make_map_strided(&P.tmARs, dtype, w.aR, B, (uint64_t)BH * m, B) &&
-            make_map_strided(&P.tmOut, dtype, Y, B, (uint64_t)BH * m, B);
+            make_map_strided(&P.tmALs, dtype, w.aL, m, (uint64_t)BH * SB, SB) &&
+            make_map_strided(&P.tmYs, dtype, w.y, m, (uint64_t)BH * SB, SB) &&
+            make_map_strided(&P.tmQs, dtype, (void*)Q, SB, (uint64_t)BH * m, SB) &&
+            make_map_strided(&P.tmARs, dtype, w.aR, SB, (uint64_t)BH * m, SB) &&
+            make_map_strided(&P.tmOut, dtype, Y, SB, (uint64_t)BH * m, SB);
   if (!ok) return 7;
   P.aL = (uint8_t*)w.aL; P.aR = (uint8_t*)w.aR; P.y = (uint8_t*)w.y;
   P.cL = w.cL; P.cR = w.cR; P.status = w.status; P.counters = counters;
   P.trace = trace_buffer();
   P.m = m; P.BH = BH; P.T = T_steps;
-  P.tiles_per_head = m / Geo<B>::kTiles;
+  P.tiles_per_head = m / (kRows / SB);
   P.tiles_per_phase = BH * P.tiles_per_head;
   P.scale = scale;
   P.n_counters = 2 * T_steps * BH;
@@ -691,7 +730,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
     cudaGetDevice(&dev);
     if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 7;
   }
-  const void* fn = (const void*)monarch_persistent<T, B>;
+  const void* fn = (const void*)monarch_persistent<T, B, SB>;
   if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
     return 7;
   const int total = 2 * T_steps * P.tiles_per_phase;
@@ -699,14 +738,14 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   if (mode == 0) {          // one launch, dependencies tracked by counters
     P.g_begin = 0; P.g_end = total; P.check_deps = 1;
     const int grid = total < num_sms ? total : num_sms;
-    monarch_persistent<T, B><<<grid, kThreads, kSmem, st>>>(P);
+    monarch_persistent<T, B, SB><<<grid, kThreads, kSmem, st>>>(P);
     n = 1;
   } else {                  // one launch per half-step (stream order is the dependency)
     P.check_deps = 0;
     for (int p = 0; p < 2 * T_steps; ++p) {
       P.g_begin = p * P.tiles_per_phase; P.g_end = P.g_begin + P.tiles_per_phase;
       const int grid = P.tiles_per_phase < num_sms ? P.tiles_per_phase : num_sms;
-      monarch_persistent<T, B><<<grid, kThreads, kSmem, st>>>(P);
+      monarch_persistent<T, B, SB><<<grid, kThreads, kSmem, st>>>(P);
       ++n;
     }
   }
@@ -718,13 +757,16 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
 inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int b, int T,
                   int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
                   bool ws_armed) {
+#define MA_TP_ARGS Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed
   if (dtype == 1) {
-    if (b == 128) return launch_t<__half, 128>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed);
-    return launch_t<__half, 64>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed);
+    if (b == 128) return launch_t<__half, 128, 128>(MA_TP_ARGS);
+    if (b == 64) return launch_t<__half, 64, 64>(MA_TP_ARGS);
+    return launch_t<__half, 64, 32>(MA_TP_ARGS);
   }
-  if (b == 128)
-    return launch_t<__nv_bfloat16, 128>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed);
-  return launch_t<__nv_bfloat16, 64>(Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed);
+  if (b == 128) return launch_t<__nv_bfloat16, 128, 128>(MA_TP_ARGS);
+  if (b == 64) return launch_t<__nv_bfloat16, 64, 64>(MA_TP_ARGS);
+  return launch_t<__nv_bfloat16, 64, 32>(MA_TP_ARGS);
+#undef MA_TP_ARGS
 }
 
 }  // namespace tp

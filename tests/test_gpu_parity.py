@@ -107,6 +107,14 @@ def test_tensor_paths_match_oracle(N, b, T, dtype, batch, heads, path):
     check(batch, heads, N, 64, b, T, dtype, rank=16, s=1.5, seed=N + T + heads, path=path)
 
 
+@pytest.mark.parametrize("path", [binding.MA_PATH_TENSOR, binding.MA_PATH_TENSOR_PHASED])
+@pytest.mark.parametrize("T,dtype,batch,heads", [(1, "bf16", 1, 1), (2, "bf16", 2, 3), (3, "f16", 1, 5),
+                                                  (2, "f16", 19, 1)])
+def test_tensor_path_block_32_on_64_row_tiles(T, dtype, batch, heads, path):
+    """b = m = 32 (N = 1024): two blocks share one 64-row MMA tile, off-diagonal P is zero."""
+    check(batch, heads, 1024, 64, 32, T, dtype, rank=16, s=1.5, seed=3 * T + heads, path=path)
+
+
 def test_tensor_paths_agree_bit_for_bit_between_launch_modes():
     """One persistent launch with dependency counters computes exactly what one launch per
     half-step computes (same kernel, same tile order inside a half-step)."""
