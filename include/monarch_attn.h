@@ -130,6 +130,14 @@ int monarch_attn_last_launch_count(void);
  * the buffer stays owned by the caller. */
 int monarch_attn_set_trace_buffer(void* device_buffer, size_t bytes);
 
+/* Test knobs of the persistent tensor path (process-wide; not for production use).
+ *   knob 1: bound, in SM clocks, of every device-side wait (value <= 0 restores the default 2e9);
+ *   knob 2: non-zero leaves the first half-step out of later single-launch runs, so that the
+ *           dependency waits of the second half-step can never be satisfied.  Together they let a
+ *           test watch a wait run out: the kernel ends by itself, results are garbage, and
+ *           monarch_attn_device_status reports MA_ERR_TIMEOUT.  Nothing faults or hangs. */
+int monarch_attn_debug_knob(int knob, long long value);
+
 /* Static, NUL-terminated description of an ma_status code. */
 const char* monarch_attn_status_string(int status);
 

@@ -63,6 +63,8 @@ def load_library(path: str = LIB_PATH):
     lib.monarch_attn_device_status.restype = i
     lib.monarch_attn_last_launch_count.argtypes = []
     lib.monarch_attn_last_launch_count.restype = i
+    lib.monarch_attn_debug_knob.argtypes = [i, ctypes.c_longlong]
+    lib.monarch_attn_debug_knob.restype = i
     lib.monarch_attn_set_trace_buffer.argtypes = [vp, sz]
     lib.monarch_attn_set_trace_buffer.restype = i
     lib.monarch_attn_status_string.argtypes = [i]
@@ -188,6 +190,10 @@ def monarch_attn_set_trace_buffer(buf=None):
         _check(lib.monarch_attn_set_trace_buffer(None, 0))
     else:
         _check(lib.monarch_attn_set_trace_buffer(buf.data_ptr(), buf.numel() * buf.element_size()))
+
+
+def monarch_attn_debug_knob(knob: int, value: int):
+    _check(load_library().monarch_attn_debug_knob(int(knob), int(value)))
 
 
 def torch_dtype(name: str) -> torch.dtype:

@@ -359,6 +359,18 @@ int monarch_attn_fwd_noalloc(const void* Q, const void* K, const void* V, void* 
                         (cudaStream_t)stream);
 }
 
+int monarch_attn_debug_knob(int knob, long long value) {
+  if (knob == 1) {
+    tp::knobs().wait_cycles = value > 0 ? value : tensor::kWaitCycles;
+  } else if (knob == 2) {
+    tp::knobs().skip_first_half_step = value != 0;
+  } else {
+    return MA_ERR_SHAPE;
+  }
+  for (int d = 0; d < kMaxDevices; ++d) g_dev[d].armed_key = -1;
+  return MA_OK;
+}
+
 int monarch_attn_set_trace_buffer(void* device_buffer, size_t bytes) {
   if (device_buffer != nullptr && bytes < (size_t)4 * 64 * 8 * sizeof(long long)) return MA_ERR_WORKSPACE;
   tp::trace_buffer() = (long long*)device_buffer;

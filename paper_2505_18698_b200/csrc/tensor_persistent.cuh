@@ -55,6 +55,7 @@ struct __align__(8) Bars {
   uint64_t s_ready[2], p_half[2], p_ready[2], o_ready[2], o_free[2], stage_ready[2], stage_free[2];
   uint32_t tmem_slot;
   volatile int abort_flag;
+  long long wait_limit;   // clocks a wait may take before it gives up
 };
 
 struct Params {
@@ -73,6 +74,7 @@ struct Params {
   int g_begin, g_end;  // tile range of this launch
   int check_deps;
   int n_counters;      // 2T * BH
+  long long wait_cycles;
   float scale;
 };
 
@@ -126,7 +128,7 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Ba
         : "memory");
     if (done) return true;
     if (bars->abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > bars->wait_limit) {
       report_timeout(status, where);
       bars->abort_flag = 1;
       return false;
@@ -217,6 +219,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
       mbar_init(&bars->stage_free[i], 1);
     }
     bars->abort_flag = 0;
+    bars->wait_limit = P.wait_cycles;
     fence_barrier_init();
     fence_proxy_async();
   }
@@ -311,7 +314,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
         } else if (!force) {
           if (bars->abort_flag) {
             force = true;
-          } else if (clock64() - t0 > kWaitCycles) {
+          } else if (clock64() - t0 > P.wait_cycles) {
             report_timeout(P.status, 10);
             bars->abort_flag = 1;
             force = true;
@@ -403,7 +406,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
         } else if (!force) {
           if (bars->abort_flag) {
             force = true;
-          } else if (clock64() - t0 > kWaitCycles) {
+          } else if (clock64() - t0 > P.wait_cycles) {
             report_timeout(P.status, 20);
             bars->abort_flag = 1;
             force = true;
@@ -675,6 +678,16 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_persistent(const __grid_c
 }
 
 // ------------------------------------------------------------------------------------ host side
+// Test knobs (process-wide): bound of the device-side waits, and a switch that leaves the first
+// half-step out of a single-launch run so that every dependency wait of the second runs out.
+struct DebugKnobs {
+  long long wait_cycles = kWaitCycles;
+  int skip_first_half_step = 0;
+};
+inline DebugKnobs& knobs() {
+  static DebugKnobs k;
+  return k;
+}
 inline long long*& trace_buffer() {
   static long long* p = nullptr;
   return p;
@@ -720,6 +733,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   P.tiles_per_phase = BH * P.tiles_per_head;
   P.scale = scale;
   P.n_counters = 2 * T_steps * BH;
+  P.wait_cycles = knobs().wait_cycles;
   if (!ws_armed) {   // status block and counters start at zero; the kernel leaves them that way
     if (cudaMemsetAsync(ws, 0, kWsStatusBytes, st) != cudaSuccess) return 7;
     if (cudaMemsetAsync(counters, 0, counters_bytes(BH, T_steps), st) != cudaSuccess) return 7;
@@ -736,7 +750,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   const int total = 2 * T_steps * P.tiles_per_phase;
   int n = 0;
   if (mode == 0) {          // one launch, dependencies tracked by counters
-    P.g_begin = 0; P.g_end = total; P.check_deps = 1;
+    P.g_begin = knobs().skip_first_half_step ? P.tiles_per_phase : 0; P.g_end = total; P.check_deps = 1;
     const int grid = total < num_sms ? total : num_sms;
     monarch_persistent<T, B, SB><<<grid, kThreads, kSmem, st>>>(P);
     n = 1;

@@ -247,3 +247,28 @@ def test_unsupported_and_error_paths_on_device():
     with pytest.raises(binding.MonarchAttnError) as e:
         binding.monarch_attn_fwd(x, x, x, b=15, T=1)
     assert e.value.code == 2
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """Failure detection without a fault: with the first half-step left out, the dependency
+    counters the second half-step waits for are never filled; every wait is bounded, so the kernel
+    ends by itself and the status word says so.  The context stays usable."""
+    Q, K, V = wl.make_qkv(1, 2, 4096, 64, "bf16", 16, 1.5, seed=61)
+    Qd, Kd, Vd = (binding.to_device(x, "bf16") for x in (Q, K, V))
+    need = binding.monarch_attn_workspace_bytes(1, 2, 4096, 64, 64, 2, Qd.dtype, binding.MA_PATH_TENSOR)
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    try:
+        binding.monarch_attn_debug_knob(1, 2_000_000)      # ~1 ms per wait
+        binding.monarch_attn_debug_knob(2, 1)
+        binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 64, 2, path=binding.MA_PATH_TENSOR, workspace=ws)
+        torch.cuda.synchronize()
+        assert binding.monarch_attn_device_status(ws) == 8
+    finally:
+        binding.monarch_attn_debug_knob(2, 0)
+        binding.monarch_attn_debug_knob(1, 0)
+    ws.zero_()
+    Y = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 64, 2, path=binding.MA_PATH_TENSOR, workspace=ws)
+    torch.cuda.synchronize()
+    assert binding.monarch_attn_device_status(ws) == 0
+    ref = mo.monarch_attention(Q, K, V, 64, 2)
+    assert rel_err(Y.float().cpu().numpy().astype(np.float64), ref) <= 1e-2
