@@ -98,6 +98,16 @@ __device__ __forceinline__ void ldsm_x2_trans(uint32_t* b, uint32_t saddr) {
                : "=r"(b[0]), "=r"(b[1])
                : "r"(saddr));
 }
+__device__ __forceinline__ void ldsm_x4(uint32_t* r, uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(saddr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t* r, uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(saddr));
+}
 __device__ __forceinline__ uint32_t movm_trans(uint32_t a) {
   uint32_t d;
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
@@ -187,6 +197,8 @@ monarch_fused_n256(const TIn* __restrict__ Q, const TIn* __restrict__ K, const T
     const bool first = step == 1, last = step == T_steps;
     // ================================================================ R half-step (Eq. 7, 9, 10)
     const uint8_t* sA = first ? sQ : sAR;          // alpha_R[k][j][:] (= Q rows when L = identity)
+    const uint32_t sA_u = (uint32_t)__cvta_generic_to_shared(sA);
+    const uint32_t sK_u = sQ_u + kTile, sV_u = sQ_u + 2 * kTile;
     uint32_t outL[2][8][2], outY[2][8][2];          // packed alpha_L / y rows g and g+8, per v block
 #pragma unroll
     for (int kt = 0; kt < 2; ++kt) {
@@ -194,18 +206,13 @@ monarch_fused_n256(const TIn* __restrict__ Q, const TIn* __restrict__ K, const T
       float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks) {
-        uint32_t a[4];
-        a[0] = lds32(sA, swz(r0 + g, 16 * ks + 2 * t));
-        a[1] = lds32(sA, swz(r0 + g + 8, 16 * ks + 2 * t));
-        a[2] = lds32(sA, swz(r0 + g, 16 * ks + 2 * t + 8));
-        a[3] = lds32(sA, swz(r0 + g + 8, 16 * ks + 2 * t + 8));
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-          uint32_t b[2];
-          b[0] = lds32(sK, swz(r0 + 8 * nt + g, 16 * ks + 2 * t));
-          b[1] = lds32(sK, swz(r0 + 8 * nt + g, 16 * ks + 2 * t + 8));
-          Mma<T>::run(s[nt], a, b);
-        }
+        // A: 16 rows x 16 k as four 8x8 matrices (rows 0-7 / 8-15, k 0-7 / 8-15), one ldmatrix;
+        // B: both 8-column tiles of K (stored [i][v]) likewise.
+        uint32_t a[4], b[4];
+        ldsm_x4(a, sA_u + swz(r0 + (lane & 7) + ((lane >> 3) & 1) * 8, 16 * ks + (lane >> 4) * 8));
+        ldsm_x4(b, sK_u + swz(r0 + (lane & 7) + (lane >> 4) * 8, 16 * ks + ((lane >> 3) & 1) * 8));
+        Mma<T>::run(s[0], a, b);
+        Mma<T>::run(s[1], a, b + 2);
       }
       // rows j = g (c0, c1) and j = g + 8 (c2, c3); columns i = 8 nt + 2t, +1
       float inv_s[2], pa_f[2][4];
@@ -233,21 +240,26 @@ monarch_fused_n256(const TIn* __restrict__ Q, const TIn* __restrict__ K, const T
       pa[1] = Mma<T>::pack(pa_f[1][0], pa_f[1][1]);
       pa[2] = Mma<T>::pack(pa_f[0][2], pa_f[0][3]);
       pa[3] = Mma<T>::pack(pa_f[1][2], pa_f[1][3]);
-      const uint32_t sK_u = sQ_u + kTile, sV_u = sQ_u + 2 * kTile;
 #pragma unroll
-      for (int nt = 0; nt < 8; ++nt) {
-        float o[4] = {0.f, 0.f, 0.f, 0.f};
-        uint32_t b[2];
-        ldsm_x2_trans(b, sK_u + swz(r0 + (lane & 15), 8 * nt));
-        Mma<T>::run(o, pa, b);
-        outL[kt][nt][0] = Mma<T>::pack(o[0] * inv_s[0], o[1] * inv_s[0]);
-        outL[kt][nt][1] = Mma<T>::pack(o[2] * inv_s[1], o[3] * inv_s[1]);
+      for (int np = 0; np < 4; ++np) {     // two 8-column tiles of v per transposing ldmatrix
+        uint32_t b[4];
+        ldsm_x4_trans(b, sK_u + swz(r0 + (lane & 15), 16 * np + (lane >> 4) * 8));
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          float o[4] = {0.f, 0.f, 0.f, 0.f};
+          Mma<T>::run(o, pa, b + 2 * q);
+          outL[kt][2 * np + q][0] = Mma<T>::pack(o[0] * inv_s[0], o[1] * inv_s[0]);
+          outL[kt][2 * np + q][1] = Mma<T>::pack(o[2] * inv_s[1], o[3] * inv_s[1]);
+        }
         if (last) {
-          float y[4] = {0.f, 0.f, 0.f, 0.f};
-          ldsm_x2_trans(b, sV_u + swz(r0 + (lane & 15), 8 * nt));
-          Mma<T>::run(y, pa, b);
-          outY[kt][nt][0] = Mma<T>::pack(y[0] * inv_s[0], y[1] * inv_s[0]);
-          outY[kt][nt][1] = Mma<T>::pack(y[2] * inv_s[1], y[3] * inv_s[1]);
+          ldsm_x4_trans(b, sV_u + swz(r0 + (lane & 15), 16 * np + (lane >> 4) * 8));
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            float y[4] = {0.f, 0.f, 0.f, 0.f};
+            Mma<T>::run(y, pa, b + 2 * q);
+            outY[kt][2 * np + q][0] = Mma<T>::pack(y[0] * inv_s[0], y[1] * inv_s[0]);
+            outY[kt][2 * np + q][1] = Mma<T>::pack(y[2] * inv_s[1], y[3] * inv_s[1]);
+          }
         }
       }
     }
@@ -270,25 +282,18 @@ monarch_fused_n256(const TIn* __restrict__ Q, const TIn* __restrict__ K, const T
 
     // ================================================================ L half-step (Eq. 8, 9 / Eq. 4)
     const uint32_t sAL_u = (uint32_t)__cvta_generic_to_shared(sAL);
-    (void)sAL_u;
 #pragma unroll
     for (int jt = 0; jt < 2; ++jt) {
       const int j = 2 * warp + jt;
       float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks) {
-        uint32_t a[4];   // rows l = g, g+8 of Qb[j]: tile rows 16 l + j
-        a[0] = lds32(sQ, swz(16 * g + j, 16 * ks + 2 * t));
-        a[1] = lds32(sQ, swz(16 * (g + 8) + j, 16 * ks + 2 * t));
-        a[2] = lds32(sQ, swz(16 * g + j, 16 * ks + 2 * t + 8));
-        a[3] = lds32(sQ, swz(16 * (g + 8) + j, 16 * ks + 2 * t + 8));
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-          uint32_t b[2];   // alpha_L[j][k = 8 nt + g][:]
-          b[0] = lds32(sAL, swz(16 * j + 8 * nt + g, 16 * ks + 2 * t));
-          b[1] = lds32(sAL, swz(16 * j + 8 * nt + g, 16 * ks + 2 * t + 8));
-          Mma<T>::run(s[nt], a, b);
-        }
+        // A: rows l of Qb[j] are tile rows 16 l + j; B: alpha_L[j][k][:] rows 16 j + k
+        uint32_t a[4], b[4];
+        ldsm_x4(a, sQ_u + swz(16 * ((lane & 7) + ((lane >> 3) & 1) * 8) + j, 16 * ks + (lane >> 4) * 8));
+        ldsm_x4(b, sAL_u + swz(16 * j + (lane & 7) + (lane >> 4) * 8, 16 * ks + ((lane >> 3) & 1) * 8));
+        Mma<T>::run(s[0], a, b);
+        Mma<T>::run(s[1], a, b + 2);
       }
       // rows l = g, g + 8; columns k = 8 nt + 2t, +1.  Z_L = scale * S' - c_L[j][k]
       const float c0 = sCL[j * 16 + 2 * t] * kLog2e, c1 = sCL[j * 16 + 2 * t + 1] * kLog2e;
@@ -309,16 +314,18 @@ monarch_fused_n256(const TIn* __restrict__ Q, const TIn* __restrict__ K, const T
         pa[1] = Mma<T>::pack(p[1][0], p[1][1]);
         pa[2] = Mma<T>::pack(p[0][2], p[0][3]);
         pa[3] = Mma<T>::pack(p[1][2], p[1][3]);
-        const uint32_t sV_u = sQ_u + 2 * kTile;
         uint32_t out[8][2];
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-          float o[4] = {0.f, 0.f, 0.f, 0.f};
-          uint32_t b[2];
-          ldsm_x2_trans(b, sV_u + swz(16 * j + (lane & 15), 8 * nt));
-          Mma<T>::run(o, pa, b);
-          out[nt][0] = Mma<T>::pack(o[0] * inv_s[0], o[1] * inv_s[0]);
-          out[nt][1] = Mma<T>::pack(o[2] * inv_s[1], o[3] * inv_s[1]);
+        for (int np = 0; np < 4; ++np) {
+          uint32_t b[4];
+          ldsm_x4_trans(b, sV_u + swz(16 * j + (lane & 15), 16 * np + (lane >> 4) * 8));
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            float o[4] = {0.f, 0.f, 0.f, 0.f};
+            Mma<T>::run(o, pa, b + 2 * q);
+            out[2 * np + q][0] = Mma<T>::pack(o[0] * inv_s[0], o[1] * inv_s[0]);
+            out[2 * np + q][1] = Mma<T>::pack(o[2] * inv_s[1], o[3] * inv_s[1]);
+          }
         }
         // only this warp reads the rows 16 l + j of Q, and it has: Y takes their place
         __syncwarp();
