@@ -45,10 +45,13 @@ typedef enum {
   MA_PATH_AUTO = 0,
   MA_PATH_GENERIC = 1, /* fp32 SIMT kernels, fp32 states; any dtype, any N = m*b that fits smem */
   MA_PATH_TENSOR = 2,  /* tcgen05/TMA kernels, 16-bit states; f16/bf16, d = 64, m = b in
-                          {32, 64, 128}: one persistent launch for all 2T half-steps */
-  MA_PATH_TENSOR_PHASED = 3, /* the same persistent kernel, one launch per half-step */
+                          {32, 64, 128}: one persistent launch for all 2T half-steps (softmax and
+                          epilogue in separate warpgroups) */
+  MA_PATH_TENSOR_PHASED = 3, /* first-generation persistent kernel, one launch per half-step */
   MA_PATH_TENSOR_BASIC = 4,  /* one CTA per tile, one launch per half-step (no pipelining);
                                 m = b in {64, 128} */
+  MA_PATH_TENSOR_CHAINED = 6, /* first-generation persistent kernel (each softmax warpgroup also
+                                 does its tile's epilogue), one launch; kept for comparison */
   MA_PATH_FUSED = 5    /* one CTA per (batch, head), everything in shared memory, one launch:
                           f16/bf16, N = 256, m = b = 16, d = 64 */
 } ma_path;

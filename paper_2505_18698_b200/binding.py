@@ -20,6 +20,7 @@ HEADER_PATH = os.path.join(os.path.dirname(_PKG_DIR), "include", "monarch_attn.h
 MA_F32, MA_F16, MA_BF16 = 0, 1, 2
 MA_PATH_AUTO, MA_PATH_GENERIC, MA_PATH_TENSOR, MA_PATH_TENSOR_PHASED, MA_PATH_TENSOR_BASIC = 0, 1, 2, 3, 4
 MA_PATH_FUSED = 5
+MA_PATH_TENSOR_CHAINED = 6
 MA_OK = 0
 
 _TORCH_TO_CODE = {torch.float32: MA_F32, torch.float16: MA_F16, torch.bfloat16: MA_BF16}

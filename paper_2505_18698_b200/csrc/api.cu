@@ -11,6 +11,7 @@
 #include "generic_kernels.cuh"
 #include "tensor_path.cuh"
 #include "tensor_persistent.cuh"
+#include "tensor_decoupled.cuh"
 #include "fused_n256.cuh"
 
 namespace ma {
@@ -141,7 +142,7 @@ static int resolve_path(const Problem& p, int path) {
   }
   if (path == MA_PATH_GENERIC) return generic_supported(p) ? path : -1;
   if (path == MA_PATH_FUSED) return fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
-  if (path == MA_PATH_TENSOR || path == MA_PATH_TENSOR_PHASED)
+  if (path == MA_PATH_TENSOR || path == MA_PATH_TENSOR_PHASED || path == MA_PATH_TENSOR_CHAINED)
     return tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
   if (path == MA_PATH_TENSOR_BASIC)
     return tensor::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
@@ -152,7 +153,8 @@ static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
   if (resolved == MA_PATH_FUSED) return kStatusBytes;   // no states leave the chip
   if (resolved == MA_PATH_TENSOR_BASIC) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
-  if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_PHASED)
+  if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_PHASED ||
+      resolved == MA_PATH_TENSOR_CHAINED)
     return tp::workspace_bytes(p.BH, p.N, p.T);
   return 0;
 }
@@ -203,7 +205,8 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
     rc = tensor::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.T, p.dtype, scale, ws, st, &launches);
   else
     rc = tp::launch(Q, K, V, Y, p.BH, p.N, p.b, p.T, p.dtype, scale, ws, st, &launches,
-                    resolved == MA_PATH_TENSOR ? 0 : 1, ws_armed);
+                    resolved == MA_PATH_TENSOR ? 0 : (resolved == MA_PATH_TENSOR_PHASED ? 1 : 2),
+                    ws_armed);
   if (rc == MA_OK) g_last_launches = launches;
   return rc;
 }

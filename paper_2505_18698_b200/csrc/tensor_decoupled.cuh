@@ -1,0 +1,597 @@
+// Persistent tensor-core kernel, second generation: the epilogue has warps of its own.
+//
+// Same tiles, same order, same dependency counters, same MMAs as `monarch_persistent`
+// (tensor_persistent.cuh); what changes is who waits for what.  There a softmax warpgroup walked
+// the whole chain of a tile (scores -> softmax -> wait for the apply MMA -> epilogue -> wait for
+// the next scores), about 2.8 us of mostly latency, and two such chains were all that tensor
+// memory and shared memory allow.  Here
+//   * two softmax warpgroups do nothing but S -> P (alternate tiles); S has three TMEM stages,
+//     so the score MMA runs up to three tiles ahead and a group never waits for it;
+//   * a third warpgroup does every epilogue (O -> 16-bit rows -> staging), so the softmax groups
+//     never wait for the apply MMA; O has a single TMEM stage, drained as soon as it is ready;
+//   * two store threads alternate tiles (TMA store, completion, dependency counter).
+// 512 threads: warp 0 TMA producer, warp 1 MMA issuer, warps 2-3 store threads, warps 4-7 and
+// 8-11 softmax groups, warps 12-15 epilogue group.
+// TMEM: S0, S1, S2 at columns 0, 128, 256; O at 384.  Shared memory: rings E (2) / L (4) / V (2) of
+// 16 KB operand tiles, two 32 KB P buffers, one 16 KB staging buffer (the last R half-step stages
+// alpha_L and y in two rounds), row statistics, c-vectors, a tile of ones.
+#pragma once
+#include "tensor_persistent.cuh"
+
+namespace ma {
+namespace tp2 {
+
+using namespace ma::tensor;
+using ma::tp::Params;
+using ma::tp::Tile;
+using ma::tp::TileIter;
+using ma::tp::stamp;
+using ma::tp::mbar_test;
+using ma::tp::mbar_arrive;
+using ma::tp::ld_acquire;
+using ma::tp::bulk_load_1d;
+using ma::tp::tmem_ld1;
+using ma::tp::tma_store_commit;
+using ma::tp::tma_store_wait_read;
+using ma::tp::tma_store_wait_all;
+
+constexpr int kThreads = 512;
+constexpr int kRingE = 2, kRingL = 4, kRingV = 2, kStagesS = 3;
+constexpr int kSlot = kTileBytes;
+
+struct Lay {
+  static constexpr int E = 0;
+  static constexpr int L = E + kRingE * kSlot;
+  static constexpr int V = L + kRingL * kSlot;
+  static constexpr int P = V + kRingV * kSlot;          // 2 x 32 KB
+  static constexpr int Stage = P + 4 * kSlot;           // 16 KB
+  static constexpr int Ones = Stage + kSlot;            // 2 KB
+  static constexpr int Vec = Ones + 2048;               // kRingL x 128 floats (c_R / c_L)
+  static constexpr int Stat = Vec + kRingL * 512;       // 4 x 128 floats (1 / row sum)
+  static constexpr int Bars = Stat + 4 * 512;
+  static constexpr int Total = Bars + 512;
+};
+constexpr int kSmem = Lay::Total + 1024;
+
+struct __align__(8) Bars {
+  uint64_t fullE[kRingE], emptyE[kRingE];
+  uint64_t fullL[kRingL], emptyL[kRingL];
+  uint64_t fullV[kRingV], emptyV[kRingV];
+  uint64_t s_ready[kStagesS];
+  uint64_t p_half[2], p_ready[2], p_free[2];
+  uint64_t o_ready, o_free, stage_ready[2], stage_free;
+  uint32_t tmem_slot;
+  volatile int abort_flag;
+  long long wait_limit;
+};
+
+// Bounded wait; see tensor_persistent.cuh (after a timeout every wait of the CTA returns at once).
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Bars* bars, int* status,
+                                              int where) {
+  const uint32_t addr = smem_u32(bar);
+  const long long t0 = clock64();
+  for (;;) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if (bars->abort_flag) return false;
+    if (clock64() - t0 > bars->wait_limit) {
+      report_timeout(status, where);
+      bars->abort_flag = 1;
+      return false;
+    }
+  }
+}
+
+template <typename T, int B, int SB>
+__global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_constant__ Params P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  Bars* bars = reinterpret_cast<Bars*>(smem + Lay::Bars);
+  constexpr int kBlocks = kRows / SB;         // blocks (k of an R tile, j of an L tile) per CTA
+  constexpr int NSUB = B / SB;                // blocks per MMA tile
+  constexpr int FT = Fmt<T>::code;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m = P.m;
+
+  if (tid == 0) {
+    for (int i = 0; i < kRingE; ++i) { mbar_init(&bars->fullE[i], 1); mbar_init(&bars->emptyE[i], 1); }
+    for (int i = 0; i < kRingL; ++i) { mbar_init(&bars->fullL[i], 1); mbar_init(&bars->emptyL[i], 1); }
+    for (int i = 0; i < kRingV; ++i) { mbar_init(&bars->fullV[i], 1); mbar_init(&bars->emptyV[i], 1); }
+    for (int i = 0; i < kStagesS; ++i) mbar_init(&bars->s_ready[i], 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars->p_half[i], 128);
+      mbar_init(&bars->p_ready[i], 128);
+      mbar_init(&bars->p_free[i], 1);
+    }
+    mbar_init(&bars->o_ready, 1);
+    mbar_init(&bars->o_free, 128);
+    mbar_init(&bars->stage_ready[0], 128);
+    mbar_init(&bars->stage_ready[1], 128);
+    mbar_init(&bars->stage_free, 1);
+    bars->abort_flag = 0;
+    bars->wait_limit = P.wait_cycles;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (tid < 128) {   // tile of ones for the column-sum MMA of the non-final L half-step
+    const uint32_t one2 = pack2<T>(1.f, 1.f);
+    *reinterpret_cast<uint4*>(smem + Lay::Ones + tid * 16) = make_uint4(one2, one2, one2, one2);
+  }
+  if (warp == 0) tmem_alloc(&bars->tmem_slot, 512);
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_slot;
+  const uint32_t tmem_o = tmem + 384;
+
+  const int first_g = P.g_begin + blockIdx.x;
+  const int stride_g = gridDim.x;
+  const int n_total = first_g < P.g_end ? (P.g_end - first_g + stride_g - 1) / stride_g : 0;
+  auto needs_v = [&](const Tile& t) { return t.isR ? t.withV : t.final_; };
+  auto rounds_of = [&](const Tile& t) { return (t.isR && t.withV) ? 2 : 1; };   // staging rounds
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const bool deps = P.check_deps != 0;
+      auto counter_of = [&](const Tile& t) { return P.counters + (t.p - 1) * P.BH + t.h; };
+      int nE = 0, nVt = 0, nv = 0;
+      TileIter itE(P, first_g, stride_g, kBlocks), itV(P, first_g, stride_g, kBlocks);
+      while (nVt < n_total && !needs_v(itV.get())) { ++nVt; itV.next(); }
+      const uint64_t pol_first = policy_evict_first();
+      int ctrE = 0, ctrV = 0;
+      if (deps && nE < n_total && itE.get().p > 0) ctrE = ld_acquire(counter_of(itE.get()));
+      if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
+      long long t0 = clock64();
+      bool force = false;
+      while (nE < n_total || nVt < n_total) {
+        bool did = false;
+        if (nE < n_total) {
+          const Tile t = itE.get();
+          const int eE = nE % kRingE, eL = nE % kRingL;
+          bool ok = force || !deps || t.p == 0 || ctrE >= P.tiles_per_head;
+          if (!ok) { ctrE = ld_acquire(counter_of(t)); ok = ctrE >= P.tiles_per_head; }
+          if (ok && (force || (mbar_test(&bars->emptyE[eE], ((nE / kRingE) & 1) ^ 1) &&
+                               mbar_test(&bars->emptyL[eL], ((nE / kRingL) & 1) ^ 1)))) {
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            uint8_t* sE = smem + Lay::E + eE * kSlot;
+            uint8_t* sL = smem + Lay::L + eL * kSlot;
+            const bool needC = !t.first;
+            float* sC = reinterpret_cast<float*>(smem + Lay::Vec) + eL * 128;
+            mbar_expect_tx(&bars->fullE[eE], kSlot);
+            mbar_expect_tx(&bars->fullL[eL], kSlot + (needC ? 512 : 0));
+            if (t.isR) {
+              const int row0 = (t.h * m + t.idx0) * SB;
+              if (needC) bulk_load_1d(sC, P.cR + row0, 512, &bars->fullL[eL]);
+              tma_load_2d(sE, t.first ? &P.tmQ : &P.tmAR, &bars->fullE[eE], 0, row0);
+              tma_load_2d(sL, &P.tmK, &bars->fullL[eL], 0, row0);
+            } else {
+              const int row0 = (t.h * SB + t.idx0) * m;
+              bulk_load_1d(sC, P.cL + row0, 512, &bars->fullL[eL]);
+              tma_load_2d(sE, &P.tmAL, &bars->fullE[eE], 0, row0);
+#pragma unroll
+              for (int tt = 0; tt < kBlocks; ++tt)
+                tma_load_3d(sL + tt * (SB * 128), &P.tmQs, &bars->fullL[eL], 0, t.idx0 + tt, t.h * m);
+            }
+            stamp(P, nE, 0);
+            ++nE;
+            itE.next();
+            if (deps && nE < n_total && itE.get().p > 0) ctrE = ld_acquire(counter_of(itE.get()));
+            did = true;
+          }
+        }
+        if (nVt < n_total) {
+          const Tile t = itV.get();
+          const int eV = nv % kRingV;
+          bool ok = force || !deps || t.p == 0 || ctrV >= P.tiles_per_head;
+          if (!ok) { ctrV = ld_acquire(counter_of(t)); ok = ctrV >= P.tiles_per_head; }
+          if (ok && (force || mbar_test(&bars->emptyV[eV], ((nv / kRingV) & 1) ^ 1))) {
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            uint8_t* sV = smem + Lay::V + eV * kSlot;
+            mbar_expect_tx(&bars->fullV[eV], kSlot);
+            if (t.isR) tma_load_2d_hint(sV, &P.tmV, &bars->fullV[eV], 0, (t.h * m + t.idx0) * SB, pol_first);
+            else tma_load_2d(sV, &P.tmY, &bars->fullV[eV], 0, (t.h * SB + t.idx0) * m);
+            ++nv;
+            do { ++nVt; itV.next(); } while (nVt < n_total && !needs_v(itV.get()));
+            if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
+            did = true;
+          }
+        }
+        if (did) {
+          t0 = clock64();
+        } else if (!force) {
+          if (bars->abort_flag) {
+            force = true;
+          } else if (clock64() - t0 > P.wait_cycles) {
+            report_timeout(P.status, 10);
+            bars->abort_flag = 1;
+            force = true;
+          }
+          __nanosleep(32);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (polling)
+    if (elect_one()) {
+      const uint32_t sE0 = smem_u32(smem + Lay::E), sL0 = smem_u32(smem + Lay::L);
+      const uint32_t sV0 = smem_u32(smem + Lay::V), sP0 = smem_u32(smem + Lay::P);
+      const uint32_t sOnes = smem_u32(smem + Lay::Ones);
+      int i1 = 0, i2 = 0, nv = 0;
+      bool half_done = false;
+      TileIter it1(P, first_g, stride_g, kBlocks), it2(P, first_g, stride_g, kBlocks);
+      long long t0 = clock64();
+      bool force = false;
+      while (i2 < n_total) {
+        bool did = false;
+        if (i2 < i1) {
+          const Tile t = it2.get();
+          const int c = i2 & 1, q = i2 >> 1, eL = i2 % kRingL;
+          const bool needV = needs_v(t);
+          const int eV = nv % kRingV;
+          const bool split = t.isR || t.final_;
+          const uint32_t sL = sL0 + eL * kSlot, sV = sV0 + eV * kSlot, sP = sP0 + c * 2 * kSlot;
+          if (split && !half_done &&
+              (force || (mbar_test(&bars->p_half[c], q & 1) && mbar_test(&bars->o_free, (i2 & 1) ^ 1) &&
+                         (!needV || mbar_test(&bars->fullV[eV], (nv / kRingV) & 1))))) {
+            tc_fence_after();
+            if (t.isR) issue_apply<B, FT, 1>(tmem_o, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
+            else issue_apply<B, FT, 1>(tmem_o, sP, sV, 16, 1);
+            half_done = true;
+            did = true;
+          }
+          if ((half_done || !split) &&
+              (force || (mbar_test(&bars->p_ready[c], q & 1) &&
+                         (split || mbar_test(&bars->o_free, (i2 & 1) ^ 1))))) {
+            tc_fence_after();
+            if (t.isR) issue_apply<B, FT, 2>(tmem_o, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
+            else if (t.final_) issue_apply<B, FT, 2>(tmem_o, sP, sV, 16, 1);
+            else issue_transposed_apply<B, FT>(tmem_o, sP, sL, sOnes);
+            umma_commit(&bars->emptyL[eL]);
+            if (needV) { umma_commit(&bars->emptyV[eV]); ++nv; }
+            umma_commit(&bars->p_free[c]);
+            umma_commit(&bars->o_ready);
+            stamp(P, i2, 4);
+            ++i2;
+            it2.next();
+            half_done = false;
+            did = true;
+          }
+        }
+        if (i1 < n_total && i1 < i2 + kStagesS) {
+          const int eE = i1 % kRingE, eL = i1 % kRingL, s = i1 % kStagesS;
+          if (force || (mbar_test(&bars->fullE[eE], (i1 / kRingE) & 1) &&
+                        mbar_test(&bars->fullL[eL], (i1 / kRingL) & 1))) {
+            const Tile t = it1.get();
+            tc_fence_after();
+            const uint32_t sE = sE0 + eE * kSlot, sL = sL0 + eL * kSlot;
+            // R: A = aR (E ring), B = K (L ring).  L: A = Qb (L ring), B = aL (E ring).
+            issue_scores<B, FT>(tmem + s * 128, t.isR ? sE : sL, t.isR ? sL : sE);
+            umma_commit(&bars->emptyE[eE]);
+            umma_commit(&bars->s_ready[s]);
+            stamp(P, i1, 1);
+            ++i1;
+            it1.next();
+            did = true;
+          }
+        }
+        if (did) {
+          t0 = clock64();
+        } else if (!force) {
+          if (bars->abort_flag) {
+            force = true;
+          } else if (clock64() - t0 > P.wait_cycles) {
+            report_timeout(P.status, 20);
+            bars->abort_flag = 1;
+            force = true;
+          }
+          __nanosleep(20);
+        }
+      }
+    }
+  } else if (warp < 4) {
+    // ------------------------------------------------------------------ store threads
+    // Thread w handles the tiles n = w, w + 2, ... and has a "staged" barrier of its own, so that
+    // each waiter is never more than one phase away from the barrier it waits on.
+    if (lane == 0) {
+      const int w = warp - 2;
+      const uint8_t* sStage = smem + Lay::Stage;
+      const uint64_t pol_first = policy_evict_first();
+      TileIter it(P, first_g, stride_g, kBlocks);
+      int round = 0;                           // staging rounds this thread has taken so far
+      for (int n = 0; n < n_total; ++n, it.next()) {
+        const Tile t = it.get();
+        const int nr = rounds_of(t);
+        if ((n & 1) == w) {
+          for (int r = 0; r < nr; ++r) {
+            wait_or_abort(&bars->stage_ready[w], (round + r) & 1, bars, P.status, 40);
+#pragma unroll
+            for (int tt = 0; tt < kBlocks; ++tt) {
+              const uint8_t* src = sStage + tt * (SB * 128);
+              if (t.isR) {
+                tma_store_3d(r == 0 ? &P.tmALs : &P.tmYs, src, 0, t.idx0 + tt, t.h * SB);
+              } else if (t.final_) {
+                tma_store_3d_hint(&P.tmOut, src, 0, t.idx0 + tt, t.h * m, pol_first);
+              } else {
+                tma_store_3d(&P.tmARs, src, 0, t.idx0 + tt, t.h * m);
+              }
+            }
+            tma_store_commit();
+            tma_store_wait_read();
+            mbar_arrive(&bars->stage_free);
+          }
+          tma_store_wait_all();                 // rows (and c_L / c_R) are in global memory
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+          __threadfence();
+          atomicAdd(P.counters + t.p * P.BH + t.h, 1);
+          stamp(P, n, 7);
+          round += nr;
+        }
+      }
+    }
+  } else if (warp < 12) {
+    // ------------------------------------------------------------------ softmax groups: S -> P
+    const int c = (warp - 4) >> 2;             // group = P buffer; takes tiles n = c, c + 2, ...
+    const int sub = warp & 3;
+    const int t_row = sub * 32 + lane;         // TMEM lane = score row owned by this thread
+    const int tile = Geo<B>::tile(t_row), r = Geo<B>::row(t_row), srow = tile * B + r;
+    const int sb = r / SB, rb = r - sb * SB;
+    const int blk = tile * NSUB + sb;
+    uint8_t* sP = smem + Lay::P + c * 2 * kSlot;
+    float* stat = reinterpret_cast<float*>(smem + Lay::Stat);
+    const bool stamper = (sub == 0 && lane == 0);
+    constexpr int NC = B / 32;
+    auto mine = [&](int cc) { return SB == B || (32 * cc) / SB == sb; };
+
+    TileIter it(P, first_g + c * stride_g, 2 * stride_g, kBlocks);
+    for (int n = c; n < n_total; n += 2, it.next()) {
+      const Tile t = it.get();
+      const int q = n >> 1, eL = n % kRingL, s = n % kStagesS;
+      const float* cv = reinterpret_cast<const float*>(smem + Lay::Vec) + eL * 128;
+      const uint32_t tS = tmem + s * 128 + ((uint32_t)(sub * 32) << 16);
+      wait_or_abort(&bars->s_ready[s], (n / kStagesS) & 1, bars, P.status, 30);
+      tc_fence_after();
+      if (stamper) stamp(P, n, 2);
+      // the state tile MMA 1 consumed is read exactly once: drop its lines from L2
+      if (t.isR) {
+        if (!t.first) discard_line(P.aR + ((size_t)(t.h * m + t.idx0) * SB + t_row) * 128);
+      } else {
+        discard_line(P.aL + ((size_t)(t.h * SB + t.idx0) * m + t_row) * 128);
+      }
+
+      float buf[32];
+      float f, inv_s, mx, sum, sz = 0.f;
+      float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      float2 a2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      const float* cvt = cv + blk * SB;
+      if (t.isR) {
+        // Z_R = scale * S / c_R (Eq. 7); c_L = sum R log R (Eq. 10)
+        float inv_c = 1.f;
+        if (!t.first) {
+          const float cr = cv[srow];
+          inv_c = cr > 1e-30f ? 1.f / cr : 0.f;
+        }
+        f = P.scale * inv_c * kLog2e;
+#pragma unroll
+        for (int cc = 0; cc < NC; ++cc) {
+          if (!mine(cc)) continue;
+          tmem_ld32(tS + 32 * cc, buf);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) m4[i & 3] = max3(m4[i & 3], buf[2 * i], buf[2 * i + 1]);
+        }
+        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        const float2 f2 = make_float2(f, f), off2 = make_float2(-mx * f, -mx * f);
+        float2 z2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        // the apply MMA of this group's previous tile must be done with the P buffer
+        wait_or_abort(&bars->p_free[c], (q & 1) ^ 1, bars, P.status, 33);
+#pragma unroll
+        for (int cc = 0; cc < NC; ++cc) {
+          float* sv = buf;
+          if (mine(cc)) {
+            tmem_ld32(tS + 32 * cc, buf);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float2 x = make_float2(sv[2 * i], sv[2 * i + 1]);
+              const float2 zz = ffma2(x, f2, off2);
+              const float2 pp = exp2_pair(zz, i);
+              z2[i & 1] = ffma2(pp, x, z2[i & 1]);
+              a2[i & 1] = fadd2(a2[i & 1], pp);
+              sv[2 * i] = pp.x;
+              sv[2 * i + 1] = pp.y;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sv[i] = 0.f;
+          }
+          store_row32<T>(sP, srow, 32 * cc, sv);
+          if (cc == NC / 2 - 1) {
+            fence_proxy_async();
+            mbar_arrive(&bars->p_half[c]);
+          }
+        }
+        sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
+        sz = (z2[0].x + z2[0].y) + (z2[1].x + z2[1].y);
+        inv_s = 1.f / sum;
+        // -c_L in log2 units, ready to be the addend of the next L half-step's logits
+        P.cL[((size_t)t.h * SB + rb) * m + t.idx0 + blk] = fast_log2(sum) - f * (sz * inv_s - mx);
+      } else {
+        // Z_L = scale * S' - c_L (Eq. 8), softmax over k = along the row
+        f = P.scale * kLog2e;
+        const float2 f2 = make_float2(f, f);
+#pragma unroll
+        for (int cc = 0; cc < NC; ++cc) {
+          if (!mine(cc)) continue;
+          tmem_ld32(tS + 32 * cc, buf);
+          tmem_ld_wait();
+          const float4* cv4 = reinterpret_cast<const float4*>(cvt + 32 * cc - sb * SB);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float4 k4 = cv4[i];
+            const float2 za = ffma2(make_float2(buf[4 * i], buf[4 * i + 1]), f2, make_float2(k4.x, k4.y));
+            const float2 zb = ffma2(make_float2(buf[4 * i + 2], buf[4 * i + 3]), f2, make_float2(k4.z, k4.w));
+            m4[0] = max3(m4[0], za.x, za.y);
+            m4[1] = max3(m4[1], zb.x, zb.y);
+          }
+        }
+        mx = fmaxf(m4[0], m4[1]);
+        const float2 nmx2 = make_float2(-mx, -mx);
+        wait_or_abort(&bars->p_free[c], (q & 1) ^ 1, bars, P.status, 33);
+#pragma unroll
+        for (int cc = 0; cc < NC; ++cc) {
+          float* sv = buf;
+          if (mine(cc)) {
+            tmem_ld32(tS + 32 * cc, buf);
+            tmem_ld_wait();
+            const float4* cv4 = reinterpret_cast<const float4*>(cvt + 32 * cc - sb * SB);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float4 k4 = cv4[i];
+              float2 za = ffma2(make_float2(sv[4 * i], sv[4 * i + 1]), f2, make_float2(k4.x, k4.y));
+              float2 zb = ffma2(make_float2(sv[4 * i + 2], sv[4 * i + 3]), f2, make_float2(k4.z, k4.w));
+              za = fadd2(za, nmx2);
+              zb = fadd2(zb, nmx2);
+              const float2 pa = exp2_pair(za, 2 * i);
+              const float2 pb = exp2_pair(zb, 2 * i + 1);
+              a2[0] = fadd2(a2[0], pa);
+              a2[1] = fadd2(a2[1], pb);
+              sv[4 * i] = pa.x;
+              sv[4 * i + 1] = pa.y;
+              sv[4 * i + 2] = pb.x;
+              sv[4 * i + 3] = pb.y;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sv[i] = 0.f;
+          }
+          store_row32<T>(sP, srow, 32 * cc, sv);
+          if (cc == NC / 2 - 1 && t.final_) {
+            fence_proxy_async();
+            mbar_arrive(&bars->p_half[c]);
+          }
+        }
+        sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
+        inv_s = 1.f / sum;
+        if (!t.final_) {
+          // MMA 2 of this half-step contracts over rows: P must be normalised before it is read.
+          // The thread re-reads its own row, rescales in fp32, writes it back.
+          const float2 is2 = make_float2(inv_s, inv_s);
+#pragma unroll
+          for (int c8 = 0; c8 < B / 8; ++c8) {
+            uint4* ptr = reinterpret_cast<uint4*>(sP + (c8 >> 3) * kTileBytes + srow * 128 +
+                                                  (((c8 & 7) ^ (srow & 7)) << 4));
+            uint4 qv = *ptr;
+            uint32_t* qp = reinterpret_cast<uint32_t*>(&qv);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 v = fmul2(unpack2<T>(qp[e]), is2);
+              qp[e] = pack2<T>(v.x, v.y);
+            }
+            *ptr = qv;
+          }
+        }
+      }
+      if (!t.isR && !t.final_) mbar_arrive(&bars->p_half[c]);
+      stat[(n & 3) * 128 + t_row] = inv_s;     // for the epilogue group
+      fence_proxy_async();
+      tc_fence_before();   // keeps the barrier's phase in step
+      mbar_arrive(&bars->p_ready[c]);
+      if (stamper) stamp(P, n, 3);
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue group: O -> rows
+    const int sub = warp & 3;
+    const int t_row = sub * 32 + lane;
+    const int tile = Geo<B>::tile(t_row), r = Geo<B>::row(t_row), srow = tile * B + r;
+    const int sb = r / SB, rb = r - sb * SB;
+    const int blk = tile * NSUB + sb;
+    uint8_t* sStage = smem + Lay::Stage;
+    const float* stat = reinterpret_cast<const float*>(smem + Lay::Stat);
+    const uint32_t tO = tmem_o + ((uint32_t)(sub * 32) << 16);
+    const bool stamper = (sub == 0 && lane == 0);
+    TileIter it(P, first_g, stride_g, kBlocks);
+    int round = 0;
+    for (int n = 0; n < n_total; ++n, it.next()) {
+      const Tile t = it.get();
+      wait_or_abort(&bars->o_ready, n & 1, bars, P.status, 31);
+      tc_fence_after();
+      if (stamper) stamp(P, n, 5);
+      const float inv_s = stat[(n & 3) * 128 + t_row];
+      if (t.final_) discard_line(P.y + ((size_t)(t.h * SB + t.idx0) * m + t_row) * 128);
+      const int nr = rounds_of(t);
+      const bool scaled = t.isR || t.final_;
+      float c1 = 0.f;
+      if (!scaled) c1 = tmem_ld1(tO + 64);
+      for (int rr = 0; rr < nr; ++rr) {
+        float buf[2][32];
+        tmem_ld32(tO + 64 * rr, buf[0]);
+        tmem_ld32(tO + 64 * rr + 32, buf[1]);
+        tmem_ld_wait();
+        if (rr == nr - 1) {                      // O is in registers: the next apply MMA may run
+          tc_fence_before();
+          mbar_arrive(&bars->o_free);
+        }
+        wait_or_abort(&bars->stage_free, ((round + rr) & 1) ^ 1, bars, P.status, 35);
+        if (t.final_) {
+          store_row32<T>(sStage, srow, 0, buf[0], inv_s);
+          store_row32<T>(sStage, srow, 32, buf[1], inv_s);
+        } else if (scaled) {
+          store_row32<T>(sStage, srow, 0, buf[0], inv_s);
+          store_row32<T>(sStage, srow, 32, buf[1], inv_s);
+        } else {
+          store_row32<T>(sStage, srow, 0, buf[0]);
+          store_row32<T>(sStage, srow, 32, buf[1]);
+        }
+        fence_proxy_async();
+        mbar_arrive(&bars->stage_ready[n & 1]);
+      }
+      if (!scaled) P.cR[((size_t)t.h * m + rb) * SB + t.idx0 + blk] = c1;
+      if (stamper) stamp(P, n, 6);
+      round += nr;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (bars->abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 200000) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 0) tmem_dealloc(tmem, 512);
+  if (tid == 0) {   // the last CTA re-arms the dependency counters
+    __threadfence();
+    if (atomicAdd(P.status + 1, 1) == (int)gridDim.x - 1) {
+      for (int i = 0; i < P.n_counters; ++i) P.counters[i] = 0;
+      P.status[1] = 0;
+    }
+  }
+}
+
+template <typename T, int B, int SB>
+inline cudaError_t launch_kernel(const Params& P, int grid, cudaStream_t st) {
+  const void* fn = (const void*)monarch_decoupled<T, B, SB>;
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+  if (e != cudaSuccess) return e;
+  monarch_decoupled<T, B, SB><<<grid, kThreads, kSmem, st>>>(P);
+  return cudaGetLastError();
+}
+
+}  // namespace tp2
+
+namespace tp {
+template <typename T, int B, int SB>
+cudaError_t launch_decoupled(const Params& P, int grid, cudaStream_t st) {
+  return tp2::launch_kernel<T, B, SB>(P, grid, st);
+}
+}  // namespace tp
+}  // namespace ma

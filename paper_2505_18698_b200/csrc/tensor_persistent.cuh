@@ -707,6 +707,10 @@ inline size_t workspace_bytes(int BH, int N, int T) {
   return ws_layout(nullptr, BH, N).bytes + counters_bytes(BH, T);
 }
 
+// Defined in tensor_decoupled.cuh (the second-generation kernel, same Params).
+template <typename T, int B, int SB>
+cudaError_t launch_decoupled(const Params& P, int grid, cudaStream_t st);
+
 template <typename T, int B, int SB>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int T_steps,
                     int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
@@ -749,10 +753,14 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
     return 7;
   const int total = 2 * T_steps * P.tiles_per_phase;
   int n = 0;
-  if (mode == 0) {          // one launch, dependencies tracked by counters
+  if (mode == 0 || mode == 2) {   // one launch, dependencies tracked by counters
     P.g_begin = knobs().skip_first_half_step ? P.tiles_per_phase : 0; P.g_end = total; P.check_deps = 1;
     const int grid = total < num_sms ? total : num_sms;
-    monarch_persistent<T, B, SB><<<grid, kThreads, kSmem, st>>>(P);
+    if (mode == 0) {
+      if (launch_decoupled<T, B, SB>(P, grid, st) != cudaSuccess) return 7;
+    } else {
+      monarch_persistent<T, B, SB><<<grid, kThreads, kSmem, st>>>(P);
+    }
     n = 1;
   } else {                  // one launch per half-step (stream order is the dependency)
     P.check_deps = 0;

@@ -94,7 +94,8 @@ def test_generic_path_on_configuration_shapes(name):
 
 
 # ------------------------------------------------------------------ tensor-core paths
-TENSOR_PATHS = [binding.MA_PATH_TENSOR, binding.MA_PATH_TENSOR_PHASED, binding.MA_PATH_TENSOR_BASIC]
+TENSOR_PATHS = [binding.MA_PATH_TENSOR, binding.MA_PATH_TENSOR_PHASED, binding.MA_PATH_TENSOR_BASIC,
+                binding.MA_PATH_TENSOR_CHAINED]
 
 
 @pytest.mark.parametrize("path", TENSOR_PATHS)
