@@ -5,16 +5,25 @@
 // the whole chain of a tile (scores -> softmax -> wait for the apply MMA -> epilogue -> wait for
 // the next scores), about 2.8 us of mostly latency, and two such chains were all that tensor
 // memory and shared memory allow.  Here
-//   * two softmax warpgroups do nothing but S -> P (alternate tiles); S has three TMEM stages,
-//     so the score MMA runs up to three tiles ahead and a group never waits for it;
+//   * two softmax warpgroups do nothing but S -> P (alternate tiles); S has three (b = 128) or four
+//     (b <= 64) TMEM stages, so the score MMA runs ahead and a group never waits for it;
 //   * a third warpgroup does every epilogue (O -> 16-bit rows -> staging), so the softmax groups
-//     never wait for the apply MMA; O has a single TMEM stage, drained as soon as it is ready;
+//     never wait for the apply MMA; O has one TMEM stage at b = 128 and two at b <= 64;
 //   * two store threads alternate tiles (TMA store, completion, dependency counter).
 // 512 threads: warp 0 TMA producer, warp 1 MMA issuer, warps 2-3 store threads, warps 4-7 and
-// 8-11 softmax groups, warps 12-15 epilogue group.
-// TMEM: S0, S1, S2 at columns 0, 128, 256; O at 384.  Shared memory: rings E (2) / L (4) / V (2) of
-// 16 KB operand tiles, two 32 KB P buffers, one 16 KB staging buffer (the last R half-step stages
-// alpha_L and y in two rounds), row statistics, c-vectors, a tile of ones.
+// 8-11 softmax groups, warps 12-15 epilogue group.  The producer and the MMA issuer poll: each
+// iteration issues all its barrier tests back to back, then acts on whatever is ready.
+// TMEM: score stages of B columns from column 0, then the O stages of 128 columns.  Shared memory
+// (see Cfg / Lay): rings E / L / V of 16 KB operand tiles, one P buffer per softmax group, one
+// 16 KB staging buffer (the last R half-step stages alpha_L and y in two rounds), row statistics,
+// c-vectors, a tile of ones.
+//
+// Measured and rejected on B200 (slower than this arrangement): issuing the first half of the apply
+// MMA while the softmax is still producing the second half of P (it holds the single O stage for
+// half a softmax); writing rows to global memory straight from the epilogue threads instead of
+// staging + TMA store (16-byte stores to rows 128 bytes apart swamp the load/store unit, the
+// softmax groups slow down by half); one store thread instead of two (the completion fence of a tile
+// is about a microsecond); separate blocking issuer threads for the two MMAs.
 #pragma once
 #include "tensor_persistent.cuh"
 
@@ -36,34 +45,69 @@ using ma::tp::tma_store_wait_read;
 using ma::tp::tma_store_wait_all;
 
 constexpr int kThreads = 512;
-constexpr int kRingE = 2, kRingL = 4, kRingV = 2, kStagesS = 3;
 constexpr int kSlot = kTileBytes;
 
+// Pipeline depths per MMA block size.  TMEM has 512 columns: a score stage takes B of them, an O
+// stage 128.  Shared memory: operand rings of 16 KB tiles, one P buffer per softmax group, one
+// staging buffer.  The L ring is the deepest: its tile (K, or the Q block of an L half-step) is held
+// from the load until the apply MMA of the tile has run, four to five microseconds.
+template <int B>
+struct Cfg;
+template <>
+struct Cfg<128> {
+  static constexpr int kRingE = 2, kRingL = 4, kRingV = 2, kStagesS = 3, kStagesO = 1;
+};
+template <>
+struct Cfg<64> {
+  static constexpr int kRingE = 3, kRingL = 5, kRingV = 2, kStagesS = 4, kStagesO = 2;
+};
+constexpr int kMaxRing = 6, kMaxStagesS = 4;
+
+template <int B>
 struct Lay {
+  using C = Cfg<B>;
+  static constexpr int kPBytes = 128 * B * 2;           // one P buffer (128 rows x B columns)
   static constexpr int E = 0;
-  static constexpr int L = E + kRingE * kSlot;
-  static constexpr int V = L + kRingL * kSlot;
-  static constexpr int P = V + kRingV * kSlot;          // 2 x 32 KB
-  static constexpr int Stage = P + 4 * kSlot;           // 16 KB
+  static constexpr int L = E + C::kRingE * kSlot;
+  static constexpr int V = L + C::kRingL * kSlot;
+  static constexpr int P = V + C::kRingV * kSlot;       // two P buffers
+  static constexpr int Stage = P + 2 * kPBytes;         // 16 KB
   static constexpr int Ones = Stage + kSlot;            // 2 KB
   static constexpr int Vec = Ones + 2048;               // kRingL x 128 floats (c_R / c_L)
-  static constexpr int Stat = Vec + kRingL * 512;       // 4 x 128 floats (1 / row sum)
+  static constexpr int Stat = Vec + C::kRingL * 512;    // 4 x 128 floats (1 / row sum)
   static constexpr int Bars = Stat + 4 * 512;
   static constexpr int Total = Bars + 512;
+  static constexpr int kSmem = Total + 1024;
+  static_assert(kSmem <= 227 * 1024, "shared memory budget");
+  static_assert(C::kStagesS * B + C::kStagesO * 128 <= 512, "tensor memory budget");
 };
-constexpr int kSmem = Lay::Total + 1024;
 
 struct __align__(8) Bars {
-  uint64_t fullE[kRingE], emptyE[kRingE];
-  uint64_t fullL[kRingL], emptyL[kRingL];
-  uint64_t fullV[kRingV], emptyV[kRingV];
-  uint64_t s_ready[kStagesS];
-  uint64_t p_half[2], p_ready[2], p_free[2];
-  uint64_t o_ready, o_free, stage_ready[2], stage_free;
+  uint64_t fullE[kMaxRing], emptyE[kMaxRing];
+  uint64_t fullL[kMaxRing], emptyL[kMaxRing];
+  uint64_t fullV[kMaxRing], emptyV[kMaxRing];
+  uint64_t s_ready[kMaxStagesS];
+  uint64_t p_ready[2], p_free[2];
+  uint64_t o_ready[2], o_free[2], stage_ready[2], stage_free;
   uint32_t tmem_slot;
   volatile int abort_flag;
   long long wait_limit;
 };
+static_assert(sizeof(Bars) <= 512, "barrier block");
+
+// Non-blocking phase test for the polling loops.  Shared memory is busy (MMA operand reads, TMA
+// writes, P stores), so one barrier read takes a hundred cycles or more: a polling thread issues
+// all its tests of an iteration back to back and only then looks at the results.
+__device__ __forceinline__ uint32_t mbar_poll(uint64_t* bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(smem_u32(bar)), "r"(parity));
+  return done;
+}
 
 // Bounded wait; see tensor_persistent.cuh (after a timeout every wait of the CTA returns at once).
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Bars* bars, int* status,
@@ -93,6 +137,11 @@ template <typename T, int B, int SB>
 __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_constant__ Params P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  using Lay = tp2::Lay<B>;
+  using C = Cfg<B>;
+  constexpr int kRingE = C::kRingE, kRingL = C::kRingL, kRingV = C::kRingV;
+  constexpr int kStagesS = C::kStagesS, kStagesO = C::kStagesO;
+  constexpr int kPBytes = Lay::kPBytes;
   Bars* bars = reinterpret_cast<Bars*>(smem + Lay::Bars);
   constexpr int kBlocks = kRows / SB;         // blocks (k of an R tile, j of an L tile) per CTA
   constexpr int NSUB = B / SB;                // blocks per MMA tile
@@ -106,12 +155,11 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
     for (int i = 0; i < kRingV; ++i) { mbar_init(&bars->fullV[i], 1); mbar_init(&bars->emptyV[i], 1); }
     for (int i = 0; i < kStagesS; ++i) mbar_init(&bars->s_ready[i], 1);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&bars->p_half[i], 128);
       mbar_init(&bars->p_ready[i], 128);
       mbar_init(&bars->p_free[i], 1);
+      mbar_init(&bars->o_ready[i], 1);
+      mbar_init(&bars->o_free[i], 128);
     }
-    mbar_init(&bars->o_ready, 1);
-    mbar_init(&bars->o_free, 128);
     mbar_init(&bars->stage_ready[0], 128);
     mbar_init(&bars->stage_ready[1], 128);
     mbar_init(&bars->stage_free, 1);
@@ -130,7 +178,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bars->tmem_slot;
-  const uint32_t tmem_o = tmem + 384;
+  const uint32_t tmem_o = tmem + kStagesS * B;   // O stage o at tmem_o + 128 o
 
   const int first_g = P.g_begin + blockIdx.x;
   const int stride_g = gridDim.x;
@@ -150,17 +198,19 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       int ctrE = 0, ctrV = 0;
       if (deps && nE < n_total && itE.get().p > 0) ctrE = ld_acquire(counter_of(itE.get()));
       if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
-      long long t0 = clock64();
-      bool force = false;
+      long long t0 = 0;
+      bool force = false, idle = false;
       while (nE < n_total || nVt < n_total) {
         bool did = false;
+        const int eE = nE % kRingE, eL = nE % kRingL, eV = nv % kRingV;
+        const uint32_t r_e = mbar_poll(&bars->emptyE[eE], ((nE / kRingE) & 1) ^ 1);
+        const uint32_t r_l = mbar_poll(&bars->emptyL[eL], ((nE / kRingL) & 1) ^ 1);
+        const uint32_t r_v = mbar_poll(&bars->emptyV[eV], ((nv / kRingV) & 1) ^ 1);
         if (nE < n_total) {
           const Tile t = itE.get();
-          const int eE = nE % kRingE, eL = nE % kRingL;
           bool ok = force || !deps || t.p == 0 || ctrE >= P.tiles_per_head;
-          if (!ok) { ctrE = ld_acquire(counter_of(t)); ok = ctrE >= P.tiles_per_head; }
-          if (ok && (force || (mbar_test(&bars->emptyE[eE], ((nE / kRingE) & 1) ^ 1) &&
-                               mbar_test(&bars->emptyL[eL], ((nE / kRingL) & 1) ^ 1)))) {
+          if (!ok && (r_e & r_l)) { ctrE = ld_acquire(counter_of(t)); ok = ctrE >= P.tiles_per_head; }
+          if (ok && (force || (r_e & r_l))) {
             asm volatile("fence.proxy.async.global;" ::: "memory");
             uint8_t* sE = smem + Lay::E + eE * kSlot;
             uint8_t* sL = smem + Lay::L + eL * kSlot;
@@ -184,16 +234,16 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             stamp(P, nE, 0);
             ++nE;
             itE.next();
+            // the next tile's counter is read now and looked at one iteration later
             if (deps && nE < n_total && itE.get().p > 0) ctrE = ld_acquire(counter_of(itE.get()));
             did = true;
           }
         }
         if (nVt < n_total) {
           const Tile t = itV.get();
-          const int eV = nv % kRingV;
           bool ok = force || !deps || t.p == 0 || ctrV >= P.tiles_per_head;
-          if (!ok) { ctrV = ld_acquire(counter_of(t)); ok = ctrV >= P.tiles_per_head; }
-          if (ok && (force || mbar_test(&bars->emptyV[eV], ((nv / kRingV) & 1) ^ 1))) {
+          if (!ok && r_v) { ctrV = ld_acquire(counter_of(t)); ok = ctrV >= P.tiles_per_head; }
+          if (ok && (force || r_v)) {
             asm volatile("fence.proxy.async.global;" ::: "memory");
             uint8_t* sV = smem + Lay::V + eV * kSlot;
             mbar_expect_tx(&bars->fullV[eV], kSlot);
@@ -206,9 +256,12 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
           }
         }
         if (did) {
-          t0 = clock64();
+          idle = false;
         } else if (!force) {
-          if (bars->abort_flag) {
+          if (!idle) {
+            idle = true;
+            t0 = clock64();
+          } else if (bars->abort_flag) {
             force = true;
           } else if (clock64() - t0 > P.wait_cycles) {
             report_timeout(P.status, 10);
@@ -226,67 +279,59 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       const uint32_t sV0 = smem_u32(smem + Lay::V), sP0 = smem_u32(smem + Lay::P);
       const uint32_t sOnes = smem_u32(smem + Lay::Ones);
       int i1 = 0, i2 = 0, nv = 0;
-      bool half_done = false;
       TileIter it1(P, first_g, stride_g, kBlocks), it2(P, first_g, stride_g, kBlocks);
-      long long t0 = clock64();
-      bool force = false;
+      long long t0 = 0;
+      bool force = false, idle = false;
       while (i2 < n_total) {
         bool did = false;
+        const int c = i2 & 1, q = i2 >> 1, eL2 = i2 % kRingL, eV = nv % kRingV;
+        const int o2 = i2 % kStagesO;
+        const int eE = i1 % kRingE, eL1 = i1 % kRingL, s1 = i1 % kStagesS;
+        const uint32_t r_ready = mbar_poll(&bars->p_ready[c], q & 1);
+        const uint32_t r_of = mbar_poll(&bars->o_free[o2], ((i2 / kStagesO) & 1) ^ 1);
+        const uint32_t r_v = mbar_poll(&bars->fullV[eV], (nv / kRingV) & 1);
+        const uint32_t r_e = mbar_poll(&bars->fullE[eE], (i1 / kRingE) & 1);
+        const uint32_t r_l = mbar_poll(&bars->fullL[eL1], (i1 / kRingL) & 1);
         if (i2 < i1) {
           const Tile t = it2.get();
-          const int c = i2 & 1, q = i2 >> 1, eL = i2 % kRingL;
           const bool needV = needs_v(t);
-          const int eV = nv % kRingV;
-          const bool split = t.isR || t.final_;
-          const uint32_t sL = sL0 + eL * kSlot, sV = sV0 + eV * kSlot, sP = sP0 + c * 2 * kSlot;
-          if (split && !half_done &&
-              (force || (mbar_test(&bars->p_half[c], q & 1) && mbar_test(&bars->o_free, (i2 & 1) ^ 1) &&
-                         (!needV || mbar_test(&bars->fullV[eV], (nv / kRingV) & 1))))) {
+          if (force || (r_ready && r_of && (!needV || r_v))) {
+            const uint32_t sL = sL0 + eL2 * kSlot, sV = sV0 + eV * kSlot, sP = sP0 + c * kPBytes;
+            const uint32_t tO = tmem_o + o2 * 128;
             tc_fence_after();
-            if (t.isR) issue_apply<B, FT, 1>(tmem_o, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
-            else issue_apply<B, FT, 1>(tmem_o, sP, sV, 16, 1);
-            half_done = true;
-            did = true;
-          }
-          if ((half_done || !split) &&
-              (force || (mbar_test(&bars->p_ready[c], q & 1) &&
-                         (split || mbar_test(&bars->o_free, (i2 & 1) ^ 1))))) {
-            tc_fence_after();
-            if (t.isR) issue_apply<B, FT, 2>(tmem_o, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
-            else if (t.final_) issue_apply<B, FT, 2>(tmem_o, sP, sV, 16, 1);
-            else issue_transposed_apply<B, FT>(tmem_o, sP, sL, sOnes);
-            umma_commit(&bars->emptyL[eL]);
+            if (t.isR) issue_apply<B, FT, 0>(tO, sP, sL, needV ? (sV - sL) : 16, needV ? 2 : 1);
+            else if (t.final_) issue_apply<B, FT, 0>(tO, sP, sV, 16, 1);
+            else issue_transposed_apply<B, FT>(tO, sP, sL, sOnes);
+            umma_commit(&bars->emptyL[eL2]);
             if (needV) { umma_commit(&bars->emptyV[eV]); ++nv; }
             umma_commit(&bars->p_free[c]);
-            umma_commit(&bars->o_ready);
+            umma_commit(&bars->o_ready[o2]);
             stamp(P, i2, 4);
             ++i2;
             it2.next();
-            half_done = false;
             did = true;
           }
         }
-        if (i1 < n_total && i1 < i2 + kStagesS) {
-          const int eE = i1 % kRingE, eL = i1 % kRingL, s = i1 % kStagesS;
-          if (force || (mbar_test(&bars->fullE[eE], (i1 / kRingE) & 1) &&
-                        mbar_test(&bars->fullL[eL], (i1 / kRingL) & 1))) {
-            const Tile t = it1.get();
-            tc_fence_after();
-            const uint32_t sE = sE0 + eE * kSlot, sL = sL0 + eL * kSlot;
-            // R: A = aR (E ring), B = K (L ring).  L: A = Qb (L ring), B = aL (E ring).
-            issue_scores<B, FT>(tmem + s * 128, t.isR ? sE : sL, t.isR ? sL : sE);
-            umma_commit(&bars->emptyE[eE]);
-            umma_commit(&bars->s_ready[s]);
-            stamp(P, i1, 1);
-            ++i1;
-            it1.next();
-            did = true;
-          }
+        if (i1 < n_total && i1 < i2 + kStagesS && (force || (r_e && r_l))) {
+          const Tile t = it1.get();
+          tc_fence_after();
+          const uint32_t sE = sE0 + eE * kSlot, sL = sL0 + eL1 * kSlot;
+          // R: A = aR (E ring), B = K (L ring).  L: A = Qb (L ring), B = aL (E ring).
+          issue_scores<B, FT>(tmem + s1 * B, t.isR ? sE : sL, t.isR ? sL : sE);
+          umma_commit(&bars->emptyE[eE]);
+          umma_commit(&bars->s_ready[s1]);
+          stamp(P, i1, 1);
+          ++i1;
+          it1.next();
+          did = true;
         }
         if (did) {
-          t0 = clock64();
+          idle = false;
         } else if (!force) {
-          if (bars->abort_flag) {
+          if (!idle) {
+            idle = true;
+            t0 = clock64();
+          } else if (bars->abort_flag) {
             force = true;
           } else if (clock64() - t0 > P.wait_cycles) {
             report_timeout(P.status, 20);
@@ -345,7 +390,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
     const int tile = Geo<B>::tile(t_row), r = Geo<B>::row(t_row), srow = tile * B + r;
     const int sb = r / SB, rb = r - sb * SB;
     const int blk = tile * NSUB + sb;
-    uint8_t* sP = smem + Lay::P + c * 2 * kSlot;
+    uint8_t* sP = smem + Lay::P + c * kPBytes;
     float* stat = reinterpret_cast<float*>(smem + Lay::Stat);
     const bool stamper = (sub == 0 && lane == 0);
     constexpr int NC = B / 32;
@@ -356,7 +401,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       const Tile t = it.get();
       const int q = n >> 1, eL = n % kRingL, s = n % kStagesS;
       const float* cv = reinterpret_cast<const float*>(smem + Lay::Vec) + eL * 128;
-      const uint32_t tS = tmem + s * 128 + ((uint32_t)(sub * 32) << 16);
+      const uint32_t tS = tmem + s * B + ((uint32_t)(sub * 32) << 16);
       wait_or_abort(&bars->s_ready[s], (n / kStagesS) & 1, bars, P.status, 30);
       tc_fence_after();
       if (stamper) stamp(P, n, 2);
@@ -414,10 +459,6 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             for (int i = 0; i < 32; ++i) sv[i] = 0.f;
           }
           store_row32<T>(sP, srow, 32 * cc, sv);
-          if (cc == NC / 2 - 1) {
-            fence_proxy_async();
-            mbar_arrive(&bars->p_half[c]);
-          }
         }
         sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
         sz = (z2[0].x + z2[0].y) + (z2[1].x + z2[1].y);
@@ -474,10 +515,6 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             for (int i = 0; i < 32; ++i) sv[i] = 0.f;
           }
           store_row32<T>(sP, srow, 32 * cc, sv);
-          if (cc == NC / 2 - 1 && t.final_) {
-            fence_proxy_async();
-            mbar_arrive(&bars->p_half[c]);
-          }
         }
         sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
         inv_s = 1.f / sum;
@@ -500,10 +537,9 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
           }
         }
       }
-      if (!t.isR && !t.final_) mbar_arrive(&bars->p_half[c]);
       stat[(n & 3) * 128 + t_row] = inv_s;     // for the epilogue group
       fence_proxy_async();
-      tc_fence_before();   // keeps the barrier's phase in step
+      tc_fence_before();
       mbar_arrive(&bars->p_ready[c]);
       if (stamper) stamp(P, n, 3);
     }
@@ -516,13 +552,15 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
     const int blk = tile * NSUB + sb;
     uint8_t* sStage = smem + Lay::Stage;
     const float* stat = reinterpret_cast<const float*>(smem + Lay::Stat);
-    const uint32_t tO = tmem_o + ((uint32_t)(sub * 32) << 16);
+    const uint32_t tO0 = tmem_o + ((uint32_t)(sub * 32) << 16);
     const bool stamper = (sub == 0 && lane == 0);
     TileIter it(P, first_g, stride_g, kBlocks);
     int round = 0;
     for (int n = 0; n < n_total; ++n, it.next()) {
       const Tile t = it.get();
-      wait_or_abort(&bars->o_ready, n & 1, bars, P.status, 31);
+      const int o = n % kStagesO;
+      const uint32_t tO = tO0 + o * 128;
+      wait_or_abort(&bars->o_ready[o], (n / kStagesO) & 1, bars, P.status, 31);
       tc_fence_after();
       if (stamper) stamp(P, n, 5);
       const float inv_s = stat[(n & 3) * 128 + t_row];
@@ -538,7 +576,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         tmem_ld_wait();
         if (rr == nr - 1) {                      // O is in registers: the next apply MMA may run
           tc_fence_before();
-          mbar_arrive(&bars->o_free);
+          mbar_arrive(&bars->o_free[o]);
         }
         wait_or_abort(&bars->stage_free, ((round + rr) & 1) ^ 1, bars, P.status, 35);
         if (t.final_) {
@@ -580,6 +618,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
 template <typename T, int B, int SB>
 inline cudaError_t launch_kernel(const Params& P, int grid, cudaStream_t st) {
   const void* fn = (const void*)monarch_decoupled<T, B, SB>;
+  constexpr int kSmem = Lay<B>::kSmem;
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
   if (e != cudaSuccess) return e;
   monarch_decoupled<T, B, SB><<<grid, kThreads, kSmem, st>>>(P);

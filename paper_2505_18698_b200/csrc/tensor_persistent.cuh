@@ -66,6 +66,7 @@ struct Params {
   float* cL;
   float* cR;
   uint8_t *aL, *aR, *y;  // state arrays (for L2 discards once a tile has been consumed)
+  uint8_t* out;         // Y (the second-generation kernel stores rows with plain stores)
   int* status;
   int* counters;       // [2T][BH] completed tiles
   long long* trace;    // optional: clock64 stamps [4 CTAs][64 tiles][8 events] (profiling aid)
@@ -729,7 +730,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
             make_map_strided(&P.tmARs, dtype, w.aR, SB, (uint64_t)BH * m, SB) &&
             make_map_strided(&P.tmOut, dtype, Y, SB, (uint64_t)BH * m, SB);
   if (!ok) return 7;
-  P.aL = (uint8_t*)w.aL; P.aR = (uint8_t*)w.aR; P.y = (uint8_t*)w.y;
+  P.aL = (uint8_t*)w.aL; P.aR = (uint8_t*)w.aR; P.y = (uint8_t*)w.y; P.out = (uint8_t*)Y;
   P.cL = w.cL; P.cR = w.cR; P.status = w.status; P.counters = counters;
   P.trace = trace_buffer();
   P.m = m; P.BH = BH; P.T = T_steps;
