@@ -109,6 +109,27 @@ __device__ __forceinline__ uint32_t mbar_poll(uint64_t* bar, uint32_t parity) {
   return done;
 }
 
+// Position in a ring of N slots (or stages): slot index and the parity of the round, kept
+// incrementally so that the polling threads do no divisions.
+template <int N>
+struct RingPos {
+  int slot = 0;
+  uint32_t par = 0;
+  __device__ __forceinline__ void advance() {
+    if (++slot == N) { slot = 0; par ^= 1; }
+  }
+};
+__device__ __forceinline__ uint32_t mbar_poll_addr(uint32_t addr, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(addr), "r"(parity));
+  return done;
+}
+
 // Bounded wait; see tensor_persistent.cuh (after a timeout every wait of the CTA returns at once).
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Bars* bars, int* status,
                                               int where) {
@@ -173,7 +194,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
     *reinterpret_cast<uint4*>(smem + Lay::Ones + tid * 16) = make_uint4(one2, one2, one2, one2);
   }
   if (warp == 0) tmem_alloc(&bars->tmem_slot, 512);
-  fence_proxy_async();
+
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -191,7 +212,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
     if (lane == 0) {
       const bool deps = P.check_deps != 0;
       auto counter_of = [&](const Tile& t) { return P.counters + (t.p - 1) * P.BH + t.h; };
-      int nE = 0, nVt = 0, nv = 0;
+      int nE = 0, nVt = 0;
       TileIter itE(P, first_g, stride_g, kBlocks), itV(P, first_g, stride_g, kBlocks);
       while (nVt < n_total && !needs_v(itV.get())) { ++nVt; itV.next(); }
       const uint64_t pol_first = policy_evict_first();
@@ -200,17 +221,25 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
       long long t0 = 0;
       bool force = false, idle = false;
+      RingPos<kRingE> rE;
+      RingPos<kRingL> rL;
+      RingPos<kRingV> rV;
+      const uint32_t bEmptyE = smem_u32(&bars->emptyE[0]), bEmptyL = smem_u32(&bars->emptyL[0]);
+      const uint32_t bEmptyV = smem_u32(&bars->emptyV[0]);
       while (nE < n_total || nVt < n_total) {
         bool did = false;
-        const int eE = nE % kRingE, eL = nE % kRingL, eV = nv % kRingV;
-        const uint32_t r_e = mbar_poll(&bars->emptyE[eE], ((nE / kRingE) & 1) ^ 1);
-        const uint32_t r_l = mbar_poll(&bars->emptyL[eL], ((nE / kRingL) & 1) ^ 1);
-        const uint32_t r_v = mbar_poll(&bars->emptyV[eV], ((nv / kRingV) & 1) ^ 1);
+        const uint32_t r_e = mbar_poll_addr(bEmptyE + rE.slot * 8, rE.par ^ 1);
+        const uint32_t r_l = mbar_poll_addr(bEmptyL + rL.slot * 8, rL.par ^ 1);
+        const uint32_t r_v = mbar_poll_addr(bEmptyV + rV.slot * 8, rV.par ^ 1);
         if (nE < n_total) {
-          const Tile t = itE.get();
-          bool ok = force || !deps || t.p == 0 || ctrE >= P.tiles_per_head;
-          if (!ok && (r_e & r_l)) { ctrE = ld_acquire(counter_of(t)); ok = ctrE >= P.tiles_per_head; }
+          bool ok = force || !deps || itE.p == 0 || ctrE >= P.tiles_per_head;
+          if (!ok && (r_e & r_l)) {
+            ctrE = ld_acquire(counter_of(itE.get()));
+            ok = ctrE >= P.tiles_per_head;
+          }
           if (ok && (force || (r_e & r_l))) {
+            const Tile t = itE.get();
+            const int eE = rE.slot, eL = rL.slot;
             asm volatile("fence.proxy.async.global;" ::: "memory");
             uint8_t* sE = smem + Lay::E + eE * kSlot;
             uint8_t* sL = smem + Lay::L + eL * kSlot;
@@ -233,25 +262,31 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             }
             stamp(P, nE, 0);
             ++nE;
+            rE.advance();
+            rL.advance();
             itE.next();
             // the next tile's counter is read now and looked at one iteration later
-            if (deps && nE < n_total && itE.get().p > 0) ctrE = ld_acquire(counter_of(itE.get()));
+            if (deps && nE < n_total && itE.p > 0) ctrE = ld_acquire(counter_of(itE.get()));
             did = true;
           }
         }
         if (nVt < n_total) {
-          const Tile t = itV.get();
-          bool ok = force || !deps || t.p == 0 || ctrV >= P.tiles_per_head;
-          if (!ok && r_v) { ctrV = ld_acquire(counter_of(t)); ok = ctrV >= P.tiles_per_head; }
+          bool ok = force || !deps || itV.p == 0 || ctrV >= P.tiles_per_head;
+          if (!ok && r_v) {
+            ctrV = ld_acquire(counter_of(itV.get()));
+            ok = ctrV >= P.tiles_per_head;
+          }
           if (ok && (force || r_v)) {
+            const Tile t = itV.get();
+            const int eV = rV.slot;
             asm volatile("fence.proxy.async.global;" ::: "memory");
             uint8_t* sV = smem + Lay::V + eV * kSlot;
             mbar_expect_tx(&bars->fullV[eV], kSlot);
             if (t.isR) tma_load_2d_hint(sV, &P.tmV, &bars->fullV[eV], 0, (t.h * m + t.idx0) * SB, pol_first);
             else tma_load_2d(sV, &P.tmY, &bars->fullV[eV], 0, (t.h * SB + t.idx0) * m);
-            ++nv;
+            rV.advance();
             do { ++nVt; itV.next(); } while (nVt < n_total && !needs_v(itV.get()));
-            if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
+            if (deps && nVt < n_total && itV.p > 0) ctrV = ld_acquire(counter_of(itV.get()));
             did = true;
           }
         }
@@ -278,24 +313,33 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       const uint32_t sE0 = smem_u32(smem + Lay::E), sL0 = smem_u32(smem + Lay::L);
       const uint32_t sV0 = smem_u32(smem + Lay::V), sP0 = smem_u32(smem + Lay::P);
       const uint32_t sOnes = smem_u32(smem + Lay::Ones);
-      int i1 = 0, i2 = 0, nv = 0;
+      int i1 = 0, i2 = 0;
       TileIter it1(P, first_g, stride_g, kBlocks), it2(P, first_g, stride_g, kBlocks);
       long long t0 = 0;
       bool force = false, idle = false;
+      RingPos<kRingE> r1E;                        // score MMA: tile i1
+      RingPos<kRingL> r1L, r2L;                   // apply MMA: tile i2
+      RingPos<kStagesS> r1S;
+      RingPos<kRingV> rV;
+      RingPos<kStagesO> r2O;
+      RingPos<2> r2P;                             // P buffer of tile i2 is i2 & 1; parity of i2 >> 1
+      uint32_t p_par = 0;
+      const uint32_t bFullE = smem_u32(&bars->fullE[0]), bFullL = smem_u32(&bars->fullL[0]);
+      const uint32_t bFullV = smem_u32(&bars->fullV[0]), bPReady = smem_u32(&bars->p_ready[0]);
+      const uint32_t bOFree = smem_u32(&bars->o_free[0]);
       while (i2 < n_total) {
         bool did = false;
-        const int c = i2 & 1, q = i2 >> 1, eL2 = i2 % kRingL, eV = nv % kRingV;
-        const int o2 = i2 % kStagesO;
-        const int eE = i1 % kRingE, eL1 = i1 % kRingL, s1 = i1 % kStagesS;
-        const uint32_t r_ready = mbar_poll(&bars->p_ready[c], q & 1);
-        const uint32_t r_of = mbar_poll(&bars->o_free[o2], ((i2 / kStagesO) & 1) ^ 1);
-        const uint32_t r_v = mbar_poll(&bars->fullV[eV], (nv / kRingV) & 1);
-        const uint32_t r_e = mbar_poll(&bars->fullE[eE], (i1 / kRingE) & 1);
-        const uint32_t r_l = mbar_poll(&bars->fullL[eL1], (i1 / kRingL) & 1);
-        if (i2 < i1) {
+        const int c = r2P.slot;
+        const uint32_t r_ready = mbar_poll_addr(bPReady + c * 8, p_par);
+        const uint32_t r_of = mbar_poll_addr(bOFree + r2O.slot * 8, r2O.par ^ 1);
+        const uint32_t r_v = mbar_poll_addr(bFullV + rV.slot * 8, rV.par);
+        const uint32_t r_e = mbar_poll_addr(bFullE + r1E.slot * 8, r1E.par);
+        const uint32_t r_l = mbar_poll_addr(bFullL + r1L.slot * 8, r1L.par);
+        if (i2 < i1 && (force || (r_ready & r_of))) {
           const Tile t = it2.get();
           const bool needV = needs_v(t);
-          if (force || (r_ready && r_of && (!needV || r_v))) {
+          if (force || !needV || r_v) {
+            const int eL2 = r2L.slot, eV = rV.slot, o2 = r2O.slot;
             const uint32_t sL = sL0 + eL2 * kSlot, sV = sV0 + eV * kSlot, sP = sP0 + c * kPBytes;
             const uint32_t tO = tmem_o + o2 * 128;
             tc_fence_after();
@@ -303,17 +347,22 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             else if (t.final_) issue_apply<B, FT, 0>(tO, sP, sV, 16, 1);
             else issue_transposed_apply<B, FT>(tO, sP, sL, sOnes);
             umma_commit(&bars->emptyL[eL2]);
-            if (needV) { umma_commit(&bars->emptyV[eV]); ++nv; }
+            if (needV) { umma_commit(&bars->emptyV[eV]); rV.advance(); }
             umma_commit(&bars->p_free[c]);
             umma_commit(&bars->o_ready[o2]);
             stamp(P, i2, 4);
             ++i2;
             it2.next();
+            r2L.advance();
+            r2O.advance();
+            r2P.advance();
+            if (r2P.slot == 0) p_par ^= 1;
             did = true;
           }
         }
-        if (i1 < n_total && i1 < i2 + kStagesS && (force || (r_e && r_l))) {
+        if (i1 < n_total && i1 < i2 + kStagesS && (force || (r_e & r_l))) {
           const Tile t = it1.get();
+          const int eE = r1E.slot, eL1 = r1L.slot, s1 = r1S.slot;
           tc_fence_after();
           const uint32_t sE = sE0 + eE * kSlot, sL = sL0 + eL1 * kSlot;
           // R: A = aR (E ring), B = K (L ring).  L: A = Qb (L ring), B = aL (E ring).
@@ -323,6 +372,9 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
           stamp(P, i1, 1);
           ++i1;
           it1.next();
+          r1E.advance();
+          r1L.advance();
+          r1S.advance();
           did = true;
         }
         if (did) {

@@ -402,18 +402,18 @@ __device__ __forceinline__ void issue_apply(uint32_t tmem_o, uint32_t sP, uint32
   const uint32_t idesc = instr_desc2(B, 64 * nb, FA, FB, 0, 1);
   constexpr int KS = B / 16;
   constexpr int ks0 = PART == 2 ? KS / 2 : 0, ks1 = PART == 1 ? KS / 2 : KS;
+  // One descriptor per operand; a k-step or tile only moves the start address (the field holds
+  // address >> 4 and shared memory ends below 2^18, so adding to the low word cannot carry out).
+  const uint64_t dP = smem_desc(sP, 16, 1024);
+  const uint64_t dX = smem_desc(sX0, x_chunk_stride, 1024);
 #pragma unroll
   for (int t = 0; t < Geo<B>::kTiles; ++t) {
 #pragma unroll
     for (int ks = ks0; ks < ks1; ++ks) {
-      const uint32_t pa = sP + (ks >> 2) * kTileBytes + t * (B * 128) + (ks & 3) * 32;
-      const uint32_t xb = sX0 + t * (B * 128) + ks * 2048;
-      if (ks == 0)
-        umma_c<false>(tmem_o + ((uint32_t)(t * 16) << 16), smem_desc(pa, 16, 1024),
-                      smem_desc(xb, x_chunk_stride, 1024), idesc);
-      else
-        umma_c<true>(tmem_o + ((uint32_t)(t * 16) << 16), smem_desc(pa, 16, 1024),
-                     smem_desc(xb, x_chunk_stride, 1024), idesc);
+      const uint64_t da = dP + (uint64_t)(((ks >> 2) * kTileBytes + t * (B * 128) + (ks & 3) * 32) >> 4);
+      const uint64_t db = dX + (uint64_t)((t * (B * 128) + ks * 2048) >> 4);
+      if (ks == 0) umma_c<false>(tmem_o + ((uint32_t)(t * 16) << 16), da, db, idesc);
+      else umma_c<true>(tmem_o + ((uint32_t)(t * 16) << 16), da, db, idesc);
     }
   }
 }
@@ -426,13 +426,16 @@ __device__ __forceinline__ void issue_transposed_apply(uint32_t tmem_o, uint32_t
   constexpr uint32_t idesc = instr_desc2(B, 64, FA, FB, 1, 1);
   constexpr uint32_t idesc1 = instr_desc2(B, 16, FA, FA, 1, 0);   // ones tile has A's format
   const uint64_t ones = smem_desc(sOnes, 16, 1024);
+  const uint64_t dP = smem_desc(sP, kTileBytes, 1024);
+  const uint64_t dX = smem_desc(sX, 16, 1024);
 #pragma unroll
   for (int t = 0; t < Geo<B>::kTiles; ++t) {
     const uint32_t d = tmem_o + ((uint32_t)(t * 16) << 16);
 #pragma unroll
     for (int ks = 0; ks < B / 16; ++ks) {
-      const uint64_t da = smem_desc(sP + t * (B * 128) + ks * 2048, kTileBytes, 1024);
-      const uint64_t db = smem_desc(sX + t * (B * 128) + ks * 2048, 16, 1024);
+      const uint64_t off = (uint64_t)((t * (B * 128) + ks * 2048) >> 4);
+      const uint64_t da = dP + off;
+      const uint64_t db = dX + off;
       if (ks == 0) {
         umma_c<false>(d, da, db, idesc);
         umma_c<false>(d + 64, da, ones, idesc1);
