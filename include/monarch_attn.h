@@ -46,7 +46,8 @@ typedef enum {
   MA_PATH_GENERIC = 1, /* fp32 SIMT kernels, fp32 states; any dtype, any N = m*b that fits smem */
   MA_PATH_TENSOR = 2,  /* tcgen05/TMA kernels, 16-bit states; f16/bf16, d = 64, m = b in
                           {32, 64, 128}: one persistent launch for all 2T half-steps (softmax and
-                          epilogue in separate warpgroups) */
+                          epilogue in separate warpgroups); bf16 with b = 32 keeps alpha_L as a
+                          hi + lo pair of bf16 arrays (one more workspace array) */
   MA_PATH_TENSOR_PHASED = 3, /* first-generation persistent kernel, one launch per half-step */
   MA_PATH_TENSOR_BASIC = 4,  /* one CTA per tile, one launch per half-step (no pipelining);
                                 m = b in {64, 128} */

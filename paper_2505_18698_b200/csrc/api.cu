@@ -133,9 +133,7 @@ static int launch_generic(const Problem& p, const void* Q, const void* K, const 
 static int resolve_path(const Problem& p, int path) {
   if (path == MA_PATH_AUTO) {
     if (fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_FUSED;
-    // b = 32 in bf16 stays on the fp32-state kernels: with 8-bit mantissas in the alpha_L state
-    // the peaky-logit configuration of that shape (C3) misses the 1e-2 tolerance on some heads.
-    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) && !(p.b == 32 && p.dtype == MA_BF16))
+    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH))
       return MA_PATH_TENSOR;
     if (generic_supported(p)) return MA_PATH_GENERIC;
     return -1;
@@ -155,7 +153,7 @@ static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_TENSOR_BASIC) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
   if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_PHASED ||
       resolved == MA_PATH_TENSOR_CHAINED)
-    return tp::workspace_bytes(p.BH, p.N, p.T);
+    return tp::workspace_bytes(p.BH, p.N, p.T, tp::uses_hilo(p.dtype, p.b));
   return 0;
 }
 

@@ -18,6 +18,14 @@
 // 16 KB staging buffer (the last R half-step stages alpha_L and y in two rounds), row statistics,
 // c-vectors, a tile of ones.
 //
+// bf16 with b = 32 (HILO): the 8-bit mantissa of alpha_L is the dominant error of a bf16 pipeline
+// when the logits are large (it is multiplied by Q into logits of size ~100), and at this shape's
+// logit scale it alone pushes some heads past 1e-2.  alpha_L is therefore stored as two bf16 arrays,
+// hi = bf16(x) and lo = bf16(x - hi) (one more staging round in the R half-steps), the L half-steps
+// load both tiles into a double-size E slot and the score MMA runs twice into the same stage; and the
+// R half-step sums (and takes the entropy over) the weights as rounded to bf16, so that the rounding
+// of a dominant weight cancels in alpha_L = sum(P K) / sum(P).
+//
 // Measured and rejected on B200 (slower than this arrangement): issuing the first half of the apply
 // MMA while the softmax is still producing the second half of P (it holds the single O stage for
 // half a softmax); writing rows to global memory straight from the epilogue threads instead of
@@ -25,6 +33,8 @@
 // softmax groups slow down by half); one store thread instead of two (the completion fence of a tile
 // is about a microsecond); separate blocking issuer threads for the two MMAs.
 #pragma once
+#include <type_traits>
+
 #include "tensor_persistent.cuh"
 
 namespace ma {
@@ -51,24 +61,31 @@ constexpr int kSlot = kTileBytes;
 // stage 128.  Shared memory: operand rings of 16 KB tiles, one P buffer per softmax group, one
 // staging buffer.  The L ring is the deepest: its tile (K, or the Q block of an L half-step) is held
 // from the load until the apply MMA of the tile has run, four to five microseconds.
-template <int B>
+// HILO (bf16 with b = 32): alpha_L travels as a hi + lo pair of 16-bit tiles, so an E slot holds
+// two tiles (32 KB) and the rings are shallower.
+template <int B, bool HILO>
 struct Cfg;
 template <>
-struct Cfg<128> {
+struct Cfg<128, false> {
   static constexpr int kRingE = 2, kRingL = 4, kRingV = 2, kStagesS = 3, kStagesO = 1;
 };
 template <>
-struct Cfg<64> {
+struct Cfg<64, false> {
   static constexpr int kRingE = 3, kRingL = 5, kRingV = 2, kStagesS = 4, kStagesO = 2;
+};
+template <>
+struct Cfg<64, true> {
+  static constexpr int kRingE = 2, kRingL = 4, kRingV = 2, kStagesS = 4, kStagesO = 2;
 };
 constexpr int kMaxRing = 6, kMaxStagesS = 4;
 
-template <int B>
+template <int B, bool HILO>
 struct Lay {
-  using C = Cfg<B>;
+  using C = Cfg<B, HILO>;
   static constexpr int kPBytes = 128 * B * 2;           // one P buffer (128 rows x B columns)
+  static constexpr int kSlotE = HILO ? 2 * kSlot : kSlot;
   static constexpr int E = 0;
-  static constexpr int L = E + C::kRingE * kSlot;
+  static constexpr int L = E + C::kRingE * kSlotE;
   static constexpr int V = L + C::kRingL * kSlot;
   static constexpr int P = V + C::kRingV * kSlot;       // two P buffers
   static constexpr int Stage = P + 2 * kPBytes;         // 16 KB
@@ -158,8 +175,10 @@ template <typename T, int B, int SB>
 __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_constant__ Params P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  using Lay = tp2::Lay<B>;
-  using C = Cfg<B>;
+  constexpr bool HILO = std::is_same<T, __nv_bfloat16>::value && SB == 32;
+  using Lay = tp2::Lay<B, HILO>;
+  using C = Cfg<B, HILO>;
+  constexpr int kSlotE = Lay::kSlotE;
   constexpr int kRingE = C::kRingE, kRingL = C::kRingL, kRingV = C::kRingV;
   constexpr int kStagesS = C::kStagesS, kStagesO = C::kStagesO;
   constexpr int kPBytes = Lay::kPBytes;
@@ -205,7 +224,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
   const int stride_g = gridDim.x;
   const int n_total = first_g < P.g_end ? (P.g_end - first_g + stride_g - 1) / stride_g : 0;
   auto needs_v = [&](const Tile& t) { return t.isR ? t.withV : t.final_; };
-  auto rounds_of = [&](const Tile& t) { return (t.isR && t.withV) ? 2 : 1; };   // staging rounds
+  // staging rounds of a tile: alpha_L (R) or alpha_R / Y (L), the low halves of alpha_L, y
+  auto rounds_of = [&](const Tile& t) { return t.isR ? 1 + (HILO ? 1 : 0) + (t.withV ? 1 : 0) : 1; };
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -241,11 +261,11 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             const Tile t = itE.get();
             const int eE = rE.slot, eL = rL.slot;
             asm volatile("fence.proxy.async.global;" ::: "memory");
-            uint8_t* sE = smem + Lay::E + eE * kSlot;
+            uint8_t* sE = smem + Lay::E + eE * kSlotE;
             uint8_t* sL = smem + Lay::L + eL * kSlot;
             const bool needC = !t.first;
             float* sC = reinterpret_cast<float*>(smem + Lay::Vec) + eL * 128;
-            mbar_expect_tx(&bars->fullE[eE], kSlot);
+            mbar_expect_tx(&bars->fullE[eE], (HILO && !t.isR) ? 2 * kSlot : kSlot);
             mbar_expect_tx(&bars->fullL[eL], kSlot + (needC ? 512 : 0));
             if (t.isR) {
               const int row0 = (t.h * m + t.idx0) * SB;
@@ -256,6 +276,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
               const int row0 = (t.h * SB + t.idx0) * m;
               bulk_load_1d(sC, P.cL + row0, 512, &bars->fullL[eL]);
               tma_load_2d(sE, &P.tmAL, &bars->fullE[eE], 0, row0);
+              if (HILO) tma_load_2d(sE + kSlot, &P.tmALlo, &bars->fullE[eE], 0, row0);
 #pragma unroll
               for (int tt = 0; tt < kBlocks; ++tt)
                 tma_load_3d(sL + tt * (SB * 128), &P.tmQs, &bars->fullL[eL], 0, t.idx0 + tt, t.h * m);
@@ -364,9 +385,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
           const Tile t = it1.get();
           const int eE = r1E.slot, eL1 = r1L.slot, s1 = r1S.slot;
           tc_fence_after();
-          const uint32_t sE = sE0 + eE * kSlot, sL = sL0 + eL1 * kSlot;
+          const uint32_t sE = sE0 + eE * kSlotE, sL = sL0 + eL1 * kSlot;
           // R: A = aR (E ring), B = K (L ring).  L: A = Qb (L ring), B = aL (E ring).
           issue_scores<B, FT>(tmem + s1 * B, t.isR ? sE : sL, t.isR ? sL : sE);
+          if (HILO && !t.isR) issue_scores<B, FT, FT, true>(tmem + s1 * B, sL, sE + kSlot);
           umma_commit(&bars->emptyE[eE]);
           umma_commit(&bars->s_ready[s1]);
           stamp(P, i1, 1);
@@ -414,7 +436,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             for (int tt = 0; tt < kBlocks; ++tt) {
               const uint8_t* src = sStage + tt * (SB * 128);
               if (t.isR) {
-                tma_store_3d(r == 0 ? &P.tmALs : &P.tmYs, src, 0, t.idx0 + tt, t.h * SB);
+                tma_store_3d(r == 0 ? &P.tmALs : ((HILO && r == 1) ? &P.tmALlos : &P.tmYs), src, 0,
+                             t.idx0 + tt, t.h * SB);
               } else if (t.final_) {
                 tma_store_3d_hint(&P.tmOut, src, 0, t.idx0 + tt, t.h * m, pol_first);
               } else {
@@ -500,7 +523,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             for (int i = 0; i < 16; ++i) {
               const float2 x = make_float2(sv[2 * i], sv[2 * i + 1]);
               const float2 zz = ffma2(x, f2, off2);
-              const float2 pp = exp2_pair(zz, i);
+              float2 pp = exp2_pair(zz, i);
+              // HILO: sums and entropy are taken over the weights as MMA 2 will see them (16-bit),
+              // so that the rounding of a dominant weight cancels in alpha_L = sum(P K) / sum(P)
+              if (HILO) pp = unpack2<T>(pack2<T>(pp.x, pp.y));
               z2[i & 1] = ffma2(pp, x, z2[i & 1]);
               a2[i & 1] = fadd2(a2[i & 1], pp);
               sv[2 * i] = pp.x;
@@ -621,19 +647,25 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       const bool scaled = t.isR || t.final_;
       float c1 = 0.f;
       if (!scaled) c1 = tmem_ld1(tO + 64);
+      float buf[2][32];
       for (int rr = 0; rr < nr; ++rr) {
-        float buf[2][32];
-        tmem_ld32(tO + 64 * rr, buf[0]);
-        tmem_ld32(tO + 64 * rr + 32, buf[1]);
-        tmem_ld_wait();
+        // what this round stages: 0 = the rows (columns 0-63 of O), 1 = low halves of the same
+        // values (alpha_L as a hi + lo pair), 2 = y (columns 64-127)
+        const int kind = (t.isR && rr > 0) ? ((HILO && rr == 1) ? 1 : 2) : 0;
+        if (kind != 1) {
+          const int col = kind == 2 ? 64 : 0;
+          tmem_ld32(tO + col, buf[0]);
+          tmem_ld32(tO + col + 32, buf[1]);
+          tmem_ld_wait();
+        }
         if (rr == nr - 1) {                      // O is in registers: the next apply MMA may run
           tc_fence_before();
           mbar_arrive(&bars->o_free[o]);
         }
         wait_or_abort(&bars->stage_free, ((round + rr) & 1) ^ 1, bars, P.status, 35);
-        if (t.final_) {
-          store_row32<T>(sStage, srow, 0, buf[0], inv_s);
-          store_row32<T>(sStage, srow, 32, buf[1], inv_s);
+        if (kind == 1) {
+          store_row32_lo<T>(sStage, srow, 0, buf[0], inv_s);
+          store_row32_lo<T>(sStage, srow, 32, buf[1], inv_s);
         } else if (scaled) {
           store_row32<T>(sStage, srow, 0, buf[0], inv_s);
           store_row32<T>(sStage, srow, 32, buf[1], inv_s);
@@ -670,7 +702,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
 template <typename T, int B, int SB>
 inline cudaError_t launch_kernel(const Params& P, int grid, cudaStream_t st) {
   const void* fn = (const void*)monarch_decoupled<T, B, SB>;
-  constexpr int kSmem = Lay<B>::kSmem;
+  constexpr int kSmem = Lay<B, std::is_same<T, __nv_bfloat16>::value && SB == 32>::kSmem;
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
   if (e != cudaSuccess) return e;
   monarch_decoupled<T, B, SB><<<grid, kThreads, kSmem, st>>>(P);

@@ -340,6 +340,24 @@ __device__ __forceinline__ void store_row32(uint8_t* tile, int srow, int col0, c
     *reinterpret_cast<uint4*>(base + (((c0 + c) ^ (srow & 7)) << 4)) = q;
   }
 }
+// The low halves of a hi + lo pair: what 16-bit rounding of v * mul dropped, rounded to 16 bits.
+template <typename T>
+__device__ __forceinline__ void store_row32_lo(uint8_t* tile, int srow, int col0, const float* v,
+                                               float mul) {
+  uint8_t* base = tile + (col0 >> 6) * kTileBytes + srow * 128;
+  const int c0 = (col0 & 63) >> 3;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t q[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float x0 = v[8 * c + 2 * e] * mul, x1 = v[8 * c + 2 * e + 1] * mul;
+      const float2 hi = unpack2<T>(pack2<T>(x0, x1));
+      q[e] = pack2<T>(x0 - hi.x, x1 - hi.y);
+    }
+    *reinterpret_cast<uint4*>(base + (((c0 + c) ^ (srow & 7)) << 4)) = make_uint4(q[0], q[1], q[2], q[3]);
+  }
+}
 // Same without scaling.
 template <typename T>
 __device__ __forceinline__ void store_row32(uint8_t* tile, int srow, int col0, const float* v) {
@@ -377,7 +395,8 @@ template <int B> struct Geo {
 
 // Issues MMA 1 (scores): both operands K-major [rows][64] tiles, K = d = 64 in four steps.
 // FA / FB: element format of the A / B operand (0 f16, 1 bf16); the two may differ.
-template <int B, int FA, int FB = FA>
+// ACC0: accumulate onto what the stage already holds (second half of a hi + lo operand pair).
+template <int B, int FA, int FB = FA, bool ACC0 = false>
 __device__ __forceinline__ void issue_scores(uint32_t tmem_s, uint32_t sA, uint32_t sB) {
   constexpr uint32_t idesc = instr_desc2(B, B, FA, FB, 0, 0);
 #pragma unroll
@@ -386,7 +405,7 @@ __device__ __forceinline__ void issue_scores(uint32_t tmem_s, uint32_t sA, uint3
     const uint64_t db = smem_desc(sB + t * (B * 128), 16, 1024);
 #pragma unroll
     for (int ks = 0; ks < kD / 16; ++ks) {
-      if (ks == 0) umma_c<false>(tmem_s + ((uint32_t)(t * 16) << 16), da, db, idesc);
+      if (ks == 0) umma_c<ACC0>(tmem_s + ((uint32_t)(t * 16) << 16), da, db, idesc);
       else umma_c<true>(tmem_s + ((uint32_t)(t * 16) << 16), da + 2 * ks, db + 2 * ks, idesc);
     }
   }

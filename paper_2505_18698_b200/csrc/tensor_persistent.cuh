@@ -63,6 +63,7 @@ struct Params {
   CUtensorMap tmALs, tmYs;                       // 3D stores of aL / y (rows m apart)
   CUtensorMap tmQs;                              // 3D strided view of Q (load)
   CUtensorMap tmARs, tmOut;                      // 3D strided stores of aR / Y
+  CUtensorMap tmALlo, tmALlos;                   // low halves of alpha_L (second-generation kernel, bf16, b = 32)
   float* cL;
   float* cR;
   uint8_t *aL, *aR, *y;  // state arrays (for L2 discards once a tile has been consumed)
@@ -704,8 +705,11 @@ inline bool supported(int N, int d, int b, int m, int dtype, int BH) {
 inline size_t counters_bytes(int BH, int T) {
   return ((size_t)2 * T * BH * sizeof(int) + 255) / 256 * 256;
 }
-inline size_t workspace_bytes(int BH, int N, int T) {
-  return ws_layout(nullptr, BH, N).bytes + counters_bytes(BH, T);
+// bf16 with b = 32 keeps alpha_L as a hi + lo pair of 16-bit arrays (see tensor_decoupled.cuh).
+inline bool uses_hilo(int dtype, int b) { return dtype == 2 && b == 32; }
+inline size_t hilo_bytes(int BH, int N) { return ((size_t)BH * N * kD * 2 + 255) / 256 * 256; }
+inline size_t workspace_bytes(int BH, int N, int T, bool hilo) {
+  return ws_layout(nullptr, BH, N).bytes + counters_bytes(BH, T) + (hilo ? hilo_bytes(BH, N) : 0);
 }
 
 // Defined in tensor_decoupled.cuh (the second-generation kernel, same Params).
@@ -720,6 +724,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   int* counters = (int*)((char*)ws + w.bytes);
   const int m = N / SB;            // = SB on this path
   const uint64_t rows = (uint64_t)BH * N;
+  void* aLlo = (char*)counters + counters_bytes(BH, T_steps);   // used when uses_hilo(dtype, SB)
   Params P;
   bool ok = make_map_rows(&P.tmQ, dtype, (void*)Q, rows) && make_map_rows(&P.tmK, dtype, (void*)K, rows) &&
             make_map_rows(&P.tmV, dtype, (void*)V, rows) && make_map_rows(&P.tmAR, dtype, w.aR, rows) &&
@@ -729,6 +734,9 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
             make_map_strided(&P.tmQs, dtype, (void*)Q, SB, (uint64_t)BH * m, SB) &&
             make_map_strided(&P.tmARs, dtype, w.aR, SB, (uint64_t)BH * m, SB) &&
             make_map_strided(&P.tmOut, dtype, Y, SB, (uint64_t)BH * m, SB);
+  if (ok && uses_hilo(dtype, SB))
+    ok = make_map_rows(&P.tmALlo, dtype, aLlo, rows) &&
+         make_map_strided(&P.tmALlos, dtype, aLlo, m, (uint64_t)BH * SB, SB);
   if (!ok) return 7;
   P.aL = (uint8_t*)w.aL; P.aR = (uint8_t*)w.aR; P.y = (uint8_t*)w.y; P.out = (uint8_t*)Y;
   P.cL = w.cL; P.cR = w.cR; P.status = w.status; P.counters = counters;
