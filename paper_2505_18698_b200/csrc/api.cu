@@ -133,7 +133,11 @@ static int launch_generic(const Problem& p, const void* Q, const void* K, const 
 static int resolve_path(const Problem& p, int path) {
   if (path == MA_PATH_AUTO) {
     if (fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_FUSED;
-    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH))
+    // bf16 with b = 32 and more than two rounds stays on the fp32-state kernels: on the peaky-logit
+    // recipe of that shape the 8-bit mantissa of alpha_R (used twice from T = 3 on) costs 4e-2 on
+    // the worst head; up to T = 2 the hi + lo alpha_L of the tensor path keeps it under 1e-2.
+    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) &&
+        !(p.b == 32 && p.dtype == MA_BF16 && p.T > 2))
       return MA_PATH_TENSOR;
     if (generic_supported(p)) return MA_PATH_GENERIC;
     return -1;

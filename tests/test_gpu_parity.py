@@ -116,6 +116,30 @@ def test_tensor_path_block_32_on_64_row_tiles(T, dtype, batch, heads, path):
     check(batch, heads, 1024, 64, 32, T, dtype, rank=16, s=1.5, seed=3 * T + heads, path=path)
 
 
+@pytest.mark.parametrize("T", [1, 2])
+def test_bf16_block_32_keeps_alpha_l_as_hi_lo_pair(T):
+    """bf16 with b = 32 on the tensor path stores alpha_L as a bf16 hi + lo pair and sums the rounded
+    weights: on the peaky-logit recipe of that shape it must stay inside the 16-bit tolerance, and
+    its workspace holds one more N x d array than the f16 one."""
+    w = wl.WORKLOADS["C3"]
+    err = check(2, 12, w.N, w.d, w.b, T, "bf16", w.rank, w.s, seed=700 + T,
+                path=binding.MA_PATH_TENSOR)
+    print(f"T={T}: {err:.3e}")
+    need_bf16 = binding.monarch_attn_workspace_bytes(2, 12, w.N, w.d, w.b, T, torch.bfloat16,
+                                                     binding.MA_PATH_TENSOR)
+    need_f16 = binding.monarch_attn_workspace_bytes(2, 12, w.N, w.d, w.b, T, torch.float16,
+                                                    binding.MA_PATH_TENSOR)
+    assert need_bf16 - need_f16 == 2 * 12 * w.N * w.d * 2
+
+
+def test_auto_keeps_bf16_block_32_with_three_rounds_on_fp32_states():
+    """From T = 3 on, bf16 alpha_R costs 4e-2 on the worst head of this recipe on the tensor path
+    (hi + lo covers alpha_L only); AUTO must take the fp32-state kernels there."""
+    w = wl.WORKLOADS["C3"]
+    err = check(2, 12, w.N, w.d, w.b, 3, "bf16", w.rank, w.s, seed=703)
+    assert err < 5e-3
+
+
 def test_tensor_paths_agree_bit_for_bit_between_launch_modes():
     """One persistent launch with dependency counters computes exactly what one launch per
     half-step computes (same kernel, same tile order inside a half-step)."""
