@@ -89,6 +89,24 @@ int monarch_attn_fwd_host(const void* Q_host, const void* K_host, const void* V_
 /* Scratch the no-allocation entry point below carries inside the library image, in bytes. */
 #define MONARCH_ATTN_NOALLOC_SCRATCH_BYTES (8u << 20)
 
+/* Forward pass on a post-padded sequence (Appendix C.3 "Padding and Masking").
+ *
+ * When the sequence length is not a multiple of the block size, the caller pads Q, K, V with rows
+ * (zeros, or any finite values) up to N = ceil(n_valid / b) * b and passes the number of real rows
+ * as n_valid.  The mask of that appendix (minus infinity added to Z_R for key columns
+ * b k + i >= n_valid, Eq. 7) makes every column of the Monarch matrix beyond n_valid exactly zero,
+ * so padded rows of V never reach the output.  Rows n_valid .. N-1 of Y are computed from the padded
+ * rows of Q and carry no meaning.
+ *
+ * Q, K, V, Y: DEVICE pointers, [batch][heads][N][d], same rules as monarch_attn_fwd_ex.
+ * n_valid must satisfy N - b < n_valid <= N (less than one block of padding, so that every key
+ * block keeps a valid key; anything else is MA_ERR_SHAPE).  n_valid == N is the unpadded pass.
+ * Runs on the generic kernels (any dtype, m need not equal b); workspace as for
+ * monarch_attn_fwd_ex with path MA_PATH_GENERIC.  Asynchronous on `stream`. */
+int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y, int batch,
+                            int heads, int N, int d, int b, int T, int dtype, float softmax_scale,
+                            int n_valid, void* workspace, size_t workspace_bytes, void* stream);
+
 /* The same forward pass for callers that must not allocate device memory.  (The paper has no
  * counterpart: this is a deployment variant of the library, not a step of the method.)
  *

@@ -56,6 +56,8 @@ def load_library(path: str = LIB_PATH):
     lib.monarch_attn_workspace_bytes.restype = sz
     lib.monarch_attn_fwd_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, sz, vp]
     lib.monarch_attn_fwd_ex.restype = i
+    lib.monarch_attn_fwd_padded.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, sz, vp]
+    lib.monarch_attn_fwd_padded.restype = i
     lib.monarch_attn_fwd_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
     lib.monarch_attn_fwd_host.restype = i
     lib.monarch_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
@@ -140,6 +142,30 @@ def monarch_attn_fwd_ex(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, wo
     _check(lib.monarch_attn_fwd_ex(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                    batch, heads, N, d, b, T, code, float(softmax_scale), int(path),
                                    workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
+    return Y
+
+
+def monarch_attn_fwd_padded(Q, K, V, b, T, n_valid, softmax_scale=None, workspace=None, Y=None,
+                            stream=None):
+    """Forward pass on post-padded CUDA tensors [batch, heads, N, d] with N a multiple of b and
+    n_valid real rows (N - b < n_valid <= N): keys beyond n_valid are masked out (App. C.3).
+    Returns Y (rows n_valid.. carry no meaning)."""
+    lib = load_library()
+    if not Q.is_cuda:
+        raise MonarchAttnError(-2, "monarch_attn_fwd_padded needs CUDA tensors; there is no CPU path")
+    batch, heads, N, d = _shape_of(Q, K, V)
+    code = _TORCH_TO_CODE[Q.dtype]
+    if softmax_scale is None:
+        softmax_scale = 1.0 / math.sqrt(d)
+    if Y is None:
+        Y = torch.empty_like(Q)
+    if workspace is None:
+        need = lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_GENERIC)
+        workspace = torch.empty(max(int(need), 256), dtype=torch.uint8, device=Q.device)
+    _check(lib.monarch_attn_fwd_padded(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                       batch, heads, N, d, b, T, code, float(softmax_scale),
+                                       int(n_valid), workspace.data_ptr(), workspace.numel(),
+                                       _stream_ptr(stream)))
     return Y
 
 

@@ -23,6 +23,7 @@ static inline int esize(int dtype) { return dtype == MA_F32 ? 4 : 2; }
 
 struct Problem {
   int batch, heads, N, d, b, T, dtype, m, BH;
+  int n_valid;   // keys b k + i >= n_valid are masked out (App. C.3); N when there is no padding
 };
 
 static int validate_shape(int batch, int heads, int N, int d, int b, int T, int dtype, Problem* p) {
@@ -30,7 +31,7 @@ static int validate_shape(int batch, int heads, int N, int d, int b, int T, int 
   if (batch <= 0 || heads <= 0 || N <= 0 || d <= 0 || b <= 0 || T < 1) return MA_ERR_SHAPE;
   if (N % b != 0) return MA_ERR_SHAPE;
   if ((long long)batch * heads > 0x7fffffffLL / 2) return MA_ERR_SHAPE;
-  *p = Problem{batch, heads, N, d, b, T, dtype, N / b, batch * heads};
+  *p = Problem{batch, heads, N, d, b, T, dtype, N / b, batch * heads, N};
   return MA_OK;
 }
 
@@ -87,7 +88,7 @@ static int launch_generic_t(const Problem& p, const TIn* Q, const TIn* K, const 
       return MA_ERR_CUDA;                                                                      \
     r_step_kernel<TIn, FIRST, WITHV><<<gr, kThreads, rs, st>>>(Q, K, V, w.aR, w.cR, w.aL,     \
                                                                 w.cL, w.y, p.N, p.d, p.b, p.m, \
-                                                                scale);                        \
+                                                                scale, p.n_valid);             \
   } while (0)
     if (first && last) MA_LAUNCH_R(true, true);
     else if (first) MA_LAUNCH_R(true, false);
@@ -253,6 +254,23 @@ int monarch_attn_fwd_ex(const void* Q, const void* K, const void* V, void* Y, in
   int r = resolve_path(p, path);
   if (r < 0) return MA_ERR_UNSUPPORTED;
   return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y, int batch,
+                            int heads, int N, int d, int b, int T, int dtype, float softmax_scale,
+                            int n_valid, void* workspace, size_t workspace_bytes, void* stream) {
+  Problem p;
+  int rc = validate_shape(batch, heads, N, d, b, T, dtype, &p);
+  if (rc != MA_OK) return rc;
+  // less than one block of padding: every key block keeps at least one valid key
+  if (n_valid > N || n_valid <= N - b) return MA_ERR_SHAPE;
+  rc = check_ptrs(Q, K, V, Y, p);
+  if (rc != MA_OK) return rc;
+  if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
+  if (!generic_supported(p)) return MA_ERR_UNSUPPORTED;
+  p.n_valid = n_valid;
+  return fwd_ex(Q, K, V, Y, p, softmax_scale, MA_PATH_GENERIC, workspace, workspace_bytes,
+                (cudaStream_t)stream);
 }
 
 int monarch_attn_fwd(const void* Q, const void* K, const void* V, void* Y, int batch, int heads,

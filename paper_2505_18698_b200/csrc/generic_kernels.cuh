@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(kThreads)
 r_step_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
               const float* __restrict__ aR, const float* __restrict__ cR,
               float* __restrict__ aL, float* __restrict__ cL, float* __restrict__ y,
-              int N, int d, int b, int m, float scale) {
+              int N, int d, int b, int m, float scale, int n_valid) {
   extern __shared__ float smem[];
   const int k = blockIdx.x, h = blockIdx.y;
   const int dp = d + 1;
@@ -91,7 +91,8 @@ r_step_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
       float acc = 0.f;
       const float* kr = Ks + i * dp;
       for (int v = 0; v < d; ++v) acc = fmaf(as[v], kr[v], acc);
-      float z = acc * f;
+      // padding mask (App. C.3, post-padding): key columns b k + i >= n_valid get -inf
+      float z = (k * b + i < n_valid) ? acc * f : -INFINITY;
       zs[i] = z;
       zmax = fmaxf(zmax, z);
     }
@@ -99,10 +100,11 @@ r_step_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
     float s = 0.f, sz = 0.f;
     for (int i = lane; i < b; i += 32) {
       float z = zs[i];
-      float p = expf(z - zmax);
+      const bool valid = z > -INFINITY;
+      float p = valid ? expf(z - zmax) : 0.f;
       zs[i] = p;
       s += p;
-      sz = fmaf(p, z, sz);
+      if (valid) sz = fmaf(p, z, sz);            // 0 log 0 = 0 for masked keys
     }
     s = warp_sum(s);
     sz = warp_sum(sz);

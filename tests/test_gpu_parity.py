@@ -297,3 +297,43 @@ def test_bounded_wait_runs_out_and_reports_timeout():
     assert binding.monarch_attn_device_status(ws) == 0
     ref = mo.monarch_attention(Q, K, V, 64, 2)
     assert rel_err(Y.float().cpu().numpy().astype(np.float64), ref) <= 1e-2
+
+
+# ------------------------------------------------------------------ padding and masking (App. C.3)
+@pytest.mark.parametrize("n_valid,b,d,T,dtype", [
+    (197, 14, 64, 2, "f32"),     # the ViT shape: N' = 210, m = 15
+    (197, 14, 64, 3, "bf16"),
+    (250, 16, 72, 3, "f16"),     # a DiT-like head width, N' = 256
+    (1000, 32, 64, 2, "bf16"),   # N' = 1024
+    (380, 24, 64, 1, "f32"),     # m = 16 != b
+    (61, 8, 16, 2, "f32"), (64, 8, 16, 2, "f32"),   # ragged and exact
+])
+def test_padded_sequences_match_masked_oracle(n_valid, b, d, T, dtype):
+    """Post-padded inputs with the key mask of App. C.3: valid rows match the oracle's masked
+    forward pass, and what sits in the padded rows of K and V cannot reach them."""
+    N = -(-n_valid // b) * b
+    Q, K, V = wl.make_qkv(2, 3, N, d, dtype, min(8, d), 1.0, seed=n_valid + T)
+    K[:, :, n_valid:] = wl.round_to_dtype(np.float32(3.0), dtype)      # junk in the padding
+    V[:, :, n_valid:] = wl.round_to_dtype(np.float32(-50.0), dtype)
+    Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))
+    Y = binding.monarch_attn_fwd_padded(Qd, Kd, Vd, b, T, n_valid).float().cpu().numpy().astype(np.float64)
+    ref = mo.monarch_attention(Q, K, V, b, T, n_valid=n_valid)
+    assert np.isfinite(Y[:, :, :n_valid]).all()
+    err = rel_err(Y[:, :, :n_valid], ref[:, :, :n_valid])
+    assert err <= TOL[dtype], err
+    # same valid rows whatever the padding holds
+    K2, V2 = K.copy(), V.copy()
+    K2[:, :, n_valid:] = 0
+    V2[:, :, n_valid:] = 0
+    Y2 = binding.monarch_attn_fwd_padded(Qd, binding.to_device(K2, dtype), binding.to_device(V2, dtype),
+                                         b, T, n_valid).float().cpu().numpy()
+    assert np.array_equal(Y2[:, :, :n_valid], Y[:, :, :n_valid].astype(np.float32))
+
+
+def test_padded_entry_point_rejects_more_than_one_block_of_padding():
+    Q, K, V = wl.make_qkv(1, 1, 64, 16, "f32", 4, 1.0, seed=1)
+    Qd, Kd, Vd = (binding.to_device(x, "f32") for x in (Q, K, V))
+    for bad in (56, 0, 65):
+        with pytest.raises(binding.MonarchAttnError) as e:
+            binding.monarch_attn_fwd_padded(Qd, Kd, Vd, 8, 2, bad)
+        assert e.value.code == 2      # MA_ERR_SHAPE
