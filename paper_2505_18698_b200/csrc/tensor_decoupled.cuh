@@ -251,13 +251,15 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         const uint32_t r_e = mbar_poll_addr(bEmptyE + rE.slot * 8, rE.par ^ 1);
         const uint32_t r_l = mbar_poll_addr(bEmptyL + rL.slot * 8, rL.par ^ 1);
         const uint32_t r_v = mbar_poll_addr(bEmptyV + rV.slot * 8, rV.par ^ 1);
-        if (nE < n_total) {
+        if (nE < n_total && (force || (r_e & r_l))) {
+          // (the prefetched counter is looked at only once the slots are free: by then its load
+          // has long landed and the thread does not stall on it)
           bool ok = force || !deps || itE.p == 0 || ctrE >= P.tiles_per_head;
-          if (!ok && (r_e & r_l)) {
+          if (!ok) {
             ctrE = ld_acquire(counter_of(itE.get()));
             ok = ctrE >= P.tiles_per_head;
           }
-          if (ok && (force || (r_e & r_l))) {
+          if (ok) {
             const Tile t = itE.get();
             const int eE = rE.slot, eL = rL.slot;
             asm volatile("fence.proxy.async.global;" ::: "memory");
@@ -291,13 +293,13 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             did = true;
           }
         }
-        if (nVt < n_total) {
+        if (nVt < n_total && (force || r_v)) {
           bool ok = force || !deps || itV.p == 0 || ctrV >= P.tiles_per_head;
-          if (!ok && r_v) {
+          if (!ok) {
             ctrV = ld_acquire(counter_of(itV.get()));
             ok = ctrV >= P.tiles_per_head;
           }
-          if (ok && (force || r_v)) {
+          if (ok) {
             const Tile t = itV.get();
             const int eV = rV.slot;
             asm volatile("fence.proxy.async.global;" ::: "memory");
