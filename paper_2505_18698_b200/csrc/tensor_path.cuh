@@ -306,10 +306,14 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
   return p;
 }
 // Pair i of a chunk: one pair in kPolyEvery takes the polynomial, the others ex2.approx
-// (i is a compile-time constant after unrolling).
-constexpr int kPolyEvery = 4;
+// (i is a compile-time constant after unrolling; 0 = never).  Alone on an SM the softmax pass is
+// bound by the special-function pipe and one pair in four on the polynomial is the fastest mix;
+// inside the persistent kernels it is bound by instruction issue (the pipe sits at 20 %), the
+// polynomial's twelve instructions cost more than the two ex2 they replace, and "never" measured
+// 4 % faster on the whole call at b = 128.
+constexpr int kPolyEvery = 0;
 __device__ __forceinline__ float2 exp2_pair(float2 z, int i) {
-  if (i % kPolyEvery == kPolyEvery - 1) return exp2_poly2(z);
+  if (kPolyEvery > 0 && i % (kPolyEvery > 0 ? kPolyEvery : 1) == kPolyEvery - 1) return exp2_poly2(z);
   return make_float2(fast_exp2(z.x), fast_exp2(z.y));
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
