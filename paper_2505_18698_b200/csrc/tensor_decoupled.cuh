@@ -502,6 +502,48 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
           inv_c = cr > 1e-30f ? 1.f / cr : 0.f;
         }
         f = P.scale * inv_c * kLog2e;
+        float2 z2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        if constexpr (SB == B) {
+          // Every row owns all B columns: 16-column chunks, the load of the next chunk in flight
+          // while the current one is worked on (TMEM reads compete with the MMAs' accumulator
+          // traffic and are the longest stall of this pass).  Measured: 2 % on the whole call; the
+          // same change in the L half-steps costs registers (spills) and loses more than it gains.
+          constexpr int NC16 = B / 16;
+          float* b0 = buf;
+          float* b1 = buf + 16;
+          tmem_ld16(tS, b0);
+#pragma unroll
+          for (int cc = 0; cc < NC16; ++cc) {
+            float* cur = (cc & 1) ? b1 : b0;
+            float* nxt = (cc & 1) ? b0 : b1;
+            tmem_ld_wait();
+            tmem_ld16(tS + 16 * ((cc + 1) % NC16), nxt);     // wraps to the first chunk of pass 2
+#pragma unroll
+            for (int i = 0; i < 8; ++i) m4[i & 3] = max3(m4[i & 3], cur[2 * i], cur[2 * i + 1]);
+          }
+          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+          const float2 f2 = make_float2(f, f), off2 = make_float2(-mx * f, -mx * f);
+          // the apply MMA of this group's previous tile must be done with the P buffer
+          wait_or_abort(&bars->p_free[c], (q & 1) ^ 1, bars, P.status, 33);
+#pragma unroll
+          for (int cc = 0; cc < NC16; ++cc) {
+            float* cur = (cc & 1) ? b1 : b0;
+            float* nxt = (cc & 1) ? b0 : b1;
+            tmem_ld_wait();
+            if (cc + 1 < NC16) tmem_ld16(tS + 16 * (cc + 1), nxt);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float2 x = make_float2(cur[2 * i], cur[2 * i + 1]);
+              const float2 zz = ffma2(x, f2, off2);
+              const float2 pp = exp2_pair(zz, i);
+              z2[i & 1] = ffma2(pp, x, z2[i & 1]);
+              a2[i & 1] = fadd2(a2[i & 1], pp);
+              cur[2 * i] = pp.x;
+              cur[2 * i + 1] = pp.y;
+            }
+            store_row16<T>(sP, srow, 16 * cc, cur);
+          }
+        } else {
 #pragma unroll
         for (int cc = 0; cc < NC; ++cc) {
           if (!mine(cc)) continue;
@@ -512,7 +554,6 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         }
         mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         const float2 f2 = make_float2(f, f), off2 = make_float2(-mx * f, -mx * f);
-        float2 z2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
         // the apply MMA of this group's previous tile must be done with the P buffer
         wait_or_abort(&bars->p_free[c], (q & 1) ^ 1, bars, P.status, 33);
 #pragma unroll
@@ -539,6 +580,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             for (int i = 0; i < 32; ++i) sv[i] = 0.f;
           }
           store_row32<T>(sP, srow, 32 * cc, sv);
+        }
         }
         sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
         sz = (z2[0].x + z2[0].y) + (z2[1].x + z2[1].y);

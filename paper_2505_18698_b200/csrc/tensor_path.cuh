@@ -199,6 +199,18 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
       : "r"(taddr)
       : "memory");
 }
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, "
+      "%12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -341,6 +353,21 @@ __device__ __forceinline__ void store_row32(uint8_t* tile, int srow, int col0, c
     q.y = pack2<T>(b.x, b.y);
     q.z = pack2<T>(cc.x, cc.y);
     q.w = pack2<T>(d.x, d.y);
+    *reinterpret_cast<uint4*>(base + (((c0 + c) ^ (srow & 7)) << 4)) = q;
+  }
+}
+// 16 consecutive columns, unscaled.
+template <typename T>
+__device__ __forceinline__ void store_row16(uint8_t* tile, int srow, int col0, const float* v) {
+  uint8_t* base = tile + (col0 >> 6) * kTileBytes + srow * 128;
+  const int c0 = (col0 & 63) >> 3;
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    uint4 q;
+    q.x = pack2<T>(v[8 * c + 0], v[8 * c + 1]);
+    q.y = pack2<T>(v[8 * c + 2], v[8 * c + 3]);
+    q.z = pack2<T>(v[8 * c + 4], v[8 * c + 5]);
+    q.w = pack2<T>(v[8 * c + 6], v[8 * c + 7]);
     *reinterpret_cast<uint4*>(base + (((c0 + c) ^ (srow & 7)) << 4)) = q;
   }
 }
