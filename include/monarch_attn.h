@@ -89,6 +89,18 @@ int monarch_attn_fwd_host(const void* Q_host, const void* K_host, const void* V_
 /* Scratch the no-allocation entry point below carries inside the library image, in bytes. */
 #define MONARCH_ATTN_NOALLOC_SCRATCH_BYTES (8u << 20)
 
+/* Forward pass on tensors laid out [batch][N][heads][d] (the layout a transformer layer has after
+ * its QKV projection, before any transpose); the paper's method is per head (Sec. 3), so only the
+ * addressing changes.  Q, K, V, Y: DEVICE pointers to contiguous [batch][N][heads][d] arrays of
+ * `dtype`, 16-byte aligned, Y not overlapping an input.  `path`: MA_PATH_AUTO, MA_PATH_TENSOR (the
+ * second-generation kernel: the head becomes a column offset in the TMA tensor maps) or
+ * MA_PATH_GENERIC; other paths give MA_ERR_UNSUPPORTED.  Workspace as for monarch_attn_fwd_ex with
+ * the same path (monarch_attn_workspace_bytes does not depend on the layout).  Everything else as
+ * monarch_attn_fwd_ex.  Asynchronous on `stream`. */
+int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, int batch, int N,
+                          int heads, int d, int b, int T, int dtype, float softmax_scale, int path,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
 /* Forward pass on a post-padded sequence (Appendix C.3 "Padding and Masking").
  *
  * When the sequence length is not a multiple of the block size, the caller pads Q, K, V with rows

@@ -56,6 +56,8 @@ def load_library(path: str = LIB_PATH):
     lib.monarch_attn_workspace_bytes.restype = sz
     lib.monarch_attn_fwd_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, sz, vp]
     lib.monarch_attn_fwd_ex.restype = i
+    lib.monarch_attn_fwd_bshd.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, sz, vp]
+    lib.monarch_attn_fwd_bshd.restype = i
     lib.monarch_attn_fwd_padded.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, sz, vp]
     lib.monarch_attn_fwd_padded.restype = i
     lib.monarch_attn_fwd_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
@@ -142,6 +144,33 @@ def monarch_attn_fwd_ex(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, wo
     _check(lib.monarch_attn_fwd_ex(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                    batch, heads, N, d, b, T, code, float(softmax_scale), int(path),
                                    workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
+    return Y
+
+
+def monarch_attn_fwd_bshd(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, workspace=None,
+                          Y=None, stream=None):
+    """Forward pass on contiguous CUDA tensors [batch, N, heads, d] (no transpose to
+    [batch, heads, N, d] needed).  path: MA_PATH_AUTO, MA_PATH_TENSOR or MA_PATH_GENERIC."""
+    lib = load_library()
+    if not Q.is_cuda:
+        raise MonarchAttnError(-2, "monarch_attn_fwd_bshd needs CUDA tensors; there is no CPU path")
+    if not (Q.shape == K.shape == V.shape and Q.dim() == 4):
+        raise ValueError("Q, K, V must share the shape [batch, N, heads, d]")
+    if not (Q.is_contiguous() and K.is_contiguous() and V.is_contiguous()):
+        raise ValueError("Q, K, V must be contiguous")
+    batch, N, heads, d = Q.shape
+    code = _TORCH_TO_CODE[Q.dtype]
+    if softmax_scale is None:
+        softmax_scale = 1.0 / math.sqrt(d)
+    if Y is None:
+        Y = torch.empty_like(Q)
+    if workspace is None:
+        need = max(lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_TENSOR),
+                   lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_GENERIC))
+        workspace = torch.zeros(max(int(need), 256), dtype=torch.uint8, device=Q.device)
+    _check(lib.monarch_attn_fwd_bshd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                     batch, N, heads, d, b, T, code, float(softmax_scale), int(path),
+                                     workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
     return Y
 
 

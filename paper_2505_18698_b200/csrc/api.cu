@@ -24,6 +24,7 @@ static inline int esize(int dtype) { return dtype == MA_F32 ? 4 : 2; }
 struct Problem {
   int batch, heads, N, d, b, T, dtype, m, BH;
   int n_valid;   // keys b k + i >= n_valid are masked out (App. C.3); N when there is no padding
+  int H;         // 0: [batch][heads][N][d]; heads: [batch][N][heads][d]
 };
 
 static int validate_shape(int batch, int heads, int N, int d, int b, int T, int dtype, Problem* p) {
@@ -31,7 +32,7 @@ static int validate_shape(int batch, int heads, int N, int d, int b, int T, int 
   if (batch <= 0 || heads <= 0 || N <= 0 || d <= 0 || b <= 0 || T < 1) return MA_ERR_SHAPE;
   if (N % b != 0) return MA_ERR_SHAPE;
   if ((long long)batch * heads > 0x7fffffffLL / 2) return MA_ERR_SHAPE;
-  *p = Problem{batch, heads, N, d, b, T, dtype, N / b, batch * heads, N};
+  *p = Problem{batch, heads, N, d, b, T, dtype, N / b, batch * heads, N, 0};
   return MA_OK;
 }
 
@@ -88,7 +89,7 @@ static int launch_generic_t(const Problem& p, const TIn* Q, const TIn* K, const 
       return MA_ERR_CUDA;                                                                      \
     r_step_kernel<TIn, FIRST, WITHV><<<gr, kThreads, rs, st>>>(Q, K, V, w.aR, w.cR, w.aL,     \
                                                                 w.cL, w.y, p.N, p.d, p.b, p.m, \
-                                                                scale, p.n_valid);             \
+                                                                scale, p.n_valid, p.H);        \
   } while (0)
     if (first && last) MA_LAUNCH_R(true, true);
     else if (first) MA_LAUNCH_R(true, false);
@@ -100,11 +101,11 @@ static int launch_generic_t(const Problem& p, const TIn* Q, const TIn* K, const 
     if (last) {
       if (set_smem((const void*)l_step_kernel<TIn, true>, ls) != cudaSuccess) return MA_ERR_CUDA;
       l_step_kernel<TIn, true><<<gl, kThreads, ls, st>>>(Q, w.aL, w.cL, w.y, w.aR, w.cR, Y, p.N,
-                                                         p.d, p.b, p.m, scale);
+                                                         p.d, p.b, p.m, scale, p.H);
     } else {
       if (set_smem((const void*)l_step_kernel<TIn, false>, ls) != cudaSuccess) return MA_ERR_CUDA;
       l_step_kernel<TIn, false><<<gl, kThreads, ls, st>>>(Q, w.aL, w.cL, w.y, w.aR, w.cR, Y, p.N,
-                                                          p.d, p.b, p.m, scale);
+                                                          p.d, p.b, p.m, scale, p.H);
     }
     ++launches;
   }
@@ -209,7 +210,7 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   else
     rc = tp::launch(Q, K, V, Y, p.BH, p.N, p.b, p.T, p.dtype, scale, ws, st, &launches,
                     resolved == MA_PATH_TENSOR ? 0 : (resolved == MA_PATH_TENSOR_PHASED ? 1 : 2),
-                    ws_armed);
+                    ws_armed, p.H);
   if (rc == MA_OK) g_last_launches = launches;
   return rc;
 }
@@ -271,6 +272,28 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
   p.n_valid = n_valid;
   return fwd_ex(Q, K, V, Y, p, softmax_scale, MA_PATH_GENERIC, workspace, workspace_bytes,
                 (cudaStream_t)stream);
+}
+
+int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, int batch, int N,
+                          int heads, int d, int b, int T, int dtype, float softmax_scale, int path,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+  Problem p;
+  int rc = validate_shape(batch, heads, N, d, b, T, dtype, &p);
+  if (rc != MA_OK) return rc;
+  rc = check_ptrs(Q, K, V, Y, p);
+  if (rc != MA_OK) return rc;
+  if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
+  // the second-generation tensor kernel and the generic kernels read this layout
+  int r = -1;
+  if (path == MA_PATH_AUTO || path == MA_PATH_TENSOR) {
+    const bool keep_fp32_states = p.b == 32 && p.dtype == MA_BF16 && p.T > 2 && path == MA_PATH_AUTO;
+    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) && !keep_fp32_states) r = MA_PATH_TENSOR;
+  }
+  if (r < 0 && (path == MA_PATH_AUTO || path == MA_PATH_GENERIC) && generic_supported(p))
+    r = MA_PATH_GENERIC;
+  if (r < 0) return MA_ERR_UNSUPPORTED;
+  p.H = heads;
+  return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
 int monarch_attn_fwd(const void* Q, const void* K, const void* V, void* Y, int batch, int heads,

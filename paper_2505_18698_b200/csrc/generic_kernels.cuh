@@ -46,13 +46,20 @@ __host__ __device__ inline size_t l_step_smem_floats(int m, int d, bool final_st
 // R half-step for key block k of head h (Eq. 7, 9 -> Eq. 10):
 //   Z_R[j,i] = scale * <aR[k,j,:], K[b k + i,:]> / cR[k,j];  R = softmax_i Z_R
 //   aL[j,k,:] = sum_i R[j,i] K[b k + i,:];  cL[j,k] = sum_i R log R;  (final) y[j,k,:] = sum_i R V
+// Element offset of row n of head h (flat index batch * heads + head) in Q, K, V, Y.
+// H = 0: [batch][heads][N][d].  H = heads > 0: [batch][N][heads][d].
+__device__ __forceinline__ size_t io_off(int h, int n, int N, int d, int H) {
+  if (H == 0) return ((size_t)h * N + n) * d;
+  return (((size_t)(h / H) * N + n) * H + (h % H)) * d;
+}
+
 // FIRST: aR = Q rows b k + j and cR = 1 (L^(0) = identity).
 template <typename TIn, bool FIRST, bool WITH_V>
 __global__ void __launch_bounds__(kThreads)
 r_step_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
               const float* __restrict__ aR, const float* __restrict__ cR,
               float* __restrict__ aL, float* __restrict__ cL, float* __restrict__ y,
-              int N, int d, int b, int m, float scale, int n_valid) {
+              int N, int d, int b, int m, float scale, int n_valid, int H) {
   extern __shared__ float smem[];
   const int k = blockIdx.x, h = blockIdx.y;
   const int dp = d + 1;
@@ -64,19 +71,18 @@ r_step_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
   float* as = zs + b;
 
   const size_t head_off = (size_t)h * N * d;
-  const TIn* Kk = K + head_off + (size_t)k * b * d;
-  const TIn* Vk = V + head_off + (size_t)k * b * d;
   for (int e = threadIdx.x; e < b * d; e += kThreads) {
     int i = e / d, v = e - i * d;
-    Ks[i * dp + v] = ld_as_float(Kk + e);
-    if (WITH_V) Vs[i * dp + v] = ld_as_float(Vk + e);
+    const size_t off = io_off(h, k * b + i, N, d, H) + v;
+    Ks[i * dp + v] = ld_as_float(K + off);
+    if (WITH_V) Vs[i * dp + v] = ld_as_float(V + off);
   }
   __syncthreads();
 
   for (int j = warp; j < b; j += kWarps) {
     float inv_c = 1.f;
     if (FIRST) {
-      const TIn* q = Q + head_off + ((size_t)k * b + j) * d;
+      const TIn* q = Q + io_off(h, k * b + j, N, d, H);
       for (int v = lane; v < d; v += 32) as[v] = ld_as_float(q + v);
     } else {
       const float* a = aR + head_off + ((size_t)k * b + j) * d;
@@ -134,7 +140,7 @@ template <typename TIn, bool FINAL>
 __global__ void __launch_bounds__(kThreads)
 l_step_kernel(const TIn* __restrict__ Q, const float* __restrict__ aL, const float* __restrict__ cL,
               const float* __restrict__ y, float* __restrict__ aR, float* __restrict__ cR,
-              TIn* __restrict__ Y, int N, int d, int b, int m, float scale) {
+              TIn* __restrict__ Y, int N, int d, int b, int m, float scale, int H) {
   extern __shared__ float smem[];
   const int j = blockIdx.x, h = blockIdx.y;
   const int dp = d + 1, mp = m + 1;
@@ -152,7 +158,7 @@ l_step_kernel(const TIn* __restrict__ Q, const float* __restrict__ aL, const flo
   for (int e = threadIdx.x; e < m * d; e += kThreads) {
     int r = e / d, v = e - r * d;
     As[r * dp + v] = aLj[e];
-    Qs[r * dp + v] = ld_as_float(Q + head_off + ((size_t)r * b + j) * d + v);
+    Qs[r * dp + v] = ld_as_float(Q + io_off(h, r * b + j, N, d, H) + v);
     if (FINAL) Xs[r * dp + v] = yj[e];
   }
   for (int k = threadIdx.x; k < m; k += kThreads) cs[k] = cL[(size_t)h * N + (size_t)j * m + k];
@@ -180,7 +186,7 @@ l_step_kernel(const TIn* __restrict__ Q, const float* __restrict__ aL, const flo
     __syncwarp();
     const float inv_s = 1.f / s;
     if (FINAL) {
-      TIn* out = Y + head_off + ((size_t)l * b + j) * d;
+      TIn* out = Y + io_off(h, l * b + j, N, d, H);
       for (int v = lane; v < d; v += 32) {
         float acc = 0.f;
         for (int k = 0; k < m; ++k) acc = fmaf(ps[k], Xs[k * dp + v], acc);

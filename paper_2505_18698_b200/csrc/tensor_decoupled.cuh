@@ -269,11 +269,14 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             float* sC = reinterpret_cast<float*>(smem + Lay::Vec) + eL * 128;
             mbar_expect_tx(&bars->fullE[eE], (HILO && !t.isR) ? 2 * kSlot : kSlot);
             mbar_expect_tx(&bars->fullL[eL], kSlot + (needC ? 512 : 0));
+            // inputs in [batch][N][heads][d]: column offset of the head, row index without it
+            const int xin = P.H ? (t.h % P.H) * kD : 0, hin = P.H ? t.h / P.H : t.h;
             if (t.isR) {
-              const int row0 = (t.h * m + t.idx0) * SB;
+              const int row0 = (t.h * m + t.idx0) * SB, row_in = (hin * m + t.idx0) * SB;
               if (needC) bulk_load_1d(sC, P.cR + row0, 512, &bars->fullL[eL]);
-              tma_load_2d(sE, t.first ? &P.tmQ : &P.tmAR, &bars->fullE[eE], 0, row0);
-              tma_load_2d(sL, &P.tmK, &bars->fullL[eL], 0, row0);
+              if (t.first) tma_load_2d(sE, &P.tmQ, &bars->fullE[eE], xin, row_in);
+              else tma_load_2d(sE, &P.tmAR, &bars->fullE[eE], 0, row0);
+              tma_load_2d(sL, &P.tmK, &bars->fullL[eL], xin, row_in);
             } else {
               const int row0 = (t.h * SB + t.idx0) * m;
               bulk_load_1d(sC, P.cL + row0, 512, &bars->fullL[eL]);
@@ -281,7 +284,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
               if (HILO) tma_load_2d(sE + kSlot, &P.tmALlo, &bars->fullE[eE], 0, row0);
 #pragma unroll
               for (int tt = 0; tt < kBlocks; ++tt)
-                tma_load_3d(sL + tt * (SB * 128), &P.tmQs, &bars->fullL[eL], 0, t.idx0 + tt, t.h * m);
+                tma_load_3d(sL + tt * (SB * 128), &P.tmQs, &bars->fullL[eL], xin, t.idx0 + tt, hin * m);
             }
             stamp(P, nE, 0);
             ++nE;
@@ -305,7 +308,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             asm volatile("fence.proxy.async.global;" ::: "memory");
             uint8_t* sV = smem + Lay::V + eV * kSlot;
             mbar_expect_tx(&bars->fullV[eV], kSlot);
-            if (t.isR) tma_load_2d_hint(sV, &P.tmV, &bars->fullV[eV], 0, (t.h * m + t.idx0) * SB, pol_first);
+            const int xin = P.H ? (t.h % P.H) * kD : 0, hin = P.H ? t.h / P.H : t.h;
+            if (t.isR) tma_load_2d_hint(sV, &P.tmV, &bars->fullV[eV], xin, (hin * m + t.idx0) * SB, pol_first);
             else tma_load_2d(sV, &P.tmY, &bars->fullV[eV], 0, (t.h * SB + t.idx0) * m);
             rV.advance();
             do { ++nVt; itV.next(); } while (nVt < n_total && !needs_v(itV.get()));
@@ -441,7 +445,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
                 tma_store_3d(r == 0 ? &P.tmALs : ((HILO && r == 1) ? &P.tmALlos : &P.tmYs), src, 0,
                              t.idx0 + tt, t.h * SB);
               } else if (t.final_) {
-                tma_store_3d_hint(&P.tmOut, src, 0, t.idx0 + tt, t.h * m, pol_first);
+                tma_store_3d_hint(&P.tmOut, src, P.H ? (t.h % P.H) * kD : 0, t.idx0 + tt,
+                                  (P.H ? t.h / P.H : t.h) * m, pol_first);
               } else {
                 tma_store_3d(&P.tmARs, src, 0, t.idx0 + tt, t.h * m);
               }

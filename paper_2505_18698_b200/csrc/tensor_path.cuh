@@ -855,6 +855,21 @@ inline bool make_map_rows(CUtensorMap* tm, int dtype, void* base, uint64_t rows)
             base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+// Row view of an input / output tensor.  H = 0: [batch*heads*N rows][64] as above, a tile is
+// addressed (0, head * N + n).  H = heads: the tensor is [batch][N][heads][64]; seen as
+// [batch * N rows][heads * 64 columns] a tile of one head is addressed (64 * head, batch * N + n).
+inline bool make_map_rows_io(CUtensorMap* tm, int dtype, void* base, uint64_t rows, int H) {
+  if (H == 0) return make_map_rows(tm, dtype, base, rows);
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)H * kD, rows / H};
+  cuuint64_t strides[1] = {(cuuint64_t)H * kD * 2};
+  cuuint32_t box[2] = {kD, kRows};
+  cuuint32_t es[2] = {1, 1};
+  return fn(tm, dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+            base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 // 3D view (64, inner, outer) of a contiguous [outer][inner][64] array; box = (64, 1, box_outer):
 // box_outer rows that are `inner` rows apart.
 inline bool make_map_strided(CUtensorMap* tm, int dtype, void* base, uint64_t inner, uint64_t outer,
@@ -863,6 +878,23 @@ inline bool make_map_strided(CUtensorMap* tm, int dtype, void* base, uint64_t in
   if (!fn) return false;
   cuuint64_t dims[3] = {kD, inner, outer};
   cuuint64_t strides[2] = {kD * 2, inner * kD * 2};
+  cuuint32_t box[3] = {kD, 1, box_outer};
+  cuuint32_t es[3] = {1, 1, 1};
+  return fn(tm, dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+            base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Strided view of an input / output tensor (rows n = inner_pos + inner * l of one head).
+// H = 0: as make_map_strided, addressed (0, inner_pos, head * m + l).  H = heads: dims
+// (heads * 64, inner, batch * m), addressed (64 * head, inner_pos, batch * m + l).
+inline bool make_map_strided_io(CUtensorMap* tm, int dtype, void* base, uint64_t inner,
+                                uint64_t outer, uint32_t box_outer, int H) {
+  if (H == 0) return make_map_strided(tm, dtype, base, inner, outer, box_outer);
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)H * kD, inner, outer / H};
+  cuuint64_t strides[2] = {(cuuint64_t)H * kD * 2, inner * (cuuint64_t)H * kD * 2};
   cuuint32_t box[3] = {kD, 1, box_outer};
   cuuint32_t es[3] = {1, 1, 1};
   return fn(tm, dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,

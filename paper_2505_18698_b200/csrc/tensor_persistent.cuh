@@ -72,6 +72,7 @@ struct Params {
   int* counters;       // [2T][BH] completed tiles
   long long* trace;    // optional: clock64 stamps [4 CTAs][64 tiles][8 events] (profiling aid)
   int m, BH, T;
+  int H;               // 0: Q, K, V, Y are [batch][heads][N][d]; heads: [batch][N][heads][d]
   int tiles_per_head, tiles_per_phase;
   int g_begin, g_end;  // tile range of this launch
   int check_deps;
@@ -719,21 +720,23 @@ cudaError_t launch_decoupled(const Params& P, int grid, cudaStream_t st);
 template <typename T, int B, int SB>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int T_steps,
                     int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
-                    bool ws_armed) {
+                    bool ws_armed, int H) {
+  if (H != 0 && mode != 0) return 4;   // only the second-generation kernel reads [batch][N][heads][d]
   const Ws w = ws_layout(ws, BH, N);
   int* counters = (int*)((char*)ws + w.bytes);
   const int m = N / SB;            // = SB on this path
   const uint64_t rows = (uint64_t)BH * N;
   void* aLlo = (char*)counters + counters_bytes(BH, T_steps);   // used when uses_hilo(dtype, SB)
   Params P;
-  bool ok = make_map_rows(&P.tmQ, dtype, (void*)Q, rows) && make_map_rows(&P.tmK, dtype, (void*)K, rows) &&
-            make_map_rows(&P.tmV, dtype, (void*)V, rows) && make_map_rows(&P.tmAR, dtype, w.aR, rows) &&
+  bool ok = make_map_rows_io(&P.tmQ, dtype, (void*)Q, rows, H) &&
+            make_map_rows_io(&P.tmK, dtype, (void*)K, rows, H) &&
+            make_map_rows_io(&P.tmV, dtype, (void*)V, rows, H) && make_map_rows(&P.tmAR, dtype, w.aR, rows) &&
             make_map_rows(&P.tmAL, dtype, w.aL, rows) && make_map_rows(&P.tmY, dtype, w.y, rows) &&
             make_map_strided(&P.tmALs, dtype, w.aL, m, (uint64_t)BH * SB, SB) &&
             make_map_strided(&P.tmYs, dtype, w.y, m, (uint64_t)BH * SB, SB) &&
-            make_map_strided(&P.tmQs, dtype, (void*)Q, SB, (uint64_t)BH * m, SB) &&
+            make_map_strided_io(&P.tmQs, dtype, (void*)Q, SB, (uint64_t)BH * m, SB, H) &&
             make_map_strided(&P.tmARs, dtype, w.aR, SB, (uint64_t)BH * m, SB) &&
-            make_map_strided(&P.tmOut, dtype, Y, SB, (uint64_t)BH * m, SB);
+            make_map_strided_io(&P.tmOut, dtype, Y, SB, (uint64_t)BH * m, SB, H);
   if (ok && uses_hilo(dtype, SB))
     ok = make_map_rows(&P.tmALlo, dtype, aLlo, rows) &&
          make_map_strided(&P.tmALlos, dtype, aLlo, m, (uint64_t)BH * SB, SB);
@@ -741,7 +744,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   P.aL = (uint8_t*)w.aL; P.aR = (uint8_t*)w.aR; P.y = (uint8_t*)w.y; P.out = (uint8_t*)Y;
   P.cL = w.cL; P.cR = w.cR; P.status = w.status; P.counters = counters;
   P.trace = trace_buffer();
-  P.m = m; P.BH = BH; P.T = T_steps;
+  P.m = m; P.BH = BH; P.T = T_steps; P.H = H;
   P.tiles_per_head = m / (kRows / SB);
   P.tiles_per_phase = BH * P.tiles_per_head;
   P.scale = scale;
@@ -787,8 +790,8 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
 
 inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int b, int T,
                   int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
-                  bool ws_armed) {
-#define MA_TP_ARGS Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed
+                  bool ws_armed, int H = 0) {
+#define MA_TP_ARGS Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed, H
   if (dtype == 1) {
     if (b == 128) return launch_t<__half, 128, 128>(MA_TP_ARGS);
     if (b == 64) return launch_t<__half, 64, 64>(MA_TP_ARGS);

@@ -337,3 +337,31 @@ def test_padded_entry_point_rejects_more_than_one_block_of_padding():
         with pytest.raises(binding.MonarchAttnError) as e:
             binding.monarch_attn_fwd_padded(Qd, Kd, Vd, 8, 2, bad)
         assert e.value.code == 2      # MA_ERR_SHAPE
+
+
+# ------------------------------------------------------------------ [batch][N][heads][d] layout
+@pytest.mark.parametrize("N,b,d,T,dtype,batch,heads,path", [
+    (4096, 64, 64, 2, "bf16", 2, 3, binding.MA_PATH_TENSOR),
+    (16384, 128, 64, 1, "f16", 1, 2, binding.MA_PATH_TENSOR),
+    (1024, 32, 64, 2, "bf16", 3, 5, binding.MA_PATH_TENSOR),      # hi + lo alpha_L, 64-row tiles
+    (4096, 64, 64, 3, "bf16", 1, 37, binding.MA_PATH_AUTO),       # more heads than fit one wave
+    (256, 16, 64, 1, "f32", 2, 3, binding.MA_PATH_AUTO),          # generic kernels
+    (210, 14, 72, 2, "f16", 2, 5, binding.MA_PATH_GENERIC),       # m != b, d != 64
+])
+def test_batch_seq_head_layout_matches_oracle(N, b, d, T, dtype, batch, heads, path):
+    """Tensors stored [batch, N, heads, d]: same result as the per-head oracle, bit for bit the
+    same as the [batch, heads, N, d] call on transposed copies."""
+    Q, K, V = wl.make_qkv(batch, heads, N, d, dtype, min(16, d), 1.5, seed=N + heads + T)
+    td = binding.torch_dtype(dtype)
+    Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))            # [batch, heads, N, d]
+    Qs, Ks, Vs = (x.transpose(1, 2).contiguous() for x in (Qd, Kd, Vd))      # [batch, N, heads, d]
+    Ys = binding.monarch_attn_fwd_bshd(Qs, Ks, Vs, b, T, path=path)
+    assert Ys.shape == Qs.shape and Ys.dtype == td
+    Y = Ys.transpose(1, 2).float().cpu().numpy().astype(np.float64)
+    ref = mo.monarch_attention(Q, K, V, b, T)
+    assert np.isfinite(Y).all()
+    assert rel_err(Y, ref) <= TOL[dtype]
+    same_path = binding.MA_PATH_AUTO if path == binding.MA_PATH_AUTO else path
+    Y2 = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, b, T, path=same_path)
+    if not (path == binding.MA_PATH_AUTO and N == 256):      # AUTO takes the fused kernel for that shape
+        assert torch.equal(Y2, Ys.transpose(1, 2))
