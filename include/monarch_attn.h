@@ -89,6 +89,20 @@ int monarch_attn_fwd_host(const void* Q_host, const void* K_host, const void* V_
 /* Scratch the no-allocation entry point below carries inside the library image, in bytes. */
 #define MONARCH_ATTN_NOALLOC_SCRATCH_BYTES (8u << 20)
 
+/* Forward pass that also returns the value of the objective it maximises (Sec. 3, Eq. 6:
+ * f(M; Q, K) = <M, scale Q K^T> + H(M); the paper reports it per iteration count as a convergence
+ * diagnostic).  After the final L update, L = softmax_k Z_L exactly and every R[k,j,:] sums to one,
+ * so f at the returned matrix is the sum over rows of log sum_k exp(Z_L[j,k,l]); the final L
+ * half-step has that number for each row anyway and writes it out:
+ *   row_lse: DEVICE pointer, [batch][heads][N] floats (natural logarithm), row b l + j of a head;
+ *   f of a head = sum of its N entries (the caller reduces; 4-byte aligned).
+ * `path`: MA_PATH_AUTO, MA_PATH_TENSOR (second-generation kernel) or MA_PATH_GENERIC.  Y, workspace
+ * and everything else as monarch_attn_fwd_ex.  Asynchronous on `stream`. */
+int monarch_attn_fwd_objective(const void* Q, const void* K, const void* V, void* Y, int batch,
+                               int heads, int N, int d, int b, int T, int dtype,
+                               float softmax_scale, int path, float* row_lse, void* workspace,
+                               size_t workspace_bytes, void* stream);
+
 /* Forward pass on tensors laid out [batch][N][heads][d] (the layout a transformer layer has after
  * its QKV projection, before any transpose); the paper's method is per head (Sec. 3), so only the
  * addressing changes.  Q, K, V, Y: DEVICE pointers to contiguous [batch][N][heads][d] arrays of

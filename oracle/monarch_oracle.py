@@ -247,6 +247,25 @@ def objective_dense(M, Q, K, scale):
     return float((M * S).sum() + _neg_xlogx_sum(M))
 
 
+def final_row_lse(R, Q, K, b, scale):
+    """Row-wise log-sum-exp of the logits of the L update that follows R (Eq. 8 with Eq. 10):
+    lse[b*l + j] = log sum_k exp(Z_L[j,k,l]).  Because that update is the exact maximiser over L
+    (L = softmax_k Z_L, so Z_L - log L is constant in k) and every R[k,j,:] sums to one, the
+    objective of Eq. 6 at (L, R) is the plain sum of these N numbers; the pin is
+    test_objective_equals_sum_of_final_row_lse."""
+    Q = np.asarray(Q, np.float64)
+    K = np.asarray(K, np.float64)
+    Qb, Kb, _ = block_views(Q, K, K, b, scale)
+    m = Q.shape[0] // b
+    logR = np.where(R > 0.0, np.log(np.where(R > 0.0, R, 1.0)), 0.0)
+    aL = np.einsum("kji,kiv->jkv", R, Kb)
+    cL = np.einsum("kji->jk", np.where(R > 0.0, R * logR, 0.0))
+    ZL = np.einsum("jkv,jlv->jkl", aL, Qb) - cL[:, :, None]
+    zmax = ZL.max(axis=1)
+    lse = zmax + np.log(np.exp(ZL - zmax[:, None, :]).sum(axis=1))          # [j, l]
+    return lse.T.reshape(m * b)                                            # row b*l + j
+
+
 def objective_factored(L, R, Q, K, scale):
     """Sec. 3 'Softmax Objective': sum over (j,k) of
     <Qb_j^T L_jk, Kb_k^T R_kj> + (1^T R_kj) H(L_jk) + (1^T L_jk) H(R_kj)."""

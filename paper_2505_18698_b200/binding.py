@@ -56,6 +56,8 @@ def load_library(path: str = LIB_PATH):
     lib.monarch_attn_workspace_bytes.restype = sz
     lib.monarch_attn_fwd_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, sz, vp]
     lib.monarch_attn_fwd_ex.restype = i
+    lib.monarch_attn_fwd_objective.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, vp, sz, vp]
+    lib.monarch_attn_fwd_objective.restype = i
     lib.monarch_attn_fwd_bshd.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, sz, vp]
     lib.monarch_attn_fwd_bshd.restype = i
     lib.monarch_attn_fwd_padded.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, sz, vp]
@@ -145,6 +147,31 @@ def monarch_attn_fwd_ex(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, wo
                                    batch, heads, N, d, b, T, code, float(softmax_scale), int(path),
                                    workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
     return Y
+
+
+def monarch_attn_fwd_objective(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, workspace=None,
+                               Y=None, stream=None):
+    """Forward pass plus the objective value: returns (Y, row_lse) with row_lse a float32 CUDA
+    tensor [batch, heads, N]; row_lse.sum(-1) is f(M^(T)) of Eq. 6 per head."""
+    lib = load_library()
+    if not Q.is_cuda:
+        raise MonarchAttnError(-2, "monarch_attn_fwd_objective needs CUDA tensors; there is no CPU path")
+    batch, heads, N, d = _shape_of(Q, K, V)
+    code = _TORCH_TO_CODE[Q.dtype]
+    if softmax_scale is None:
+        softmax_scale = 1.0 / math.sqrt(d)
+    if Y is None:
+        Y = torch.empty_like(Q)
+    lse = torch.empty((batch, heads, N), dtype=torch.float32, device=Q.device)
+    if workspace is None:
+        need = max(lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_TENSOR),
+                   lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_GENERIC))
+        workspace = torch.zeros(max(int(need), 256), dtype=torch.uint8, device=Q.device)
+    _check(lib.monarch_attn_fwd_objective(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                          batch, heads, N, d, b, T, code, float(softmax_scale),
+                                          int(path), lse.data_ptr(), workspace.data_ptr(),
+                                          workspace.numel(), _stream_ptr(stream)))
+    return Y, lse
 
 
 def monarch_attn_fwd_bshd(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, workspace=None,

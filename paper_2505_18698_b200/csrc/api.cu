@@ -25,6 +25,7 @@ struct Problem {
   int batch, heads, N, d, b, T, dtype, m, BH;
   int n_valid;   // keys b k + i >= n_valid are masked out (App. C.3); N when there is no padding
   int H;         // 0: [batch][heads][N][d]; heads: [batch][N][heads][d]
+  float* lse;    // optional output [batch*heads][N]: row log-sum-exp of the final L half-step
 };
 
 static int validate_shape(int batch, int heads, int N, int d, int b, int T, int dtype, Problem* p) {
@@ -32,7 +33,7 @@ static int validate_shape(int batch, int heads, int N, int d, int b, int T, int 
   if (batch <= 0 || heads <= 0 || N <= 0 || d <= 0 || b <= 0 || T < 1) return MA_ERR_SHAPE;
   if (N % b != 0) return MA_ERR_SHAPE;
   if ((long long)batch * heads > 0x7fffffffLL / 2) return MA_ERR_SHAPE;
-  *p = Problem{batch, heads, N, d, b, T, dtype, N / b, batch * heads, N, 0};
+  *p = Problem{batch, heads, N, d, b, T, dtype, N / b, batch * heads, N, 0, nullptr};
   return MA_OK;
 }
 
@@ -101,11 +102,11 @@ static int launch_generic_t(const Problem& p, const TIn* Q, const TIn* K, const 
     if (last) {
       if (set_smem((const void*)l_step_kernel<TIn, true>, ls) != cudaSuccess) return MA_ERR_CUDA;
       l_step_kernel<TIn, true><<<gl, kThreads, ls, st>>>(Q, w.aL, w.cL, w.y, w.aR, w.cR, Y, p.N,
-                                                         p.d, p.b, p.m, scale, p.H);
+                                                         p.d, p.b, p.m, scale, p.H, p.lse);
     } else {
       if (set_smem((const void*)l_step_kernel<TIn, false>, ls) != cudaSuccess) return MA_ERR_CUDA;
       l_step_kernel<TIn, false><<<gl, kThreads, ls, st>>>(Q, w.aL, w.cL, w.y, w.aR, w.cR, Y, p.N,
-                                                          p.d, p.b, p.m, scale, p.H);
+                                                          p.d, p.b, p.m, scale, p.H, nullptr);
     }
     ++launches;
   }
@@ -210,7 +211,7 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   else
     rc = tp::launch(Q, K, V, Y, p.BH, p.N, p.b, p.T, p.dtype, scale, ws, st, &launches,
                     resolved == MA_PATH_TENSOR ? 0 : (resolved == MA_PATH_TENSOR_PHASED ? 1 : 2),
-                    ws_armed, p.H);
+                    ws_armed, p.H, p.lse);
   if (rc == MA_OK) g_last_launches = launches;
   return rc;
 }
@@ -272,6 +273,30 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
   p.n_valid = n_valid;
   return fwd_ex(Q, K, V, Y, p, softmax_scale, MA_PATH_GENERIC, workspace, workspace_bytes,
                 (cudaStream_t)stream);
+}
+
+int monarch_attn_fwd_objective(const void* Q, const void* K, const void* V, void* Y, int batch,
+                               int heads, int N, int d, int b, int T, int dtype,
+                               float softmax_scale, int path, float* row_lse, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+  Problem p;
+  int rc = validate_shape(batch, heads, N, d, b, T, dtype, &p);
+  if (rc != MA_OK) return rc;
+  rc = check_ptrs(Q, K, V, Y, p);
+  if (rc != MA_OK) return rc;
+  if (!row_lse) return MA_ERR_NULL;
+  if (((uintptr_t)row_lse & 3) != 0) return MA_ERR_ALIGN;
+  if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
+  int r = -1;
+  if ((path == MA_PATH_AUTO || path == MA_PATH_TENSOR) &&
+      tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) &&
+      !(path == MA_PATH_AUTO && p.b == 32 && p.dtype == MA_BF16 && p.T > 2))
+    r = MA_PATH_TENSOR;
+  if (r < 0 && (path == MA_PATH_AUTO || path == MA_PATH_GENERIC) && generic_supported(p))
+    r = MA_PATH_GENERIC;
+  if (r < 0) return MA_ERR_UNSUPPORTED;
+  p.lse = row_lse;
+  return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
 int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, int batch, int N,

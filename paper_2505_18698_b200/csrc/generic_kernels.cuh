@@ -140,7 +140,8 @@ template <typename TIn, bool FINAL>
 __global__ void __launch_bounds__(kThreads)
 l_step_kernel(const TIn* __restrict__ Q, const float* __restrict__ aL, const float* __restrict__ cL,
               const float* __restrict__ y, float* __restrict__ aR, float* __restrict__ cR,
-              TIn* __restrict__ Y, int N, int d, int b, int m, float scale, int H) {
+              TIn* __restrict__ Y, int N, int d, int b, int m, float scale, int H,
+              float* __restrict__ row_lse) {
   extern __shared__ float smem[];
   const int j = blockIdx.x, h = blockIdx.y;
   const int dp = d + 1, mp = m + 1;
@@ -186,6 +187,8 @@ l_step_kernel(const TIn* __restrict__ Q, const float* __restrict__ aL, const flo
     __syncwarp();
     const float inv_s = 1.f / s;
     if (FINAL) {
+      // log-sum-exp of row b l + j: summed over a head's rows it is the objective (Eq. 6)
+      if (row_lse != nullptr && lane == 0) row_lse[(size_t)h * N + (size_t)l * b + j] = zmax + logf(s);
       TIn* out = Y + io_off(h, l * b + j, N, d, H);
       for (int v = lane; v < d; v += 32) {
         float acc = 0.f;

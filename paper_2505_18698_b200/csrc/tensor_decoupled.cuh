@@ -645,6 +645,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         }
         sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
         inv_s = 1.f / sum;
+        // Row b l + j (l = rb, j = idx0 + blk) of the final L half-step: its log-sum-exp; summed over
+        // the rows of a head it is the value of the objective (Eq. 6) at the returned matrix.
+        if (t.final_ && P.lse != nullptr)
+          P.lse[(size_t)t.h * (SB * m) + (size_t)rb * SB + t.idx0 + blk] = (mx + fast_log2(sum)) * kLn2;
         if (!t.final_) {
           // MMA 2 of this half-step contracts over rows: P must be normalised before it is read.
           // The thread re-reads its own row, rescales in fp32, writes it back.

@@ -67,7 +67,8 @@ struct Params {
   float* cL;
   float* cR;
   uint8_t *aL, *aR, *y;  // state arrays (for L2 discards once a tile has been consumed)
-  uint8_t* out;         // Y (the second-generation kernel stores rows with plain stores)
+  uint8_t* out;         // Y
+  float* lse;           // optional [BH][N]: log-sum-exp of each row of the final L half-step
   int* status;
   int* counters;       // [2T][BH] completed tiles
   long long* trace;    // optional: clock64 stamps [4 CTAs][64 tiles][8 events] (profiling aid)
@@ -720,8 +721,8 @@ cudaError_t launch_decoupled(const Params& P, int grid, cudaStream_t st);
 template <typename T, int B, int SB>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int T_steps,
                     int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
-                    bool ws_armed, int H) {
-  if (H != 0 && mode != 0) return 4;   // only the second-generation kernel reads [batch][N][heads][d]
+                    bool ws_armed, int H, float* lse) {
+  if ((H != 0 || lse != nullptr) && mode != 0) return 4;   // second-generation kernel only   // only the second-generation kernel reads [batch][N][heads][d]
   const Ws w = ws_layout(ws, BH, N);
   int* counters = (int*)((char*)ws + w.bytes);
   const int m = N / SB;            // = SB on this path
@@ -744,7 +745,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   P.aL = (uint8_t*)w.aL; P.aR = (uint8_t*)w.aR; P.y = (uint8_t*)w.y; P.out = (uint8_t*)Y;
   P.cL = w.cL; P.cR = w.cR; P.status = w.status; P.counters = counters;
   P.trace = trace_buffer();
-  P.m = m; P.BH = BH; P.T = T_steps; P.H = H;
+  P.m = m; P.BH = BH; P.T = T_steps; P.H = H; P.lse = lse;
   P.tiles_per_head = m / (kRows / SB);
   P.tiles_per_phase = BH * P.tiles_per_head;
   P.scale = scale;
@@ -790,8 +791,8 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
 
 inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int b, int T,
                   int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
-                  bool ws_armed, int H = 0) {
-#define MA_TP_ARGS Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed, H
+                  bool ws_armed, int H = 0, float* lse = nullptr) {
+#define MA_TP_ARGS Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed, H, lse
   if (dtype == 1) {
     if (b == 128) return launch_t<__half, 128, 128>(MA_TP_ARGS);
     if (b == 64) return launch_t<__half, 64, 64>(MA_TP_ARGS);

@@ -365,3 +365,33 @@ def test_batch_seq_head_layout_matches_oracle(N, b, d, T, dtype, batch, heads, p
     Y2 = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, b, T, path=same_path)
     if not (path == binding.MA_PATH_AUTO and N == 256):      # AUTO takes the fused kernel for that shape
         assert torch.equal(Y2, Ys.transpose(1, 2))
+
+
+# ------------------------------------------------------------------ objective value (Eq. 6)
+@pytest.mark.parametrize("N,b,d,dtype,path,tol", [
+    (256, 16, 64, "f32", binding.MA_PATH_GENERIC, 1e-5),
+    (210, 14, 40, "f32", binding.MA_PATH_GENERIC, 1e-5),
+    (4096, 64, 64, "bf16", binding.MA_PATH_TENSOR, 2e-3),
+    (16384, 128, 64, "f16", binding.MA_PATH_TENSOR, 2e-3),
+    (1024, 32, 64, "bf16", binding.MA_PATH_TENSOR, 2e-3),
+])
+def test_objective_value_matches_oracle_and_ascends(N, b, d, dtype, path, tol):
+    """row_lse summed over a head is f(M^(T)) of Eq. 6 at the returned matrix (oracle: the dense
+    definition for small N, the factored form otherwise), and f does not decrease with T."""
+    Q, K, V = wl.make_qkv(1, 2, N, d, dtype, min(8, d), 1.0, seed=N + b)
+    Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))
+    scale = 1.0 / np.sqrt(d)
+    prev = None
+    for T in (1, 2, 3):
+        Y, lse = binding.monarch_attn_fwd_objective(Qd, Kd, Vd, b, T, path=path)
+        f_gpu = lse.double().sum(-1).cpu().numpy()[0]
+        Y2 = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, b, T, path=path)
+        assert torch.equal(Y, Y2)                          # the extra output changes nothing else
+        for h in range(2):
+            _, L, R = mo.monarch_attention_head(Q[0, h], K[0, h], V[0, h], b, T, return_factors=True)
+            f_ref = (mo.objective_dense(mo.dense_monarch(L, R), Q[0, h], K[0, h], scale) if N <= 256
+                     else mo.objective_factored(L, R, Q[0, h], K[0, h], scale))
+            assert abs(f_gpu[h] - f_ref) <= tol * abs(f_ref), (T, h, f_gpu[h], f_ref)
+        if prev is not None:
+            assert np.all(f_gpu >= prev - tol * np.abs(prev))
+        prev = f_gpu

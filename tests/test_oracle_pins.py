@@ -266,3 +266,17 @@ def test_argument_errors():
         mo.monarch_attention_head(Q, K, V, b=4, T=0)
     with pytest.raises(ValueError):
         mo.monarch_attention_head(Q, K, V, b=5, T=1)
+
+
+@pytest.mark.parametrize("N,b,T", [(12, 4, 1), (16, 4, 2), (24, 6, 3), (20, 2, 2), (18, 9, 2)])
+def test_objective_equals_sum_of_final_row_lse(N, b, T):
+    """After the final L update the objective of Eq. 6 at the returned (L, R) is the sum over rows
+    of the log-sum-exp of that update's logits (the quantity the GPU path can emit for free)."""
+    rng = np.random.default_rng(N * 31 + b + T)
+    Q, K, V = (rng.standard_normal((N, 5)) * 1.3 for _ in range(3))
+    scale = 0.37
+    _, L, R = mo.monarch_attention_head(Q, K, V, b, T, scale=scale, return_factors=True)
+    f_dense = mo.objective_dense(mo.dense_monarch(L, R), Q, K, scale)
+    lse = mo.final_row_lse(R, Q, K, b, scale)
+    assert lse.shape == (N,)
+    assert abs(lse.sum() - f_dense) < 1e-9 * max(1.0, abs(f_dense))
