@@ -395,3 +395,28 @@ def test_objective_value_matches_oracle_and_ascends(N, b, d, dtype, path, tol):
         if prev is not None:
             assert np.all(f_gpu >= prev - tol * np.abs(prev))
         prev = f_gpu
+
+
+# ------------------------------------------------------------------ the shapes of the paper's experiments
+@pytest.mark.parametrize("n_valid,b,d,T,dtype", [
+    (197, 14, 64, 3, "f16"),       # ViT-B: N = 197 -> 210, m = 15 (Sec. 5, App. D)
+    (384, 24, 64, 1, "f16"), (384, 48, 64, 1, "f16"), (384, 96, 64, 1, "bf16"), (384, 128, 64, 1, "f32"),  # RoBERTa
+    (2048, 32, 64, 1, "bf16"), (8192, 64, 64, 1, "bf16"),     # BART: (b, m) = (32, 64), (64, 128)
+    (256, 16, 72, 3, "f16"),       # DiT-XL: d = 72
+    (7600, 128, 48, 2, "f32"),     # GPS graph transformer: N = 7600 -> 7680, d = 48
+])
+def test_shapes_of_the_papers_experiments(n_valid, b, d, T, dtype):
+    """Sequence length, block size, head width and step count of each experiment in the paper
+    (synthetic values: the models and datasets are not here), through the public entry points."""
+    N = -(-n_valid // b) * b
+    Q, K, V = wl.make_qkv(1, 2, N, d, dtype, min(8, d), 1.0, seed=n_valid + b)
+    Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))
+    if N != n_valid:
+        Y = binding.monarch_attn_fwd_padded(Qd, Kd, Vd, b, T, n_valid)
+        ref = mo.monarch_attention(Q, K, V, b, T, n_valid=n_valid)
+    else:
+        Y = binding.monarch_attn_fwd(Qd, Kd, Vd, b, T)
+        ref = mo.monarch_attention(Q, K, V, b, T)
+    Y = Y.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(Y[:, :, :n_valid]).all()
+    assert rel_err(Y[:, :, :n_valid], ref[:, :, :n_valid]) <= TOL[dtype]
