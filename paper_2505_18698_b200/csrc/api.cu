@@ -154,6 +154,18 @@ static int resolve_path(const Problem& p, int path) {
   return -1;
 }
 
+// Path choice of the entry points that only the second-generation tensor kernel and the generic
+// kernels serve (other layout, extra outputs): AUTO, TENSOR or GENERIC; -1 if none applies.
+static int resolve_tensor_or_generic(const Problem& p, int path) {
+  if (path == MA_PATH_AUTO || path == MA_PATH_TENSOR) {
+    const int r = resolve_path(p, path);
+    if (r == MA_PATH_TENSOR) return r;
+    if (path == MA_PATH_TENSOR) return -1;
+  }
+  if ((path == MA_PATH_AUTO || path == MA_PATH_GENERIC) && generic_supported(p)) return MA_PATH_GENERIC;
+  return -1;
+}
+
 static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
   if (resolved == MA_PATH_FUSED) return kStatusBytes;   // no states leave the chip
@@ -287,13 +299,7 @@ int monarch_attn_fwd_objective(const void* Q, const void* K, const void* V, void
   if (!row_lse) return MA_ERR_NULL;
   if (((uintptr_t)row_lse & 3) != 0) return MA_ERR_ALIGN;
   if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
-  int r = -1;
-  if ((path == MA_PATH_AUTO || path == MA_PATH_TENSOR) &&
-      tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) &&
-      !(path == MA_PATH_AUTO && p.b == 32 && p.dtype == MA_BF16 && p.T > 2))
-    r = MA_PATH_TENSOR;
-  if (r < 0 && (path == MA_PATH_AUTO || path == MA_PATH_GENERIC) && generic_supported(p))
-    r = MA_PATH_GENERIC;
+  const int r = resolve_tensor_or_generic(p, path);
   if (r < 0) return MA_ERR_UNSUPPORTED;
   p.lse = row_lse;
   return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);
@@ -308,14 +314,7 @@ int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, 
   rc = check_ptrs(Q, K, V, Y, p);
   if (rc != MA_OK) return rc;
   if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
-  // the second-generation tensor kernel and the generic kernels read this layout
-  int r = -1;
-  if (path == MA_PATH_AUTO || path == MA_PATH_TENSOR) {
-    const bool keep_fp32_states = p.b == 32 && p.dtype == MA_BF16 && p.T > 2 && path == MA_PATH_AUTO;
-    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) && !keep_fp32_states) r = MA_PATH_TENSOR;
-  }
-  if (r < 0 && (path == MA_PATH_AUTO || path == MA_PATH_GENERIC) && generic_supported(p))
-    r = MA_PATH_GENERIC;
+  const int r = resolve_tensor_or_generic(p, path);
   if (r < 0) return MA_ERR_UNSUPPORTED;
   p.H = heads;
   return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);
