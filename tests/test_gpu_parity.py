@@ -420,3 +420,19 @@ def test_shapes_of_the_papers_experiments(n_valid, b, d, T, dtype):
     Y = Y.float().cpu().numpy().astype(np.float64)
     assert np.isfinite(Y[:, :, :n_valid]).all()
     assert rel_err(Y[:, :, :n_valid], ref[:, :, :n_valid]) <= TOL[dtype]
+
+
+# ------------------------------------------------------------------ determinism
+@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5"])
+def test_results_are_bit_identical_from_call_to_call(name):
+    """No arithmetic depends on scheduling (the dependency counters only order tiles), so repeated
+    calls must agree bit for bit; a missing fence or a reused buffer shows up here as a mismatch."""
+    w = wl.WORKLOADS[name]
+    Q, K, V = wl.make_qkv(2, 3, w.N, w.d, w.dtype, w.rank, w.s, seed=900 + w.seed)
+    Qd, Kd, Vd = (binding.to_device(x, w.dtype) for x in (Q, K, V))
+    Y0 = binding.monarch_attn_fwd(Qd, Kd, Vd, w.b, w.T).clone()
+    Y = torch.empty_like(Y0)
+    for _ in range(60):
+        binding.monarch_attn_fwd(Qd, Kd, Vd, w.b, w.T, Y=Y)
+        assert torch.equal(Y, Y0)
+    assert binding.monarch_attn_device_status() == 0
