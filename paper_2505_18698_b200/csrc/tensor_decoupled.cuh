@@ -171,7 +171,11 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Ba
   }
 }
 
-template <typename T, int B, int SB>
+// EXTRA: the rarely used hooks (inputs laid out [batch][N][heads][d], row log-sum-exp output) are
+// compiled into a second instantiation: in the plain one they cost 4 % even when switched off (the
+// producer's instruction stream is on the critical path and the compiler predicates the head
+// index division instead of branching around it).
+template <typename T, int B, int SB, bool EXTRA>
 __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_constant__ Params P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -270,7 +274,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             mbar_expect_tx(&bars->fullE[eE], (HILO && !t.isR) ? 2 * kSlot : kSlot);
             mbar_expect_tx(&bars->fullL[eL], kSlot + (needC ? 512 : 0));
             // inputs in [batch][N][heads][d]: column offset of the head, row index without it
-            const int xin = P.H ? (t.h % P.H) * kD : 0, hin = P.H ? t.h / P.H : t.h;
+            const int xin = (EXTRA && P.H) ? (t.h % P.H) * kD : 0, hin = (EXTRA && P.H) ? t.h / P.H : t.h;
             if (t.isR) {
               const int row0 = (t.h * m + t.idx0) * SB, row_in = (hin * m + t.idx0) * SB;
               if (needC) bulk_load_1d(sC, P.cR + row0, 512, &bars->fullL[eL]);
@@ -308,7 +312,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             asm volatile("fence.proxy.async.global;" ::: "memory");
             uint8_t* sV = smem + Lay::V + eV * kSlot;
             mbar_expect_tx(&bars->fullV[eV], kSlot);
-            const int xin = P.H ? (t.h % P.H) * kD : 0, hin = P.H ? t.h / P.H : t.h;
+            const int xin = (EXTRA && P.H) ? (t.h % P.H) * kD : 0, hin = (EXTRA && P.H) ? t.h / P.H : t.h;
             if (t.isR) tma_load_2d_hint(sV, &P.tmV, &bars->fullV[eV], xin, (hin * m + t.idx0) * SB, pol_first);
             else tma_load_2d(sV, &P.tmY, &bars->fullV[eV], 0, (t.h * SB + t.idx0) * m);
             rV.advance();
@@ -445,8 +449,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
                 tma_store_3d(r == 0 ? &P.tmALs : ((HILO && r == 1) ? &P.tmALlos : &P.tmYs), src, 0,
                              t.idx0 + tt, t.h * SB);
               } else if (t.final_) {
-                tma_store_3d_hint(&P.tmOut, src, P.H ? (t.h % P.H) * kD : 0, t.idx0 + tt,
-                                  (P.H ? t.h / P.H : t.h) * m, pol_first);
+                tma_store_3d_hint(&P.tmOut, src, (EXTRA && P.H) ? (t.h % P.H) * kD : 0, t.idx0 + tt,
+                                  ((EXTRA && P.H) ? t.h / P.H : t.h) * m, pol_first);
               } else {
                 tma_store_3d(&P.tmARs, src, 0, t.idx0 + tt, t.h * m);
               }
@@ -647,7 +651,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         inv_s = 1.f / sum;
         // Row b l + j (l = rb, j = idx0 + blk) of the final L half-step: its log-sum-exp; summed over
         // the rows of a head it is the value of the objective (Eq. 6) at the returned matrix.
-        if (t.final_ && P.lse != nullptr)
+        if (EXTRA && t.final_ && P.lse != nullptr)
           P.lse[(size_t)t.h * (SB * m) + (size_t)rb * SB + t.idx0 + blk] = (mx + fast_log2(sum)) * kLn2;
         if (!t.final_) {
           // MMA 2 of this half-step contracts over rows: P must be normalised before it is read.
@@ -752,14 +756,19 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
   }
 }
 
-template <typename T, int B, int SB>
-inline cudaError_t launch_kernel(const Params& P, int grid, cudaStream_t st) {
-  const void* fn = (const void*)monarch_decoupled<T, B, SB>;
+template <typename T, int B, int SB, bool EXTRA>
+inline cudaError_t launch_kernel_x(const Params& P, int grid, cudaStream_t st) {
+  const void* fn = (const void*)monarch_decoupled<T, B, SB, EXTRA>;
   constexpr int kSmem = Lay<B, std::is_same<T, __nv_bfloat16>::value && SB == 32>::kSmem;
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
   if (e != cudaSuccess) return e;
-  monarch_decoupled<T, B, SB><<<grid, kThreads, kSmem, st>>>(P);
+  monarch_decoupled<T, B, SB, EXTRA><<<grid, kThreads, kSmem, st>>>(P);
   return cudaGetLastError();
+}
+template <typename T, int B, int SB>
+inline cudaError_t launch_kernel(const Params& P, int grid, cudaStream_t st) {
+  if (P.H != 0 || P.lse != nullptr) return launch_kernel_x<T, B, SB, true>(P, grid, st);
+  return launch_kernel_x<T, B, SB, false>(P, grid, st);
 }
 
 }  // namespace tp2
