@@ -171,7 +171,8 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Ba
   }
 }
 
-// EXTRA: the rarely used hooks (inputs laid out [batch][N][heads][d], row log-sum-exp output) are
+// EXTRA: the rarely used hooks (inputs laid out [batch][N][heads][d], row log-sum-exp output, time
+// stamps for the trace buffer) are
 // compiled into a second instantiation: in the plain one they cost 4 % even when switched off (the
 // producer's instruction stream is on the critical path and the compiler predicates the head
 // index division instead of branching around it).
@@ -290,7 +291,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
               for (int tt = 0; tt < kBlocks; ++tt)
                 tma_load_3d(sL + tt * (SB * 128), &P.tmQs, &bars->fullL[eL], xin, t.idx0 + tt, hin * m);
             }
-            stamp(P, nE, 0);
+            if (EXTRA) stamp(P, nE, 0);
             ++nE;
             rE.advance();
             rL.advance();
@@ -381,7 +382,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             if (needV) { umma_commit(&bars->emptyV[eV]); rV.advance(); }
             umma_commit(&bars->p_free[c]);
             umma_commit(&bars->o_ready[o2]);
-            stamp(P, i2, 4);
+            if (EXTRA) stamp(P, i2, 4);
             ++i2;
             it2.next();
             r2L.advance();
@@ -401,7 +402,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
           if (HILO && !t.isR) issue_scores<B, FT, FT, true>(tmem + s1 * B, sL, sE + kSlot);
           umma_commit(&bars->emptyE[eE]);
           umma_commit(&bars->s_ready[s1]);
-          stamp(P, i1, 1);
+          if (EXTRA) stamp(P, i1, 1);
           ++i1;
           it1.next();
           r1E.advance();
@@ -463,7 +464,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
           asm volatile("fence.proxy.async.global;" ::: "memory");
           __threadfence();
           atomicAdd(P.counters + t.p * P.BH + t.h, 1);
-          stamp(P, n, 7);
+          if (EXTRA) stamp(P, n, 7);
           round += nr;
         }
       }
@@ -490,7 +491,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       const uint32_t tS = tmem + s * B + ((uint32_t)(sub * 32) << 16);
       wait_or_abort(&bars->s_ready[s], (n / kStagesS) & 1, bars, P.status, 30);
       tc_fence_after();
-      if (stamper) stamp(P, n, 2);
+      if (EXTRA && stamper) stamp(P, n, 2);
       // the state tile MMA 1 consumed is read exactly once: drop its lines from L2
       if (t.isR) {
         if (!t.first) discard_line(P.aR + ((size_t)(t.h * m + t.idx0) * SB + t_row) * 128);
@@ -676,7 +677,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       fence_proxy_async();
       tc_fence_before();
       mbar_arrive(&bars->p_ready[c]);
-      if (stamper) stamp(P, n, 3);
+      if (EXTRA && stamper) stamp(P, n, 3);
     }
   } else {
     // ------------------------------------------------------------------ epilogue group: O -> rows
@@ -697,7 +698,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       const uint32_t tO = tO0 + o * 128;
       wait_or_abort(&bars->o_ready[o], (n / kStagesO) & 1, bars, P.status, 31);
       tc_fence_after();
-      if (stamper) stamp(P, n, 5);
+      if (EXTRA && stamper) stamp(P, n, 5);
       const float inv_s = stat[(n & 3) * 128 + t_row];
       if (t.final_) discard_line(P.y + ((size_t)(t.h * SB + t.idx0) * m + t_row) * 128);
       const int nr = rounds_of(t);
@@ -734,7 +735,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         mbar_arrive(&bars->stage_ready[n & 1]);
       }
       if (!scaled) P.cR[((size_t)t.h * m + rb) * SB + t.idx0 + blk] = c1;
-      if (stamper) stamp(P, n, 6);
+      if (EXTRA && stamper) stamp(P, n, 6);
       round += nr;
     }
   }
@@ -767,7 +768,8 @@ inline cudaError_t launch_kernel_x(const Params& P, int grid, cudaStream_t st) {
 }
 template <typename T, int B, int SB>
 inline cudaError_t launch_kernel(const Params& P, int grid, cudaStream_t st) {
-  if (P.H != 0 || P.lse != nullptr) return launch_kernel_x<T, B, SB, true>(P, grid, st);
+  if (P.H != 0 || P.lse != nullptr || P.trace != nullptr)
+    return launch_kernel_x<T, B, SB, true>(P, grid, st);
   return launch_kernel_x<T, B, SB, false>(P, grid, st);
 }
 
