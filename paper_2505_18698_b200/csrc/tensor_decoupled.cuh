@@ -272,21 +272,22 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             uint8_t* sL = smem + Lay::L + eL * kSlot;
             const bool needC = !t.first;
             float* sC = reinterpret_cast<float*>(smem + Lay::Vec) + eL * 128;
-            mbar_expect_tx(&bars->fullE[eE], (HILO && !t.isR) ? 2 * kSlot : kSlot);
-            mbar_expect_tx(&bars->fullL[eL], kSlot + (needC ? 512 : 0));
+            // one "operands landed" barrier per tile (indexed like the L ring) for E, L and c
+            mbar_expect_tx(&bars->fullL[eL],
+                           ((HILO && !t.isR) ? 3 * kSlot : 2 * kSlot) + (needC ? 512 : 0));
             // inputs in [batch][N][heads][d]: column offset of the head, row index without it
             const int xin = (EXTRA && P.H) ? (t.h % P.H) * kD : 0, hin = (EXTRA && P.H) ? t.h / P.H : t.h;
             if (t.isR) {
               const int row0 = (t.h * m + t.idx0) * SB, row_in = (hin * m + t.idx0) * SB;
               if (needC) bulk_load_1d(sC, P.cR + row0, 512, &bars->fullL[eL]);
-              if (t.first) tma_load_2d(sE, &P.tmQ, &bars->fullE[eE], xin, row_in);
-              else tma_load_2d(sE, &P.tmAR, &bars->fullE[eE], 0, row0);
+              if (t.first) tma_load_2d(sE, &P.tmQ, &bars->fullL[eL], xin, row_in);
+              else tma_load_2d(sE, &P.tmAR, &bars->fullL[eL], 0, row0);
               tma_load_2d(sL, &P.tmK, &bars->fullL[eL], xin, row_in);
             } else {
               const int row0 = (t.h * SB + t.idx0) * m;
               bulk_load_1d(sC, P.cL + row0, 512, &bars->fullL[eL]);
-              tma_load_2d(sE, &P.tmAL, &bars->fullE[eE], 0, row0);
-              if (HILO) tma_load_2d(sE + kSlot, &P.tmALlo, &bars->fullE[eE], 0, row0);
+              tma_load_2d(sE, &P.tmAL, &bars->fullL[eL], 0, row0);
+              if (HILO) tma_load_2d(sE + kSlot, &P.tmALlo, &bars->fullL[eL], 0, row0);
 #pragma unroll
               for (int tt = 0; tt < kBlocks; ++tt)
                 tma_load_3d(sL + tt * (SB * 128), &P.tmQs, &bars->fullL[eL], xin, t.idx0 + tt, hin * m);
@@ -356,7 +357,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       RingPos<kStagesO> r2O;
       RingPos<2> r2P;                             // P buffer of tile i2 is i2 & 1; parity of i2 >> 1
       uint32_t p_par = 0;
-      const uint32_t bFullE = smem_u32(&bars->fullE[0]), bFullL = smem_u32(&bars->fullL[0]);
+      const uint32_t bFullL = smem_u32(&bars->fullL[0]);
       const uint32_t bFullV = smem_u32(&bars->fullV[0]), bPReady = smem_u32(&bars->p_ready[0]);
       const uint32_t bOFree = smem_u32(&bars->o_free[0]);
       while (i2 < n_total) {
@@ -365,7 +366,6 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         const uint32_t r_ready = mbar_poll_addr(bPReady + c * 8, p_par);
         const uint32_t r_of = mbar_poll_addr(bOFree + r2O.slot * 8, r2O.par ^ 1);
         const uint32_t r_v = mbar_poll_addr(bFullV + rV.slot * 8, rV.par);
-        const uint32_t r_e = mbar_poll_addr(bFullE + r1E.slot * 8, r1E.par);
         const uint32_t r_l = mbar_poll_addr(bFullL + r1L.slot * 8, r1L.par);
         if (i2 < i1 && (force || (r_ready & r_of))) {
           const Tile t = it2.get();
@@ -392,7 +392,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             did = true;
           }
         }
-        if (i1 < n_total && i1 < i2 + kStagesS && (force || (r_e & r_l))) {
+        if (i1 < n_total && i1 < i2 + kStagesS && (force || r_l)) {
           const Tile t = it1.get();
           const int eE = r1E.slot, eL1 = r1L.slot, s1 = r1S.slot;
           tc_fence_after();
