@@ -288,9 +288,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
               bulk_load_1d(sC, P.cL + row0, 512, &bars->fullL[eL]);
               tma_load_2d(sE, &P.tmAL, &bars->fullL[eL], 0, row0);
               if (HILO) tma_load_2d(sE + kSlot, &P.tmALlo, &bars->fullL[eL], 0, row0);
-#pragma unroll
-              for (int tt = 0; tt < kBlocks; ++tt)
-                tma_load_3d(sL + tt * (SB * 128), &P.tmQs, &bars->fullL[eL], xin, t.idx0 + tt, hin * m);
+              // one box: kBlocks blocks (positions j) of SB rows (l) each, block after block
+              tma_load_3d(sL, &P.tmQs, &bars->fullL[eL], xin, hin * m, t.idx0);
             }
             if (EXTRA) stamp(P, nE, 0);
             ++nE;
@@ -443,18 +442,15 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         if ((n & 1) == w) {
           for (int r = 0; r < nr; ++r) {
             wait_or_abort(&bars->stage_ready[w], (round + r) & 1, bars, P.status, 40);
-#pragma unroll
-            for (int tt = 0; tt < kBlocks; ++tt) {
-              const uint8_t* src = sStage + tt * (SB * 128);
-              if (t.isR) {
-                tma_store_3d(r == 0 ? &P.tmALs : ((HILO && r == 1) ? &P.tmALlos : &P.tmYs), src, 0,
-                             t.idx0 + tt, t.h * SB);
-              } else if (t.final_) {
-                tma_store_3d_hint(&P.tmOut, src, (EXTRA && P.H) ? (t.h % P.H) * kD : 0, t.idx0 + tt,
-                                  ((EXTRA && P.H) ? t.h / P.H : t.h) * m, pol_first);
-              } else {
-                tma_store_3d(&P.tmARs, src, 0, t.idx0 + tt, t.h * m);
-              }
+            // one box per round: the tile's kBlocks blocks of SB rows (blocked views)
+            if (t.isR) {
+              tma_store_3d(r == 0 ? &P.tmALs : ((HILO && r == 1) ? &P.tmALlos : &P.tmYs), sStage, 0,
+                           t.h * SB, t.idx0);
+            } else if (t.final_) {
+              tma_store_3d_hint(&P.tmOut, sStage, (EXTRA && P.H) ? (t.h % P.H) * kD : 0,
+                                ((EXTRA && P.H) ? t.h / P.H : t.h) * m, t.idx0, pol_first);
+            } else {
+              tma_store_3d(&P.tmARs, sStage, 0, t.h * m, t.idx0);
             }
             tma_store_commit();
             tma_store_wait_read();

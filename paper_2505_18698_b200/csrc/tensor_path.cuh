@@ -902,6 +902,24 @@ inline bool make_map_strided_io(CUtensorMap* tm, int dtype, void* base, uint64_t
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same strided view with the two outer dimensions swapped, (64, outer, inner), so that ONE box
+// (64, box_outer, box_inner) brings box_inner blocks of box_outer rows each, block after block in
+// shared memory: what the per-block boxes of make_map_strided_io need box_inner copies for.
+// Addressed (64 * head or 0, outer index, inner index).
+inline bool make_map_blocked_io(CUtensorMap* tm, int dtype, void* base, uint64_t inner,
+                                uint64_t outer, uint32_t box_outer, uint32_t box_inner, int H) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t pitch = (cuuint64_t)(H ? H : 1) * kD * 2;      // bytes between consecutive rows
+  cuuint64_t dims[3] = {(cuuint64_t)(H ? H : 1) * kD, H ? outer / H : outer, inner};
+  cuuint64_t strides[2] = {inner * pitch, pitch};
+  cuuint32_t box[3] = {kD, box_outer, box_inner};
+  cuuint32_t es[3] = {1, 1, 1};
+  return fn(tm, dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+            base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <typename T, int B>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int T_steps,
                     int dtype, float scale, const Ws& w, cudaStream_t st, int* launches) {

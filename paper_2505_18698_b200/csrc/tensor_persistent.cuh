@@ -733,14 +733,24 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
             make_map_rows_io(&P.tmK, dtype, (void*)K, rows, H) &&
             make_map_rows_io(&P.tmV, dtype, (void*)V, rows, H) && make_map_rows(&P.tmAR, dtype, w.aR, rows) &&
             make_map_rows(&P.tmAL, dtype, w.aL, rows) && make_map_rows(&P.tmY, dtype, w.y, rows) &&
-            make_map_strided(&P.tmALs, dtype, w.aL, m, (uint64_t)BH * SB, SB) &&
-            make_map_strided(&P.tmYs, dtype, w.y, m, (uint64_t)BH * SB, SB) &&
-            make_map_strided_io(&P.tmQs, dtype, (void*)Q, SB, (uint64_t)BH * m, SB, H) &&
-            make_map_strided(&P.tmARs, dtype, w.aR, SB, (uint64_t)BH * m, SB) &&
-            make_map_strided_io(&P.tmOut, dtype, Y, SB, (uint64_t)BH * m, SB, H);
-  if (ok && uses_hilo(dtype, SB))
-    ok = make_map_rows(&P.tmALlo, dtype, aLlo, rows) &&
-         make_map_strided(&P.tmALlos, dtype, aLlo, m, (uint64_t)BH * SB, SB);
+            true;
+  constexpr uint32_t kBlk = kRows / SB;     // blocks per tile
+  if (ok && mode == 0) {   // second-generation kernel: one box per tile (blocked views)
+    ok = make_map_blocked_io(&P.tmALs, dtype, w.aL, m, (uint64_t)BH * SB, SB, kBlk, 0) &&
+         make_map_blocked_io(&P.tmYs, dtype, w.y, m, (uint64_t)BH * SB, SB, kBlk, 0) &&
+         make_map_blocked_io(&P.tmQs, dtype, (void*)Q, SB, (uint64_t)BH * m, SB, kBlk, H) &&
+         make_map_blocked_io(&P.tmARs, dtype, w.aR, SB, (uint64_t)BH * m, SB, kBlk, 0) &&
+         make_map_blocked_io(&P.tmOut, dtype, Y, SB, (uint64_t)BH * m, SB, kBlk, H);
+    if (ok && uses_hilo(dtype, SB))
+      ok = make_map_rows(&P.tmALlo, dtype, aLlo, rows) &&
+           make_map_blocked_io(&P.tmALlos, dtype, aLlo, m, (uint64_t)BH * SB, SB, kBlk, 0);
+  } else if (ok) {         // first-generation kernel: one box per block
+    ok = make_map_strided(&P.tmALs, dtype, w.aL, m, (uint64_t)BH * SB, SB) &&
+         make_map_strided(&P.tmYs, dtype, w.y, m, (uint64_t)BH * SB, SB) &&
+         make_map_strided(&P.tmQs, dtype, (void*)Q, SB, (uint64_t)BH * m, SB) &&
+         make_map_strided(&P.tmARs, dtype, w.aR, SB, (uint64_t)BH * m, SB) &&
+         make_map_strided(&P.tmOut, dtype, Y, SB, (uint64_t)BH * m, SB);
+  }
   if (!ok) return 7;
   P.aL = (uint8_t*)w.aL; P.aR = (uint8_t*)w.aR; P.y = (uint8_t*)w.y; P.out = (uint8_t*)Y;
   P.cL = w.cL; P.cR = w.cR; P.status = w.status; P.counters = counters;
