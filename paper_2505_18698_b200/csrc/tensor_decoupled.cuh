@@ -597,6 +597,57 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         // Z_L = scale * S' - c_L (Eq. 8), softmax over k = along the row
         f = P.scale * kLog2e;
         const float2 f2 = make_float2(f, f);
+        if constexpr (SB == B) {
+          // Pass 1 forms the logits z = f s + c, takes their maximum and writes them back over s in
+          // TMEM, so that pass 2 is the same loop as in the R half-step (no second read of the
+          // c-vector, no second multiply-add); 16-column chunks, next load in flight.
+          constexpr int NC16 = B / 16;
+          float* b0 = buf;
+          float* b1 = buf + 16;
+          tmem_ld16(tS, b0);
+#pragma unroll
+          for (int cc = 0; cc < NC16; ++cc) {
+            float* cur = (cc & 1) ? b1 : b0;
+            float* nxt = (cc & 1) ? b0 : b1;
+            tmem_ld_wait();
+            if (cc + 1 < NC16) tmem_ld16(tS + 16 * (cc + 1), nxt);
+            const float4* cv4 = reinterpret_cast<const float4*>(cvt + 16 * cc);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float4 k4 = cv4[i];
+              const float2 za = ffma2(make_float2(cur[4 * i], cur[4 * i + 1]), f2, make_float2(k4.x, k4.y));
+              const float2 zb = ffma2(make_float2(cur[4 * i + 2], cur[4 * i + 3]), f2, make_float2(k4.z, k4.w));
+              m4[0] = max3(m4[0], za.x, za.y);
+              m4[1] = max3(m4[1], zb.x, zb.y);
+              cur[4 * i] = za.x;
+              cur[4 * i + 1] = za.y;
+              cur[4 * i + 2] = zb.x;
+              cur[4 * i + 3] = zb.y;
+            }
+            tmem_st16(tS + 16 * cc, cur);
+          }
+          tmem_st_wait();                        // the logits are in TMEM before they are read back
+          mx = fmaxf(m4[0], m4[1]);
+          const float2 nmx2 = make_float2(-mx, -mx);
+          wait_or_abort(&bars->p_free[c], (q & 1) ^ 1, bars, P.status, 33);
+          tmem_ld16(tS, b0);
+#pragma unroll
+          for (int cc = 0; cc < NC16; ++cc) {
+            float* cur = (cc & 1) ? b1 : b0;
+            float* nxt = (cc & 1) ? b0 : b1;
+            tmem_ld_wait();
+            if (cc + 1 < NC16) tmem_ld16(tS + 16 * (cc + 1), nxt);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float2 zz = fadd2(make_float2(cur[2 * i], cur[2 * i + 1]), nmx2);
+              const float2 pp = exp2_pair(zz, i);
+              a2[i & 1] = fadd2(a2[i & 1], pp);
+              cur[2 * i] = pp.x;
+              cur[2 * i + 1] = pp.y;
+            }
+            store_row16<T>(sP, srow, 16 * cc, cur);
+          }
+        } else {
 #pragma unroll
         for (int cc = 0; cc < NC; ++cc) {
           if (!mine(cc)) continue;
@@ -643,6 +694,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             for (int i = 0; i < 32; ++i) sv[i] = 0.f;
           }
           store_row32<T>(sP, srow, 32 * cc, sv);
+        }
         }
         sum = (a2[0].x + a2[0].y) + (a2[1].x + a2[1].y);
         inv_s = 1.f / sum;
