@@ -629,7 +629,9 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
           tmem_st_wait();                        // the logits are in TMEM before they are read back
           mx = fmaxf(m4[0], m4[1]);
           const float2 nmx2 = make_float2(-mx, -mx);
-          wait_or_abort(&bars->p_free[c], (q & 1) ^ 1, bars, P.status, 33);
+          // final: the weights go to the P buffer as they are formed (normalised in the epilogue);
+          // non-final: they go back to TMEM and a third pass writes them normalised
+          if (t.final_) wait_or_abort(&bars->p_free[c], (q & 1) ^ 1, bars, P.status, 33);
           tmem_ld16(tS, b0);
 #pragma unroll
           for (int cc = 0; cc < NC16; ++cc) {
@@ -645,7 +647,31 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
               cur[2 * i] = pp.x;
               cur[2 * i + 1] = pp.y;
             }
-            store_row16<T>(sP, srow, 16 * cc, cur);
+            if (t.final_) store_row16<T>(sP, srow, 16 * cc, cur);
+            else tmem_st16(tS + 16 * cc, cur);
+          }
+          if (!t.final_) {
+            // MMA 2 of this half-step contracts over rows, so P must be normalised before it is
+            // read: third pass, fp32 weights from TMEM times 1 / sum, one rounding to 16 bits.
+            tmem_st_wait();
+            const float is_ = 1.f / ((a2[0].x + a2[0].y) + (a2[1].x + a2[1].y));
+            const float2 is2 = make_float2(is_, is_);
+            wait_or_abort(&bars->p_free[c], (q & 1) ^ 1, bars, P.status, 33);
+            tmem_ld16(tS, b0);
+#pragma unroll
+            for (int cc = 0; cc < NC16; ++cc) {
+              float* cur = (cc & 1) ? b1 : b0;
+              float* nxt = (cc & 1) ? b0 : b1;
+              tmem_ld_wait();
+              if (cc + 1 < NC16) tmem_ld16(tS + 16 * (cc + 1), nxt);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float2 v = fmul2(make_float2(cur[2 * i], cur[2 * i + 1]), is2);
+                cur[2 * i] = v.x;
+                cur[2 * i + 1] = v.y;
+              }
+              store_row16<T>(sP, srow, 16 * cc, cur);
+            }
           }
         } else {
 #pragma unroll
@@ -702,7 +728,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         // the rows of a head it is the value of the objective (Eq. 6) at the returned matrix.
         if (EXTRA && t.final_ && P.lse != nullptr)
           P.lse[(size_t)t.h * (SB * m) + (size_t)rb * SB + t.idx0 + blk] = (mx + fast_log2(sum)) * kLn2;
-        if (!t.final_) {
+        if (!t.final_ && SB != B) {
           // MMA 2 of this half-step contracts over rows: P must be normalised before it is read.
           // The thread re-reads its own row, rescales in fp32, writes it back.
           const float2 is2 = make_float2(inv_s, inv_s);
