@@ -210,7 +210,7 @@ def time_e2e(w, steps, warmup, torch, binding, dist=None):
 
 # DRAM bytes of ONE launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
 # ncu; see the summaries under profiles/ named for each kernel and workload).
-NCU_TRAFFIC_BYTES = {"C5": 183.9e6 + 31.3e6, "C4": 176.1e6 + 22.1e6, "C3": 132.7e6 + 43.3e6, "C2": 75.6e6 + 4.4e6}
+NCU_TRAFFIC_BYTES = {"C5": 185.5e6 + 31.7e6, "C4": 174.9e6 + 20.7e6, "C3": 132.7e6 + 42.5e6, "C2": 75.6e6 + 4.4e6}
 
 
 def roofline(w, ms, peaks, which):
