@@ -53,8 +53,11 @@ typedef enum {
                                 m = b in {64, 128} */
   MA_PATH_TENSOR_CHAINED = 6, /* first-generation persistent kernel (each softmax warpgroup also
                                  does its tile's epilogue), one launch; kept for comparison */
-  MA_PATH_FUSED = 5    /* one CTA per (batch, head), everything in shared memory, one launch:
+  MA_PATH_FUSED = 5,   /* one CTA per (batch, head), everything in shared memory, one launch:
                           f16/bf16, N = 256, m = b = 16, d = 64 */
+  MA_PATH_FUSED_SMALL = 7 /* the same idea for any block shape: f16/bf16, m and b <= 32 (m need not
+                             equal b), d <= 64 a multiple of 8, N <= 580 for T = 1 and <= 440 for
+                             T > 1 (the states of a head must fit shared memory); f16 arithmetic */
 } ma_path;
 
 /* T-step MonarchAttention forward (Eq. 7-10 then Eq. 4) with scale = 1/sqrt(d).
@@ -107,8 +110,8 @@ int monarch_attn_fwd_objective(const void* Q, const void* K, const void* V, void
  * its QKV projection, before any transpose); the paper's method is per head (Sec. 3), so only the
  * addressing changes.  Q, K, V, Y: DEVICE pointers to contiguous [batch][N][heads][d] arrays of
  * `dtype`, 16-byte aligned, Y not overlapping an input.  `path`: MA_PATH_AUTO, MA_PATH_TENSOR (the
- * second-generation kernel: the head becomes a column offset in the TMA tensor maps) or
- * MA_PATH_GENERIC; other paths give MA_ERR_UNSUPPORTED.  Workspace as for monarch_attn_fwd_ex with
+ * second-generation kernel: the head becomes a column offset in the TMA tensor maps),
+ * MA_PATH_FUSED_SMALL or MA_PATH_GENERIC; other paths give MA_ERR_UNSUPPORTED.  Workspace as for monarch_attn_fwd_ex with
  * the same path (monarch_attn_workspace_bytes does not depend on the layout).  Everything else as
  * monarch_attn_fwd_ex.  Asynchronous on `stream`. */
 int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, int batch, int N,
@@ -127,8 +130,9 @@ int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, 
  * Q, K, V, Y: DEVICE pointers, [batch][heads][N][d], same rules as monarch_attn_fwd_ex.
  * n_valid must satisfy N - b < n_valid <= N (less than one block of padding, so that every key
  * block keeps a valid key; anything else is MA_ERR_SHAPE).  n_valid == N is the unpadded pass.
- * Runs on the generic kernels (any dtype, m need not equal b); workspace as for
- * monarch_attn_fwd_ex with path MA_PATH_GENERIC.  Asynchronous on `stream`. */
+ * Runs on the general fused kernel (MA_PATH_FUSED_SMALL) where that supports the shape and dtype,
+ * else on the generic kernels (any dtype, m need not equal b); a workspace sized for
+ * monarch_attn_fwd_ex with path MA_PATH_GENERIC serves both.  Asynchronous on `stream`. */
 int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y, int batch,
                             int heads, int N, int d, int b, int T, int dtype, float softmax_scale,
                             int n_valid, void* workspace, size_t workspace_bytes, void* stream);

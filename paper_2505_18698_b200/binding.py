@@ -21,6 +21,7 @@ MA_F32, MA_F16, MA_BF16 = 0, 1, 2
 MA_PATH_AUTO, MA_PATH_GENERIC, MA_PATH_TENSOR, MA_PATH_TENSOR_PHASED, MA_PATH_TENSOR_BASIC = 0, 1, 2, 3, 4
 MA_PATH_FUSED = 5
 MA_PATH_TENSOR_CHAINED = 6
+MA_PATH_FUSED_SMALL = 7
 MA_OK = 0
 
 _TORCH_TO_CODE = {torch.float32: MA_F32, torch.float16: MA_F16, torch.bfloat16: MA_BF16}
@@ -177,7 +178,7 @@ def monarch_attn_fwd_objective(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_A
 def monarch_attn_fwd_bshd(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, workspace=None,
                           Y=None, stream=None):
     """Forward pass on contiguous CUDA tensors [batch, N, heads, d] (no transpose to
-    [batch, heads, N, d] needed).  path: MA_PATH_AUTO, MA_PATH_TENSOR or MA_PATH_GENERIC."""
+    [batch, heads, N, d] needed).  path: MA_PATH_AUTO, MA_PATH_TENSOR, MA_PATH_FUSED_SMALL or MA_PATH_GENERIC."""
     lib = load_library()
     if not Q.is_cuda:
         raise MonarchAttnError(-2, "monarch_attn_fwd_bshd needs CUDA tensors; there is no CPU path")

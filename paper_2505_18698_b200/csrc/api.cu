@@ -13,6 +13,7 @@
 #include "tensor_persistent.cuh"
 #include "tensor_decoupled.cuh"
 #include "fused_n256.cuh"
+#include "fused_small.cuh"
 
 namespace ma {
 
@@ -142,10 +143,13 @@ static int resolve_path(const Problem& p, int path) {
     if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) &&
         !(p.b == 32 && p.dtype == MA_BF16 && p.T > 2))
       return MA_PATH_TENSOR;
+    if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
     if (generic_supported(p)) return MA_PATH_GENERIC;
     return -1;
   }
   if (path == MA_PATH_GENERIC) return generic_supported(p) ? path : -1;
+  if (path == MA_PATH_FUSED_SMALL)
+    return fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T) ? path : -1;
   if (path == MA_PATH_FUSED) return fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
   if (path == MA_PATH_TENSOR || path == MA_PATH_TENSOR_PHASED || path == MA_PATH_TENSOR_CHAINED)
     return tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
@@ -154,13 +158,21 @@ static int resolve_path(const Problem& p, int path) {
   return -1;
 }
 
-// Path choice of the entry points that only the second-generation tensor kernel and the generic
-// kernels serve (other layout, extra outputs): AUTO, TENSOR or GENERIC; -1 if none applies.
-static int resolve_tensor_or_generic(const Problem& p, int path) {
+// Path choice of the entry points that only the second-generation tensor kernel, the general fused
+// kernel (layout and padding, no extra outputs: `with_fused_small`) and the generic kernels serve:
+// AUTO, TENSOR, FUSED_SMALL or GENERIC; -1 if none applies.
+static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused_small = false) {
   if (path == MA_PATH_AUTO || path == MA_PATH_TENSOR) {
     const int r = resolve_path(p, path);
     if (r == MA_PATH_TENSOR) return r;
     if (path == MA_PATH_TENSOR) return -1;
+  }
+  if (with_fused_small && (path == MA_PATH_AUTO || path == MA_PATH_FUSED_SMALL)) {
+    const bool ok = fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T);
+    // AUTO keeps the N = 256 special case's shapes on the kernels they have always used
+    if (ok && (path == MA_PATH_FUSED_SMALL || !fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)))
+      return MA_PATH_FUSED_SMALL;
+    if (path == MA_PATH_FUSED_SMALL) return -1;
   }
   if ((path == MA_PATH_AUTO || path == MA_PATH_GENERIC) && generic_supported(p)) return MA_PATH_GENERIC;
   return -1;
@@ -168,7 +180,7 @@ static int resolve_tensor_or_generic(const Problem& p, int path) {
 
 static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
-  if (resolved == MA_PATH_FUSED) return kStatusBytes;   // no states leave the chip
+  if (resolved == MA_PATH_FUSED || resolved == MA_PATH_FUSED_SMALL) return kStatusBytes;   // no states leave the chip
   if (resolved == MA_PATH_TENSOR_BASIC) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
   if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_PHASED ||
       resolved == MA_PATH_TENSOR_CHAINED)
@@ -213,6 +225,11 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   if (resolved == MA_PATH_GENERIC) return launch_generic(p, Q, K, V, Y, scale, ws, st);
   if (resolved == MA_PATH_FUSED) {
     int rc = fused::launch(Q, K, V, Y, p.BH, p.T, p.dtype, scale, st);
+    if (rc == MA_OK) g_last_launches = 1;
+    return rc;
+  }
+  if (resolved == MA_PATH_FUSED_SMALL) {
+    int rc = fsmall::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.m, p.T, p.dtype, scale, p.n_valid, p.H, st);
     if (rc == MA_OK) g_last_launches = 1;
     return rc;
   }
@@ -281,10 +298,12 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
   rc = check_ptrs(Q, K, V, Y, p);
   if (rc != MA_OK) return rc;
   if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
-  if (!generic_supported(p)) return MA_ERR_UNSUPPORTED;
+  const int r = fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)
+                    ? MA_PATH_FUSED_SMALL
+                    : (generic_supported(p) ? MA_PATH_GENERIC : -1);
+  if (r < 0) return MA_ERR_UNSUPPORTED;
   p.n_valid = n_valid;
-  return fwd_ex(Q, K, V, Y, p, softmax_scale, MA_PATH_GENERIC, workspace, workspace_bytes,
-                (cudaStream_t)stream);
+  return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
 int monarch_attn_fwd_objective(const void* Q, const void* K, const void* V, void* Y, int batch,
@@ -314,7 +333,7 @@ int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, 
   rc = check_ptrs(Q, K, V, Y, p);
   if (rc != MA_OK) return rc;
   if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
-  const int r = resolve_tensor_or_generic(p, path);
+  const int r = resolve_tensor_or_generic(p, path, true);
   if (r < 0) return MA_ERR_UNSUPPORTED;
   p.H = heads;
   return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);

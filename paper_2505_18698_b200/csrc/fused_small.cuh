@@ -1,0 +1,502 @@
+// Fused per-head kernel for short sequences of any block shape: N = m*b with m, b <= 32,
+// d <= 64 (a multiple of 8), f16/bf16, optional key padding mask (App. C.3) and either layout.
+//
+// One CTA (8 warps) per (batch, head), one launch for all T rounds.  Q, K, V are read from HBM
+// once, the states alpha_L, alpha_R, y, c_L (Sec. 3 'Implementation') never leave shared memory,
+// Y is written once.  It covers the shapes whose blocks do not fill a 64-row tensor-core tile and
+// are not the 16 x 16 special case of the N = 256 kernel: e.g. N = 210 as 15 blocks of 14 with 197
+// valid keys, or N = 384 as 16 blocks of 24.
+//
+// Layout.  Every tile (Q, K, V and the states) is stored with the SAME row order, row = k*b + i
+// for block k and in-block position i, 128 bytes per row (d padded with zeros to 64).  The
+// permutation between the two half-steps (Eq. 9, 10) is therefore only a choice of operand rows:
+// an R half-step reads the b consecutive rows of block k, an L half-step reads the m rows (l, j)
+// that sit b rows apart.  16-byte chunks are XOR-swizzled with (i & 7) ^ (k & 7), which makes
+// 8-row fragment loads conflict-free in both directions.  A warp owns block k (R) or position j
+// (L) entirely, so inside a half-step no two warps touch the same rows and the outputs can take
+// the place of dead inputs: on the last round alpha_L goes over K, y over V, Y over Q.
+//
+// Contractions are warp-level mma.sync m16n8k16 in f16 (bf16 inputs are converted on the way in,
+// as in the N = 256 kernel).  Blocks are padded to 16 or 32 rows/columns in registers only:
+// operand rows past the block are clamped to its last row (finite values), score columns past the
+// block or past n_valid get -inf, weight rows past the block are zeroed before a transposed
+// product, and output rows past the block are not stored.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fused_n256.cuh"
+
+namespace ma {
+namespace fsmall {
+
+using fused::Mma;
+using fused::col_sum;
+using fused::ex2;
+using fused::kLn2;
+using fused::kLog2e;
+using fused::ldsm_x2_trans;
+using fused::ldsm_x4;
+using fused::ldsm_x4_trans;
+using fused::lg2;
+using fused::movm_trans;
+using fused::quad_max;
+using fused::quad_sum;
+
+constexpr int kThreads = 256, kWarps = 8, kRowBytes = 128, kMaxSmem = 227 * 1024;
+
+// Byte offset of element (block k, position i, column col) in a tile.
+__device__ __forceinline__ uint32_t at(int k, int i, int b, int col) {
+  const int chunk = (col >> 3) ^ (i & 7) ^ (k & 7);
+  return (uint32_t)((k * b + i) * kRowBytes + (chunk << 4) + ((col & 7) << 1));
+}
+
+// Element offset of row n of head h in Q, K, V, Y (H = 0: [batch][heads][N][d]; else
+// [batch][N][H][d]).
+__device__ __forceinline__ size_t row_off(int h, int n, int N, int d, int H) {
+  if (H == 0) return ((size_t)h * N + n) * d;
+  return (((size_t)(h / H) * N + n) * H + (h % H)) * d;
+}
+
+inline size_t smem_bytes(int N, int T) {
+  return (size_t)(T == 1 ? 3 : 4) * N * kRowBytes + (size_t)N * 4 + 1024;
+}
+
+// BP, MP: b and m rounded up to 16 or 32.
+template <typename TIn, int BP, int MP>
+__global__ void __launch_bounds__(kThreads, (BP == 16 && MP == 16) ? 2 : 1)
+monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
+                    TIn* __restrict__ Y, int N, int d, int b, int m, int T_steps, float scale,
+                    int n_valid, int H) {
+  typedef __half T;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int tile = N * kRowBytes;
+  uint8_t* sQ = smem;
+  uint8_t* sK = sQ + tile;
+  uint8_t* sV = sK + tile;                         // V, loaded when the last round starts ...
+  uint8_t* sALx = sV;                              // ... alpha_L of the earlier rounds until then
+  uint8_t* sARx = sV + tile;                       // T > 1 only
+  float* sCL = reinterpret_cast<float*>(smem + (T_steps == 1 ? 3 : 4) * (size_t)tile);   // [k*b + j]
+  const uint32_t sQ_u = (uint32_t)__cvta_generic_to_shared(sQ);
+  const uint32_t sK_u = sQ_u + tile, sV_u = sK_u + tile;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int h_idx = blockIdx.x;
+  // Contractions over d always run over the 64 padded columns (zeros beyond d: the inputs are
+  // zero-filled on the way in and the states are products with them), so every loop unrolls.
+  constexpr int ksteps = 4;
+
+  // ---- load Q, K (and V when there is one round): 16-byte chunks; columns d..63 are zero
+  auto load_tile = [&](const TIn* __restrict__ src, int a) {
+    uint8_t* dst = smem + (size_t)a * tile;
+    for (int idx = tid; idx < N * 8; idx += kThreads) {
+      const int row = idx >> 3, ch = idx & 7;
+      const int k = row / b, i = row - k * b;
+      const uint32_t off = at(k, i, b, ch * 8);
+      if (ch * 8 < d) {
+        const TIn* gp = src + row_off(h_idx, row, N, d, H) + ch * 8;
+        if (Mma<TIn>::is_f16) {
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sQ_u + a * tile + off), "l"(gp));
+        } else {
+          *reinterpret_cast<uint4*>(dst + off) =
+              fused::to_f16x8(__ldg(reinterpret_cast<const uint4*>(gp)), gp);
+        }
+      } else {
+        *reinterpret_cast<uint4*>(dst + off) = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+  };
+  load_tile(Q, 0);
+  load_tile(K, 1);
+  if (T_steps == 1) load_tile(V, 2);
+  asm volatile("cp.async.commit_group;");
+  asm volatile("cp.async.wait_group 0;");
+  __syncthreads();
+
+  const float fl = scale * kLog2e;
+  for (int step = 1; step <= T_steps; ++step) {
+    const bool first = step == 1, last = step == T_steps;
+    if (last && !first) {   // alpha_L of the round before is dead: V takes its buffer
+      load_tile(V, 2);
+      asm volatile("cp.async.commit_group;");
+      asm volatile("cp.async.wait_group 0;");
+      __syncthreads();
+    }
+    // ================================================================ R half-step (Eq. 7, 9, 10)
+    // tile k: Z_R[j,i] = fl * <alpha_R(k,j), K(k,i)>, softmax over i, alpha_L(k,j) = sum_i R K(k,i)
+    {
+      const uint32_t sA_u = first ? sQ_u : (uint32_t)__cvta_generic_to_shared(sARx);
+      uint8_t* dstL = last ? sK : sALx;
+      for (int k = warp; k < m; k += kWarps) {
+        uint32_t outL[BP / 16][8][2], outY[BP / 16][8][2];
+#pragma unroll
+        for (int rt = 0; rt < BP / 16; ++rt) {
+          const int j0 = 16 * rt;
+          if (j0 >= b) continue;
+          float s[BP / 8][4];
+#pragma unroll
+          for (int nt = 0; nt < BP / 8; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
+          const int ja = min(j0 + (lane & 7) + ((lane >> 3) & 1) * 8, b - 1);
+#pragma unroll
+          for (int ks = 0; ks < ksteps; ++ks) {
+            uint32_t a[4];
+            ldsm_x4(a, sA_u + at(k, ja, b, 16 * ks + (lane >> 4) * 8));
+#pragma unroll
+            for (int cp = 0; cp < BP / 16; ++cp) {
+              uint32_t bf[4];
+              const int ib = min(16 * cp + (lane & 7) + (lane >> 4) * 8, b - 1);
+              ldsm_x4(bf, sK_u + at(k, ib, b, 16 * ks + ((lane >> 3) & 1) * 8));
+              Mma<T>::run(s[2 * cp], a, bf);
+              Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+            }
+          }
+          // rows j = j0 + g (c0, c1) and j0 + g + 8 (c2, c3); columns i = 8 nt + 2t, +1
+          float inv_s[2];
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            const int j = j0 + g + 8 * hh;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < BP / 8; ++nt)
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const int i = 8 * nt + 2 * t + e;
+                const bool valid = i < b && k * b + i < n_valid;
+                const float z = valid ? s[nt][2 * hh + e] * fl : -INFINITY;
+                s[nt][2 * hh + e] = z;
+                mx = fmaxf(mx, z);
+              }
+            mx = quad_max(mx);
+            float sum = 0.f, sz = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < BP / 8; ++nt)
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const float z = s[nt][2 * hh + e];
+                const float p = ex2(z - mx);                 // 0 for masked columns
+                s[nt][2 * hh + e] = p;
+                sum += p;
+                if (z > -INFINITY) sz = fmaf(p, z, sz);      // 0 log 0 = 0
+              }
+            sum = quad_sum(sum);
+            sz = quad_sum(sz);
+            inv_s[hh] = 1.f / sum;
+            // c_L = sum R log R (natural log): ln2 * (sum p z / sum - max - log2 sum)
+            if (t == 0 && j < b) sCL[k * b + j] = kLn2 * (sz * inv_s[hh] - mx - lg2(sum));
+          }
+          uint32_t pa[BP / 16][4];
+#pragma unroll
+          for (int kk = 0; kk < BP / 16; ++kk) {
+            pa[kk][0] = Mma<T>::pack(s[2 * kk][0], s[2 * kk][1]);
+            pa[kk][1] = Mma<T>::pack(s[2 * kk][2], s[2 * kk][3]);
+            pa[kk][2] = Mma<T>::pack(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+            pa[kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+          }
+#pragma unroll
+          for (int np = 0; np < 4; ++np) {     // two 8-column tiles of v per transposing ldmatrix
+            if (np >= ksteps) {
+              outL[rt][2 * np][0] = outL[rt][2 * np][1] = 0u;
+              outL[rt][2 * np + 1][0] = outL[rt][2 * np + 1][1] = 0u;
+              outY[rt][2 * np][0] = outY[rt][2 * np][1] = 0u;
+              outY[rt][2 * np + 1][0] = outY[rt][2 * np + 1][1] = 0u;
+              continue;
+            }
+            float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            float y[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+            for (int kk = 0; kk < BP / 16; ++kk) {
+              uint32_t bf[4];
+              const int ib = min(16 * kk + (lane & 15), b - 1);
+              ldsm_x4_trans(bf, sK_u + at(k, ib, b, 16 * np + (lane >> 4) * 8));
+              Mma<T>::run(o[0], pa[kk], bf);
+              Mma<T>::run(o[1], pa[kk], bf + 2);
+              if (last) {
+                ldsm_x4_trans(bf, sV_u + at(k, ib, b, 16 * np + (lane >> 4) * 8));
+                Mma<T>::run(y[0], pa[kk], bf);
+                Mma<T>::run(y[1], pa[kk], bf + 2);
+              }
+            }
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              outL[rt][2 * np + q][0] = Mma<T>::pack(o[q][0] * inv_s[0], o[q][1] * inv_s[0]);
+              outL[rt][2 * np + q][1] = Mma<T>::pack(o[q][2] * inv_s[1], o[q][3] * inv_s[1]);
+              outY[rt][2 * np + q][0] = Mma<T>::pack(y[q][0] * inv_s[0], y[q][1] * inv_s[0]);
+              outY[rt][2 * np + q][1] = Mma<T>::pack(y[q][2] * inv_s[1], y[q][3] * inv_s[1]);
+            }
+          }
+        }
+        // this warp alone reads block k of K and V: on the last round the results take their place
+        __syncwarp();
+#pragma unroll
+        for (int rt = 0; rt < BP / 16; ++rt) {
+          if (16 * rt >= b) continue;
+#pragma unroll
+          for (int nt = 0; nt < 8; ++nt) {
+            if (nt >= 2 * ksteps) continue;
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+              const int j = 16 * rt + g + 8 * hh;
+              if (j >= b) continue;
+              const uint32_t off = at(k, j, b, 8 * nt + 2 * t);
+              *reinterpret_cast<uint32_t*>(dstL + off) = outL[rt][nt][hh];
+              if (last) *reinterpret_cast<uint32_t*>(sV + off) = outY[rt][nt][hh];
+            }
+          }
+        }
+      }
+    }
+    __syncthreads();
+
+    // ================================================================ L half-step (Eq. 8, 9 / Eq. 4)
+    // tile j: Z_L[l,k] = fl * <Q(l,j), alpha_L(k,j)> - c_L(k,j), softmax over k
+    {
+      const uint32_t sAL_u = last ? sK_u : (uint32_t)__cvta_generic_to_shared(sALx);
+      for (int j = warp; j < b; j += kWarps) {
+        float c[MP / 8][2];
+#pragma unroll
+        for (int nt = 0; nt < MP / 8; ++nt)
+#pragma unroll
+          for (int e = 0; e < 2; ++e)
+            c[nt][e] = sCL[min(8 * nt + 2 * t + e, m - 1) * b + j] * kLog2e;
+        float pn[MP / 16][2][MP / 8][2];           // normalised weights [row tile][half][nt][e]
+#pragma unroll
+        for (int rt = 0; rt < MP / 16; ++rt) {
+          const int l0 = 16 * rt;
+          if (l0 >= m) {
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+              for (int nt = 0; nt < MP / 8; ++nt) pn[rt][hh][nt][0] = pn[rt][hh][nt][1] = 0.f;
+            continue;
+          }
+          float s[MP / 8][4];
+#pragma unroll
+          for (int nt = 0; nt < MP / 8; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
+          const int la = min(l0 + (lane & 7) + ((lane >> 3) & 1) * 8, m - 1);
+#pragma unroll
+          for (int ks = 0; ks < ksteps; ++ks) {
+            uint32_t a[4];
+            ldsm_x4(a, sQ_u + at(la, j, b, 16 * ks + (lane >> 4) * 8));
+#pragma unroll
+            for (int cp = 0; cp < MP / 16; ++cp) {
+              uint32_t bf[4];
+              const int kb = min(16 * cp + (lane & 7) + (lane >> 4) * 8, m - 1);
+              ldsm_x4(bf, sAL_u + at(kb, j, b, 16 * ks + ((lane >> 3) & 1) * 8));
+              Mma<T>::run(s[2 * cp], a, bf);
+              Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+            }
+          }
+          float inv_s[2];
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            float mx = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < MP / 8; ++nt)
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const float z = (8 * nt + 2 * t + e < m) ? fmaf(s[nt][2 * hh + e], fl, -c[nt][e])
+                                                         : -INFINITY;
+                s[nt][2 * hh + e] = z;
+                mx = fmaxf(mx, z);
+              }
+            mx = quad_max(mx);
+            float sum = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < MP / 8; ++nt)
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const float p = ex2(s[nt][2 * hh + e] - mx);
+                s[nt][2 * hh + e] = p;
+                sum += p;
+              }
+            inv_s[hh] = 1.f / quad_sum(sum);
+          }
+          if (last) {
+            // Y(l,j) = sum_k L[j,k,l] y(k,j)   (A = weights rows l, B = y rows (k,j) transposed)
+            uint32_t pa[MP / 16][4];
+#pragma unroll
+            for (int kk = 0; kk < MP / 16; ++kk) {
+              pa[kk][0] = Mma<T>::pack(s[2 * kk][0], s[2 * kk][1]);
+              pa[kk][1] = Mma<T>::pack(s[2 * kk][2], s[2 * kk][3]);
+              pa[kk][2] = Mma<T>::pack(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+              pa[kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+            }
+            uint32_t out[8][2];
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+              if (np >= ksteps) continue;
+              float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+              for (int kk = 0; kk < MP / 16; ++kk) {
+                uint32_t bf[4];
+                const int kb = min(16 * kk + (lane & 15), m - 1);
+                ldsm_x4_trans(bf, sV_u + at(kb, j, b, 16 * np + (lane >> 4) * 8));
+                Mma<T>::run(o[0], pa[kk], bf);
+                Mma<T>::run(o[1], pa[kk], bf + 2);
+              }
+#pragma unroll
+              for (int q = 0; q < 2; ++q) {
+                out[2 * np + q][0] = Mma<T>::pack(o[q][0] * inv_s[0], o[q][1] * inv_s[0]);
+                out[2 * np + q][1] = Mma<T>::pack(o[q][2] * inv_s[1], o[q][3] * inv_s[1]);
+              }
+            }
+            // only this warp reads the rows (l, j) of Q, and it has: Y takes their place
+            __syncwarp();
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+              if (nt >= 2 * ksteps) continue;
+#pragma unroll
+              for (int hh = 0; hh < 2; ++hh) {
+                const int l = l0 + g + 8 * hh;
+                if (l < m) *reinterpret_cast<uint32_t*>(sQ + at(l, j, b, 8 * nt + 2 * t)) = out[nt][hh];
+              }
+            }
+            __syncwarp();
+          } else {
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+              const bool row_ok = l0 + g + 8 * hh < m;     // rows past the block must not count
+#pragma unroll
+              for (int nt = 0; nt < MP / 8; ++nt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                  pn[rt][hh][nt][e] = row_ok ? s[nt][2 * hh + e] * inv_s[hh] : 0.f;
+            }
+          }
+        }
+        if (!last) {
+          // alpha_R(k,j) = sum_l L[j,k,l] Q(l,j) / c_R, c_R(k,j) = sum_l L[j,k,l]: the contraction
+          // runs over the ROW index of the weights, so the A fragments are their transpose.
+          // The result does not change when column k is multiplied by any g_k > 0: g_k = 2^-(exponent
+          // of the column's largest weight) keeps every column's significant weights in the normal
+          // f16 range however small c_R is.
+          uint32_t tp[MP / 16][2][MP / 8];
+          float cs[MP / 8][2];
+#pragma unroll
+          for (int nt = 0; nt < MP / 8; ++nt) {
+            float gk[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              float cm = 0.f;
+#pragma unroll
+              for (int rt = 0; rt < MP / 16; ++rt) cm = fmaxf(cm, fmaxf(pn[rt][0][nt][e], pn[rt][1][nt][e]));
+              cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 4));
+              cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 8));
+              cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 16));
+              gk[e] = cm > 0.f ? __uint_as_float((253u << 23) - (__float_as_uint(cm) & 0x7f800000u)) : 0.f;
+            }
+            // column sums of the weights AS ROUNDED to 16 bit: numerator (the MMA below) and
+            // denominator of the weighted mean must see the same weights
+            float c0 = 0.f, c1 = 0.f;
+#pragma unroll
+            for (int rt = 0; rt < MP / 16; ++rt)
+#pragma unroll
+              for (int hh = 0; hh < 2; ++hh) {
+                const uint32_t u = Mma<T>::pack(pn[rt][hh][nt][0] * gk[0], pn[rt][hh][nt][1] * gk[1]);
+                tp[rt][hh][nt] = u;
+                const float2 f = Mma<T>::unpack(u);
+                c0 += f.x;
+                c1 += f.y;
+              }
+            cs[nt][0] = col_sum(c0);
+            cs[nt][1] = col_sum(c1);
+          }
+#pragma unroll
+          for (int kt = 0; kt < MP / 16; ++kt) {
+            if (16 * kt >= m) continue;
+            // 1 / c_R of rows k = 16 kt + g and + 8: column k = 8 nt + 2 t' + e sits in lane t'
+            float ic[2];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+              const float v0 = __shfl_sync(0xffffffffu, cs[2 * kt + hh][0], g >> 1);
+              const float v1 = __shfl_sync(0xffffffffu, cs[2 * kt + hh][1], g >> 1);
+              const float cr = (g & 1) ? v1 : v0;
+              ic[hh] = cr > 1e-30f ? 1.f / cr : 0.f;
+            }
+            uint32_t pa[MP / 16][4];
+#pragma unroll
+            for (int ls = 0; ls < MP / 16; ++ls) {
+              pa[ls][0] = movm_trans(tp[ls][0][2 * kt]);       // rows k 0-7,  cols l 0-7
+              pa[ls][1] = movm_trans(tp[ls][0][2 * kt + 1]);   // rows k 8-15, cols l 0-7
+              pa[ls][2] = movm_trans(tp[ls][1][2 * kt]);       // rows k 0-7,  cols l 8-15
+              pa[ls][3] = movm_trans(tp[ls][1][2 * kt + 1]);   // rows k 8-15, cols l 8-15
+            }
+#pragma unroll
+            for (int nt = 0; nt < 2 * ksteps; ++nt) {
+              float o[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+              for (int ls = 0; ls < MP / 16; ++ls) {
+                uint32_t bf[2];   // B[kk = l][n = v] = Q(l,j)[v], read transposed
+                const int lb = min(16 * ls + (lane & 15), m - 1);
+                ldsm_x2_trans(bf, sQ_u + at(lb, j, b, 8 * nt));
+                Mma<T>::run(o, pa[ls], bf);
+              }
+              const int k0 = 16 * kt + g;
+              if (k0 < m)
+                *reinterpret_cast<uint32_t*>(sARx + at(k0, j, b, 8 * nt + 2 * t)) =
+                    Mma<T>::pack(o[0] * ic[0], o[1] * ic[0]);
+              if (k0 + 8 < m)
+                *reinterpret_cast<uint32_t*>(sARx + at(k0 + 8, j, b, 8 * nt + 2 * t)) =
+                    Mma<T>::pack(o[2] * ic[1], o[3] * ic[1]);
+            }
+          }
+        }
+      }
+    }
+    __syncthreads();
+  }
+
+  // ---- Y sits where Q was: 16-byte copies out
+  for (int idx = tid; idx < N * 8; idx += kThreads) {
+    const int row = idx >> 3, ch = idx & 7;
+    if (ch * 8 >= d) continue;
+    const int k = row / b, i = row - k * b;
+    const uint4 v = *reinterpret_cast<const uint4*>(sQ + at(k, i, b, ch * 8));
+    TIn* gp = Y + row_off(h_idx, row, N, d, H) + ch * 8;
+    *reinterpret_cast<uint4*>(gp) = fused::from_f16x8(v, gp);
+  }
+}
+
+inline bool supported(int N, int d, int b, int m, int dtype, int T) {
+  return (dtype == 1 || dtype == 2) && d % 8 == 0 && d <= 64 && b <= 32 && m <= 32 &&
+         smem_bytes(N, T) <= (size_t)kMaxSmem;
+}
+
+template <typename TIn, int BP, int MP>
+inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
+                    int m, int T, float scale, int n_valid, int H, cudaStream_t st) {
+  auto kern = monarch_fused_small<TIn, BP, MP>;
+  const size_t smem = smem_bytes(N, T);
+  if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+      cudaSuccess)
+    return 7;
+  kern<<<BH, kThreads, smem, st>>>((const TIn*)Q, (const TIn*)K, (const TIn*)V, (TIn*)Y, N, d, b, m, T,
+                                   scale, n_valid, H);
+  return cudaGetLastError() == cudaSuccess ? 0 : 7;
+}
+
+template <typename TIn>
+inline int launch_d(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
+                    int m, int T, float scale, int n_valid, int H, cudaStream_t st) {
+  if (b <= 16 && m <= 16) return launch_t<TIn, 16, 16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
+  if (b <= 16) return launch_t<TIn, 16, 32>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
+  if (m <= 16) return launch_t<TIn, 32, 16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
+  return launch_t<TIn, 32, 32>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
+}
+
+inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
+                  int m, int T, int dtype, float scale, int n_valid, int H, cudaStream_t st) {
+  if (dtype == 1) return launch_d<__half>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
+  return launch_d<__nv_bfloat16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
+}
+
+}  // namespace fsmall
+}  // namespace ma

@@ -197,6 +197,67 @@ def test_fused_kernel_is_the_default_for_its_shape_and_launches_once():
     assert torch.equal(a, b_)
 
 
+# ------------------------------------------------------------------ general fused per-head kernel
+@pytest.mark.parametrize("N,b,d,T,dtype", [
+    (256, 16, 64, 1, "f16"), (256, 16, 64, 3, "bf16"),      # 16 x 16 blocks (the special case's shape)
+    (210, 14, 64, 2, "f16"), (210, 15, 64, 2, "bf16"),      # blocks that do not fill 16 rows
+    (384, 24, 64, 1, "f16"), (384, 16, 64, 1, "bf16"),      # b > 16 with m = 16, and the reverse
+    (576, 32, 64, 1, "f16"),                                # largest single-round sequence, m = 18
+    (416, 13, 64, 2, "bf16"), (330, 11, 48, 2, "f16"),      # m = 32 / 30 with a short block, d = 48
+    (320, 32, 64, 3, "f16"), (100, 10, 40, 3, "f16"),       # d = 40: a half 16-column step
+    (60, 6, 8, 2, "f16"), (27, 3, 24, 4, "bf16"), (31, 31, 16, 2, "f16"), (29, 1, 32, 2, "f16"),
+])
+def test_general_fused_kernel_matches_oracle(N, b, d, T, dtype):
+    """Any m, b <= 32 and d <= 64 in one launch per call, states in shared memory (Sec. 3)."""
+    rank, s = (min(8, d), 1.0) if T <= 2 else (min(16, d), 1.5)
+    check(2, 3, N, d, b, T, dtype, rank=rank, s=s, seed=N + 3 * T, path=binding.MA_PATH_FUSED_SMALL)
+    assert binding.monarch_attn_last_launch_count() == 1
+
+
+def test_general_fused_kernel_many_heads_and_agreement_with_the_special_case():
+    check(151, 3, 210, 64, 14, 2, "f16", rank=8, s=1.0, seed=5, path=binding.MA_PATH_FUSED_SMALL)
+    Q, K, V = wl.make_qkv(3, 4, 256, 64, "f16", 8, 2.0, seed=21)
+    Qd, Kd, Vd = (binding.to_device(x, "f16") for x in (Q, K, V))
+    for T in (1, 2):
+        a = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 16, T, path=binding.MA_PATH_FUSED_SMALL).float()
+        b_ = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 16, T, path=binding.MA_PATH_FUSED).float()
+        assert float((a - b_).norm() / b_.norm()) <= 2e-3
+
+
+def test_general_fused_kernel_is_the_default_where_it_applies():
+    """AUTO: 16-bit inputs with small blocks take the one-launch kernel, with or without padding
+    and in either layout; fp32 inputs and sequences too long for shared memory do not."""
+    Q, K, V = wl.make_qkv(2, 2, 384, 64, "f16", 8, 1.0, seed=3)
+    Qd, Kd, Vd = (binding.to_device(x, "f16") for x in (Q, K, V))
+    a = binding.monarch_attn_fwd(Qd, Kd, Vd, 24, 1)
+    assert binding.monarch_attn_last_launch_count() == 1
+    assert torch.equal(a, binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 24, 1, path=binding.MA_PATH_FUSED_SMALL))
+    binding.monarch_attn_fwd_padded(Qd, Kd, Vd, 24, 1, 380)
+    assert binding.monarch_attn_last_launch_count() == 1
+    Qs, Ks, Vs = (x.transpose(1, 2).contiguous() for x in (Qd, Kd, Vd))
+    c = binding.monarch_attn_fwd_bshd(Qs, Ks, Vs, 24, 1)
+    assert binding.monarch_attn_last_launch_count() == 1
+    assert torch.equal(c.transpose(1, 2), a)
+    binding.monarch_attn_fwd(Qd, Kd, Vd, 24, 2)                    # N = 384 fits for two rounds too
+    assert binding.monarch_attn_last_launch_count() == 1
+    Q, K, V = wl.make_qkv(1, 2, 384, 64, "f32", 8, 1.0, seed=3)
+    x = [binding.to_device(t_, "f32") for t_ in (Q, K, V)]
+    binding.monarch_attn_fwd(*x, 24, 1)
+    assert binding.monarch_attn_last_launch_count() == 2           # generic: one launch per half-step
+    with pytest.raises(binding.MonarchAttnError) as e:
+        binding.monarch_attn_fwd_ex(*x, 24, 1, path=binding.MA_PATH_FUSED_SMALL)
+    assert e.value.code == 4
+    Q, K, V = wl.make_qkv(1, 1, 480, 64, "f16", 8, 1.0, seed=3)
+    x = [binding.to_device(t_, "f16") for t_ in (Q, K, V)]
+    binding.monarch_attn_fwd_ex(*x, 24, 1, path=binding.MA_PATH_FUSED_SMALL)     # one round: fits
+    with pytest.raises(binding.MonarchAttnError) as e:
+        binding.monarch_attn_fwd_ex(*x, 24, 2, path=binding.MA_PATH_FUSED_SMALL)
+    assert e.value.code == 4
+    with pytest.raises(binding.MonarchAttnError) as e:                           # m = 40 > 32
+        binding.monarch_attn_fwd_ex(*x, 12, 1, path=binding.MA_PATH_FUSED_SMALL)
+    assert e.value.code == 4
+
+
 # ------------------------------------------------------------------ properties at any size
 @pytest.mark.parametrize("path", [binding.MA_PATH_GENERIC, binding.MA_PATH_AUTO])
 def test_constant_v_and_zero_q(path):
@@ -355,6 +416,8 @@ def test_padded_entry_point_rejects_more_than_one_block_of_padding():
     (4096, 64, 64, 3, "bf16", 1, 37, binding.MA_PATH_AUTO),       # more heads than fit one wave
     (256, 16, 64, 1, "f32", 2, 3, binding.MA_PATH_AUTO),          # generic kernels
     (210, 14, 72, 2, "f16", 2, 5, binding.MA_PATH_GENERIC),       # m != b, d != 64
+    (210, 14, 64, 2, "f16", 2, 5, binding.MA_PATH_FUSED_SMALL),   # one CTA per head, strided rows
+    (384, 24, 48, 1, "bf16", 3, 2, binding.MA_PATH_AUTO),
 ])
 def test_batch_seq_head_layout_matches_oracle(N, b, d, T, dtype, batch, heads, path):
     """Tensors stored [batch, N, heads, d]: same result as the per-head oracle, bit for bit the
