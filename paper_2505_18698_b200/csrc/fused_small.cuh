@@ -46,6 +46,15 @@ using fused::quad_max;
 using fused::quad_sum;
 
 constexpr int kThreads = 256, kWarps = 8, kRowBytes = 128, kMaxSmem = 227 * 1024;
+constexpr int kDumpBytes = kThreads * 16;   // where stmatrix rows past the end of a block go
+
+// Four 8x8 16-bit matrices from accumulator-layout registers; lane L gives the address of row L & 7
+// of matrix L >> 3.
+__device__ __forceinline__ void stsm_x4(uint32_t saddr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(saddr), "r"(r0),
+               "r"(r1), "r"(r2), "r"(r3)
+               : "memory");
+}
 
 // Byte offset of element (block k, position i, column col) in a tile.
 __device__ __forceinline__ uint32_t at(int k, int i, int b, int col) {
@@ -53,15 +62,8 @@ __device__ __forceinline__ uint32_t at(int k, int i, int b, int col) {
   return (uint32_t)((k * b + i) * kRowBytes + (chunk << 4) + ((col & 7) << 1));
 }
 
-// Element offset of row n of head h in Q, K, V, Y (H = 0: [batch][heads][N][d]; else
-// [batch][N][H][d]).
-__device__ __forceinline__ size_t row_off(int h, int n, int N, int d, int H) {
-  if (H == 0) return ((size_t)h * N + n) * d;
-  return (((size_t)(h / H) * N + n) * H + (h % H)) * d;
-}
-
 inline size_t smem_bytes(int N, int T) {
-  return (size_t)(T == 1 ? 3 : 4) * N * kRowBytes + (size_t)N * 4 + 1024;
+  return (size_t)(T == 1 ? 3 : 4) * N * kRowBytes + (((size_t)N * 4 + 15) & ~(size_t)15) + kDumpBytes + 1024;
 }
 
 // BP, MP: b and m rounded up to 16 or 32.
@@ -77,10 +79,16 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   uint8_t* sQ = smem;
   uint8_t* sK = sQ + tile;
   uint8_t* sV = sK + tile;                         // V, loaded when the last round starts ...
-  uint8_t* sALx = sV;                              // ... alpha_L of the earlier rounds until then
-  uint8_t* sARx = sV + tile;                       // T > 1 only
+  //                                                  ... alpha_L of the earlier rounds until then;
+  // alpha_R (T > 1 only) follows it
   float* sCL = reinterpret_cast<float*>(smem + (T_steps == 1 ? 3 : 4) * (size_t)tile);   // [k*b + j]
   const uint32_t sQ_u = (uint32_t)__cvta_generic_to_shared(sQ);
+  // stmatrix writes whole 8-row matrices: rows past a block's end land in a per-lane dump slot
+  const uint32_t dump_u =
+      (uint32_t)__cvta_generic_to_shared(reinterpret_cast<uint8_t*>(sCL) + (((size_t)N * 4 + 15) & ~(size_t)15)) +
+      threadIdx.x * 16;   // 16-byte aligned like every stmatrix row
+  const int st_row = (threadIdx.x & 7) + ((threadIdx.x >> 3) & 1) * 8;   // row within a 16-row tile
+  const int st_nt = (threadIdx.x >> 4) & 1;                              // which of a pair of 8-column tiles
   const uint32_t sK_u = sQ_u + tile, sV_u = sK_u + tile;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -90,15 +98,21 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   // zero-filled on the way in and the states are products with them), so every loop unrolls.
   constexpr int ksteps = 4;
 
+  // Rows of this head in global memory, and row / b without a division (exact for row < 2^16).
+  const size_t head_base = H == 0 ? (size_t)h_idx * N * d : ((size_t)(h_idx / H) * N * H + (h_idx % H)) * d;
+  const size_t row_stride = H == 0 ? (size_t)d : (size_t)H * d;
+  const uint32_t magic = 0xffffffffu / (uint32_t)b + 1u;
+  auto block_of = [&](int row) { return b == 1 ? row : (int)__umulhi((uint32_t)row, magic); };
+
   // ---- load Q, K (and V when there is one round): 16-byte chunks; columns d..63 are zero
   auto load_tile = [&](const TIn* __restrict__ src, int a) {
     uint8_t* dst = smem + (size_t)a * tile;
-    for (int idx = tid; idx < N * 8; idx += kThreads) {
-      const int row = idx >> 3, ch = idx & 7;
-      const int k = row / b, i = row - k * b;
+    const int ch = tid & 7;
+    for (int row = tid >> 3; row < N; row += kThreads / 8) {
+      const int k = block_of(row), i = row - k * b;
       const uint32_t off = at(k, i, b, ch * 8);
       if (ch * 8 < d) {
-        const TIn* gp = src + row_off(h_idx, row, N, d, H) + ch * 8;
+        const TIn* gp = src + head_base + row * row_stride + ch * 8;
         if (Mma<TIn>::is_f16) {
           asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sQ_u + a * tile + off), "l"(gp));
         } else {
@@ -129,8 +143,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
     // ================================================================ R half-step (Eq. 7, 9, 10)
     // tile k: Z_R[j,i] = fl * <alpha_R(k,j), K(k,i)>, softmax over i, alpha_L(k,j) = sum_i R K(k,i)
     {
-      const uint32_t sA_u = first ? sQ_u : (uint32_t)__cvta_generic_to_shared(sARx);
-      uint8_t* dstL = last ? sK : sALx;
+      const uint32_t sA_u = first ? sQ_u : sV_u + tile;   // alpha_R (= Q rows while L is the identity)
       for (int k = warp; k < m; k += kWarps) {
         uint32_t outL[BP / 16][8][2], outY[BP / 16][8][2];
 #pragma unroll
@@ -233,20 +246,21 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
         }
         // this warp alone reads block k of K and V: on the last round the results take their place
         __syncwarp();
+        const uint32_t dstL_u = last ? sK_u : sV_u;     // alpha_L of earlier rounds shares V's buffer
 #pragma unroll
         for (int rt = 0; rt < BP / 16; ++rt) {
           if (16 * rt >= b) continue;
+          const int j = 16 * rt + st_row;
+          const uint32_t row_u = (uint32_t)((k * b + j) * kRowBytes);
+          const int x = (j & 7) ^ (k & 7);
 #pragma unroll
-          for (int nt = 0; nt < 8; ++nt) {
-            if (nt >= 2 * ksteps) continue;
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-              const int j = 16 * rt + g + 8 * hh;
-              if (j >= b) continue;
-              const uint32_t off = at(k, j, b, 8 * nt + 2 * t);
-              *reinterpret_cast<uint32_t*>(dstL + off) = outL[rt][nt][hh];
-              if (last) *reinterpret_cast<uint32_t*>(sV + off) = outY[rt][nt][hh];
-            }
+          for (int np = 0; np < 4; ++np) {
+            const uint32_t off = row_u + (uint32_t)(((2 * np + st_nt) ^ x) << 4);
+            stsm_x4(j < b ? dstL_u + off : dump_u, outL[rt][2 * np][0], outL[rt][2 * np][1],
+                    outL[rt][2 * np + 1][0], outL[rt][2 * np + 1][1]);
+            if (last)
+              stsm_x4(j < b ? sV_u + off : dump_u, outY[rt][2 * np][0], outY[rt][2 * np][1],
+                      outY[rt][2 * np + 1][0], outY[rt][2 * np + 1][1]);
           }
         }
       }
@@ -256,7 +270,8 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
     // ================================================================ L half-step (Eq. 8, 9 / Eq. 4)
     // tile j: Z_L[l,k] = fl * <Q(l,j), alpha_L(k,j)> - c_L(k,j), softmax over k
     {
-      const uint32_t sAL_u = last ? sK_u : (uint32_t)__cvta_generic_to_shared(sALx);
+      const uint32_t sAL_u = last ? sK_u : sV_u;      // alpha_L of earlier rounds shares V's buffer
+      const uint32_t sAR_u = sV_u + tile;
       for (int j = warp; j < b; j += kWarps) {
         float c[MP / 8][2];
 #pragma unroll
@@ -350,14 +365,14 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             }
             // only this warp reads the rows (l, j) of Q, and it has: Y takes their place
             __syncwarp();
+            {
+              const int l = l0 + st_row;
+              const uint32_t row_u = sQ_u + (uint32_t)((l * b + j) * kRowBytes);
+              const int x = (j & 7) ^ (l & 7);
 #pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-              if (nt >= 2 * ksteps) continue;
-#pragma unroll
-              for (int hh = 0; hh < 2; ++hh) {
-                const int l = l0 + g + 8 * hh;
-                if (l < m) *reinterpret_cast<uint32_t*>(sQ + at(l, j, b, 8 * nt + 2 * t)) = out[nt][hh];
-              }
+              for (int np = 0; np < 4; ++np)
+                stsm_x4(l < m ? row_u + (uint32_t)(((2 * np + st_nt) ^ x) << 4) : dump_u, out[2 * np][0],
+                        out[2 * np][1], out[2 * np + 1][0], out[2 * np + 1][1]);
             }
             __syncwarp();
           } else {
@@ -429,23 +444,23 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
               pa[ls][2] = movm_trans(tp[ls][1][2 * kt]);       // rows k 0-7,  cols l 8-15
               pa[ls][3] = movm_trans(tp[ls][1][2 * kt + 1]);   // rows k 8-15, cols l 8-15
             }
+            const int kr = 16 * kt + st_row;                   // alpha_R row (kr, j) this lane addresses
+            const uint32_t row_u = sAR_u + (uint32_t)((kr * b + j) * kRowBytes);
+            const int x = (j & 7) ^ (kr & 7);
 #pragma unroll
-            for (int nt = 0; nt < 2 * ksteps; ++nt) {
-              float o[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int np = 0; np < ksteps; ++np) {
+              float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
               for (int ls = 0; ls < MP / 16; ++ls) {
-                uint32_t bf[2];   // B[kk = l][n = v] = Q(l,j)[v], read transposed
+                uint32_t bf[4];   // B[kk = l][n = v] = Q(l,j)[v], read transposed; two 8-column tiles
                 const int lb = min(16 * ls + (lane & 15), m - 1);
-                ldsm_x2_trans(bf, sQ_u + at(lb, j, b, 8 * nt));
-                Mma<T>::run(o, pa[ls], bf);
+                ldsm_x4_trans(bf, sQ_u + at(lb, j, b, 16 * np + (lane >> 4) * 8));
+                Mma<T>::run(o[0], pa[ls], bf);
+                Mma<T>::run(o[1], pa[ls], bf + 2);
               }
-              const int k0 = 16 * kt + g;
-              if (k0 < m)
-                *reinterpret_cast<uint32_t*>(sARx + at(k0, j, b, 8 * nt + 2 * t)) =
-                    Mma<T>::pack(o[0] * ic[0], o[1] * ic[0]);
-              if (k0 + 8 < m)
-                *reinterpret_cast<uint32_t*>(sARx + at(k0 + 8, j, b, 8 * nt + 2 * t)) =
-                    Mma<T>::pack(o[2] * ic[1], o[3] * ic[1]);
+              stsm_x4(kr < m ? row_u + (uint32_t)(((2 * np + st_nt) ^ x) << 4) : dump_u,
+                      Mma<T>::pack(o[0][0] * ic[0], o[0][1] * ic[0]), Mma<T>::pack(o[0][2] * ic[1], o[0][3] * ic[1]),
+                      Mma<T>::pack(o[1][0] * ic[0], o[1][1] * ic[0]), Mma<T>::pack(o[1][2] * ic[1], o[1][3] * ic[1]));
             }
           }
         }
@@ -455,13 +470,14 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   }
 
   // ---- Y sits where Q was: 16-byte copies out
-  for (int idx = tid; idx < N * 8; idx += kThreads) {
-    const int row = idx >> 3, ch = idx & 7;
-    if (ch * 8 >= d) continue;
-    const int k = row / b, i = row - k * b;
-    const uint4 v = *reinterpret_cast<const uint4*>(sQ + at(k, i, b, ch * 8));
-    TIn* gp = Y + row_off(h_idx, row, N, d, H) + ch * 8;
-    *reinterpret_cast<uint4*>(gp) = fused::from_f16x8(v, gp);
+  if ((tid & 7) * 8 < d) {
+    const int ch = tid & 7;
+    for (int row = tid >> 3; row < N; row += kThreads / 8) {
+      const int k = block_of(row), i = row - k * b;
+      const uint4 v = *reinterpret_cast<const uint4*>(sQ + at(k, i, b, ch * 8));
+      TIn* gp = Y + head_base + row * row_stride + ch * 8;
+      *reinterpret_cast<uint4*>(gp) = fused::from_f16x8(v, gp);
+    }
   }
 }
 
