@@ -54,7 +54,8 @@ typedef enum {
   MA_PATH_TENSOR_CHAINED = 6, /* first-generation persistent kernel (each softmax warpgroup also
                                  does its tile's epilogue), one launch; kept for comparison */
   MA_PATH_FUSED = 5,   /* one CTA per (batch, head), everything in shared memory, one launch:
-                          f16/bf16, N = 256, m = b = 16, d = 64 */
+                          f16/bf16, N = 256, m = b = 16, d = 64 only; kept for comparison (AUTO
+                          takes MA_PATH_FUSED_SMALL for this shape too) */
   MA_PATH_FUSED_SMALL = 7 /* the same idea for any block shape: f16/bf16, m and b <= 32 (m need not
                              equal b), d <= 64 a multiple of 8, N <= 580 for T = 1 and <= 440 for
                              T > 1 (the states of a head must fit shared memory); f16 arithmetic */

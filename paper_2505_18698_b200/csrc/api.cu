@@ -136,7 +136,11 @@ static int launch_generic(const Problem& p, const void* Q, const void* K, const 
 // ------------------------------------------------------------------ path selection
 static int resolve_path(const Problem& p, int path) {
   if (path == MA_PATH_AUTO) {
-    if (fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_FUSED;
+    // Short sequences with small blocks: one CTA per head, states in shared memory.  The general
+    // kernel is the faster of the two fused kernels on the N = 256, b = 16 shape as well (matrix
+    // stores, per-warp pipelined loads), so AUTO never picks MA_PATH_FUSED.
+    if (p.b <= 16 && p.m <= 16 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T))
+      return MA_PATH_FUSED_SMALL;
     // bf16 with b = 32 and more than two rounds stays on the fp32-state kernels: on the peaky-logit
     // recipe of that shape the 8-bit mantissa of alpha_R (used twice from T = 3 on) costs 4e-2 on
     // the worst head; up to T = 2 the hi + lo alpha_L of the tensor path keeps it under 1e-2.
@@ -168,10 +172,7 @@ static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused
     if (path == MA_PATH_TENSOR) return -1;
   }
   if (with_fused_small && (path == MA_PATH_AUTO || path == MA_PATH_FUSED_SMALL)) {
-    const bool ok = fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T);
-    // AUTO keeps the N = 256 special case's shapes on the kernels they have always used
-    if (ok && (path == MA_PATH_FUSED_SMALL || !fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)))
-      return MA_PATH_FUSED_SMALL;
+    if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
     if (path == MA_PATH_FUSED_SMALL) return -1;
   }
   if ((path == MA_PATH_AUTO || path == MA_PATH_GENERIC) && generic_supported(p)) return MA_PATH_GENERIC;

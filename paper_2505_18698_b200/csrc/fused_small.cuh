@@ -77,8 +77,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int tile = N * kRowBytes;
   uint8_t* sQ = smem;
-  uint8_t* sK = sQ + tile;
-  uint8_t* sV = sK + tile;                         // V, loaded when the last round starts ...
+  // then K, then V (loaded when the last round starts) ...
   //                                                  ... alpha_L of the earlier rounds until then;
   // alpha_R (T > 1 only) follows it
   float* sCL = reinterpret_cast<float*>(smem + (T_steps == 1 ? 3 : 4) * (size_t)tile);   // [k*b + j]
@@ -98,53 +97,75 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   // zero-filled on the way in and the states are products with them), so every loop unrolls.
   constexpr int ksteps = 4;
 
-  // Rows of this head in global memory, and row / b without a division (exact for row < 2^16).
+  // Rows of this head in global memory.
   const size_t head_base = H == 0 ? (size_t)h_idx * N * d : ((size_t)(h_idx / H) * N * H + (h_idx % H)) * d;
   const size_t row_stride = H == 0 ? (size_t)d : (size_t)H * d;
-  const uint32_t magic = 0xffffffffu / (uint32_t)b + 1u;
-  auto block_of = [&](int row) { return b == 1 ? row : (int)__umulhi((uint32_t)row, magic); };
 
-  // ---- load Q, K (and V when there is one round): 16-byte chunks; columns d..63 are zero
-  auto load_tile = [&](const TIn* __restrict__ src, int a) {
-    uint8_t* dst = smem + (size_t)a * tile;
-    const int ch = tid & 7;
-    for (int row = tid >> 3; row < N; row += kThreads / 8) {
-      const int k = block_of(row), i = row - k * b;
-      const uint32_t off = at(k, i, b, ch * 8);
+  // ---- loads.  A warp copies the blocks it owns in the first R half-step itself (Q, K and, when
+  // there is one round, V of block k = warp, warp + 8, ...), one asynchronous group per block, and
+  // starts on a block as soon as that group has landed: no CTA-wide wait before the first tile.
+  // The raw 16-bit values are copied; bf16 is converted to f16 in place by the lane that copied it.
+  auto load_block = [&](const TIn* __restrict__ src, int a, int k) {
+    for (int idx = lane; idx < b * 8; idx += 32) {
+      const int i = idx >> 3, ch = idx & 7;
+      const uint32_t off = (uint32_t)(a * tile) + at(k, i, b, ch * 8);
       if (ch * 8 < d) {
-        const TIn* gp = src + head_base + row * row_stride + ch * 8;
-        if (Mma<TIn>::is_f16) {
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sQ_u + a * tile + off), "l"(gp));
-        } else {
-          *reinterpret_cast<uint4*>(dst + off) =
-              fused::to_f16x8(__ldg(reinterpret_cast<const uint4*>(gp)), gp);
-        }
+        const TIn* gp = src + head_base + (size_t)(k * b + i) * row_stride + ch * 8;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sQ_u + off), "l"(gp) : "memory");
       } else {
-        *reinterpret_cast<uint4*>(dst + off) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(smem + off) = make_uint4(0u, 0u, 0u, 0u);   // columns d..63
       }
     }
   };
-  load_tile(Q, 0);
-  load_tile(K, 1);
-  if (T_steps == 1) load_tile(V, 2);
-  asm volatile("cp.async.commit_group;");
-  asm volatile("cp.async.wait_group 0;");
-  __syncthreads();
+  auto convert_block = [&](int a, int k) {
+    if (!Mma<TIn>::is_f16) {
+      for (int idx = lane; idx < b * 8; idx += 32) {
+        const int i = idx >> 3, ch = idx & 7;
+        if (ch * 8 >= d) continue;
+        uint4* p = reinterpret_cast<uint4*>(smem + (size_t)a * tile + at(k, i, b, ch * 8));
+        *p = fused::to_f16x8(*p, (const TIn*)nullptr);
+      }
+    }
+  };
+  auto wait_pending = [&](int n) {   // until at most n of this thread's copy groups are in flight
+    if (n <= 0) asm volatile("cp.async.wait_group 0;" ::: "memory");
+    else if (n == 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else if (n == 2) asm volatile("cp.async.wait_group 2;" ::: "memory");
+    else asm volatile("cp.async.wait_group 3;" ::: "memory");
+  };
+  int my_tiles = 0;                  // blocks this warp owns in an R half-step (at most 4)
+  for (int k = warp; k < m; k += kWarps) {
+    load_block(Q, 0, k);
+    load_block(K, 1, k);
+    if (T_steps == 1) load_block(V, 2, k);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    ++my_tiles;
+  }
 
   const float fl = scale * kLog2e;
   for (int step = 1; step <= T_steps; ++step) {
     const bool first = step == 1, last = step == T_steps;
     if (last && !first) {   // alpha_L of the round before is dead: V takes its buffer
-      load_tile(V, 2);
-      asm volatile("cp.async.commit_group;");
-      asm volatile("cp.async.wait_group 0;");
-      __syncthreads();
+      for (int k = warp; k < m; k += kWarps) {
+        load_block(V, 2, k);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      }
     }
     // ================================================================ R half-step (Eq. 7, 9, 10)
     // tile k: Z_R[j,i] = fl * <alpha_R(k,j), K(k,i)>, softmax over i, alpha_L(k,j) = sum_i R K(k,i)
     {
       const uint32_t sA_u = first ? sQ_u : sV_u + tile;   // alpha_R (= Q rows while L is the identity)
-      for (int k = warp; k < m; k += kWarps) {
+      int it = 0;
+      for (int k = warp; k < m; k += kWarps, ++it) {
+        if (first || last) {          // block k may still be on its way
+          wait_pending(my_tiles - 1 - it);
+          if (first) {
+            convert_block(0, k);
+            convert_block(1, k);
+          }
+          if (last) convert_block(2, k);
+          __syncwarp();
+        }
         uint32_t outL[BP / 16][8][2], outY[BP / 16][8][2];
 #pragma unroll
         for (int rt = 0; rt < BP / 16; ++rt) {
@@ -387,6 +408,16 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             }
           }
         }
+        if (last) {
+          // the m rows (l, j) of Y are complete: this warp copies them out, 16 bytes per lane
+          for (int idx = lane; idx < m * 8; idx += 32) {
+            const int l = idx >> 3, ch = idx & 7;
+            if (ch * 8 >= d) continue;
+            const uint4 v = *reinterpret_cast<const uint4*>(sQ + at(l, j, b, ch * 8));
+            TIn* gp = Y + head_base + (size_t)(l * b + j) * row_stride + ch * 8;
+            *reinterpret_cast<uint4*>(gp) = fused::from_f16x8(v, gp);
+          }
+        }
         if (!last) {
           // alpha_R(k,j) = sum_l L[j,k,l] Q(l,j) / c_R, c_R(k,j) = sum_l L[j,k,l]: the contraction
           // runs over the ROW index of the weights, so the A fragments are their transpose.
@@ -469,16 +500,6 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
     __syncthreads();
   }
 
-  // ---- Y sits where Q was: 16-byte copies out
-  if ((tid & 7) * 8 < d) {
-    const int ch = tid & 7;
-    for (int row = tid >> 3; row < N; row += kThreads / 8) {
-      const int k = block_of(row), i = row - k * b;
-      const uint4 v = *reinterpret_cast<const uint4*>(sQ + at(k, i, b, ch * 8));
-      TIn* gp = Y + head_base + row * row_stride + ch * 8;
-      *reinterpret_cast<uint4*>(gp) = fused::from_f16x8(v, gp);
-    }
-  }
 }
 
 inline bool supported(int N, int d, int b, int m, int dtype, int T) {

@@ -187,14 +187,17 @@ def test_fused_kernel_matches_oracle(batch, heads, T, dtype):
           path=binding.MA_PATH_FUSED)
 
 
-def test_fused_kernel_is_the_default_for_its_shape_and_launches_once():
+def test_a_fused_kernel_is_the_default_for_short_sequences_and_launches_once():
     Q, K, V = wl.make_qkv(2, 2, 256, 64, "f16", 8, 2.0, seed=12)
     Qd, Kd, Vd = (binding.to_device(x, "f16") for x in (Q, K, V))
     a = binding.monarch_attn_fwd(Qd, Kd, Vd, 16, 2)
     assert binding.monarch_attn_last_launch_count() == 1
-    b_ = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 16, 2, path=binding.MA_PATH_FUSED)
+    b_ = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 16, 2, path=binding.MA_PATH_FUSED_SMALL)
+    assert binding.monarch_attn_last_launch_count() == 1
     torch.cuda.synchronize()
     assert torch.equal(a, b_)
+    binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 16, 2, path=binding.MA_PATH_FUSED)
+    assert binding.monarch_attn_last_launch_count() == 1
 
 
 # ------------------------------------------------------------------ general fused per-head kernel
