@@ -62,6 +62,13 @@ __device__ __forceinline__ uint32_t at(int k, int i, int b, int col) {
   return (uint32_t)((k * b + i) * kRowBytes + (chunk << 4) + ((col & 7) << 1));
 }
 
+// The same for the 16-column step `step` when the lane's chunk within the step is c (0 or 1):
+// rowx(k, i, b, c) ^ (step << 5), valid on top of any 128-byte aligned tile address -- one XOR per
+// fragment load instead of the whole index computation.
+__device__ __forceinline__ uint32_t rowx(int k, int i, int b, int c) {
+  return (uint32_t)((k * b + i) * kRowBytes + ((c ^ (i & 7) ^ (k & 7)) << 4));
+}
+
 inline size_t smem_bytes(int N, int T) {
   return (size_t)(T == 1 ? 3 : 4) * N * kRowBytes + (((size_t)N * 4 + 15) & ~(size_t)15) + kDumpBytes + 1024;
 }
@@ -106,8 +113,8 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   // starts on a block as soon as that group has landed: no CTA-wide wait before the first tile.
   // The raw 16-bit values are copied; bf16 is converted to f16 in place by the lane that copied it.
   auto load_block = [&](const TIn* __restrict__ src, int a, int k) {
-    for (int idx = lane; idx < b * 8; idx += 32) {
-      const int i = idx >> 3, ch = idx & 7;
+    const int ch = lane & 7;
+    for (int i = lane >> 3; i < b; i += 4) {
       const uint32_t off = (uint32_t)(a * tile) + at(k, i, b, ch * 8);
       if (ch * 8 < d) {
         const TIn* gp = src + head_base + (size_t)(k * b + i) * row_stride + ch * 8;
@@ -119,8 +126,8 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   };
   auto convert_block = [&](int a, int k) {
     if (!Mma<TIn>::is_f16) {
-      for (int idx = lane; idx < b * 8; idx += 32) {
-        const int i = idx >> 3, ch = idx & 7;
+      const int ch = lane & 7;
+      for (int i = lane >> 3; i < b; i += 4) {
         if (ch * 8 >= d) continue;
         uint4* p = reinterpret_cast<uint4*>(smem + (size_t)a * tile + at(k, i, b, ch * 8));
         *p = fused::to_f16x8(*p, (const TIn*)nullptr);
@@ -176,16 +183,20 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
           for (int nt = 0; nt < BP / 8; ++nt)
 #pragma unroll
             for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
-          const int ja = min(j0 + (lane & 7) + ((lane >> 3) & 1) * 8, b - 1);
+          const uint32_t a_u =
+              sA_u + rowx(k, min(j0 + (lane & 7) + ((lane >> 3) & 1) * 8, b - 1), b, lane >> 4);
+          uint32_t b_u[BP / 16];
+#pragma unroll
+          for (int cp = 0; cp < BP / 16; ++cp)
+            b_u[cp] = sK_u + rowx(k, min(16 * cp + (lane & 7) + (lane >> 4) * 8, b - 1), b, (lane >> 3) & 1);
 #pragma unroll
           for (int ks = 0; ks < ksteps; ++ks) {
             uint32_t a[4];
-            ldsm_x4(a, sA_u + at(k, ja, b, 16 * ks + (lane >> 4) * 8));
+            ldsm_x4(a, a_u ^ (ks << 5));
 #pragma unroll
             for (int cp = 0; cp < BP / 16; ++cp) {
               uint32_t bf[4];
-              const int ib = min(16 * cp + (lane & 7) + (lane >> 4) * 8, b - 1);
-              ldsm_x4(bf, sK_u + at(k, ib, b, 16 * ks + ((lane >> 3) & 1) * 8));
+              ldsm_x4(bf, b_u[cp] ^ (ks << 5));
               Mma<T>::run(s[2 * cp], a, bf);
               Mma<T>::run(s[2 * cp + 1], a, bf + 2);
             }
@@ -232,6 +243,9 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             pa[kk][2] = Mma<T>::pack(s[2 * kk + 1][0], s[2 * kk + 1][1]);
             pa[kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
           }
+          uint32_t v_off[BP / 16];    // rows (k, i) of K and V as the second product's B operand
+#pragma unroll
+          for (int kk = 0; kk < BP / 16; ++kk) v_off[kk] = rowx(k, min(16 * kk + (lane & 15), b - 1), b, lane >> 4);
 #pragma unroll
           for (int np = 0; np < 4; ++np) {     // two 8-column tiles of v per transposing ldmatrix
             if (np >= ksteps) {
@@ -246,12 +260,11 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
 #pragma unroll
             for (int kk = 0; kk < BP / 16; ++kk) {
               uint32_t bf[4];
-              const int ib = min(16 * kk + (lane & 15), b - 1);
-              ldsm_x4_trans(bf, sK_u + at(k, ib, b, 16 * np + (lane >> 4) * 8));
+              ldsm_x4_trans(bf, (sK_u + v_off[kk]) ^ (np << 5));
               Mma<T>::run(o[0], pa[kk], bf);
               Mma<T>::run(o[1], pa[kk], bf + 2);
               if (last) {
-                ldsm_x4_trans(bf, sV_u + at(k, ib, b, 16 * np + (lane >> 4) * 8));
+                ldsm_x4_trans(bf, (sV_u + v_off[kk]) ^ (np << 5));
                 Mma<T>::run(y[0], pa[kk], bf);
                 Mma<T>::run(y[1], pa[kk], bf + 2);
               }
@@ -272,11 +285,10 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
         for (int rt = 0; rt < BP / 16; ++rt) {
           if (16 * rt >= b) continue;
           const int j = 16 * rt + st_row;
-          const uint32_t row_u = (uint32_t)((k * b + j) * kRowBytes);
-          const int x = (j & 7) ^ (k & 7);
+          const uint32_t row_u = rowx(k, j, b, st_nt);
 #pragma unroll
           for (int np = 0; np < 4; ++np) {
-            const uint32_t off = row_u + (uint32_t)(((2 * np + st_nt) ^ x) << 4);
+            const uint32_t off = row_u ^ (np << 5);
             stsm_x4(j < b ? dstL_u + off : dump_u, outL[rt][2 * np][0], outL[rt][2 * np][1],
                     outL[rt][2 * np + 1][0], outL[rt][2 * np + 1][1]);
             if (last)
@@ -316,16 +328,20 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
           for (int nt = 0; nt < MP / 8; ++nt)
 #pragma unroll
             for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
-          const int la = min(l0 + (lane & 7) + ((lane >> 3) & 1) * 8, m - 1);
+          const uint32_t a_u =
+              sQ_u + rowx(min(l0 + (lane & 7) + ((lane >> 3) & 1) * 8, m - 1), j, b, lane >> 4);
+          uint32_t b_u[MP / 16];
+#pragma unroll
+          for (int cp = 0; cp < MP / 16; ++cp)
+            b_u[cp] = sAL_u + rowx(min(16 * cp + (lane & 7) + (lane >> 4) * 8, m - 1), j, b, (lane >> 3) & 1);
 #pragma unroll
           for (int ks = 0; ks < ksteps; ++ks) {
             uint32_t a[4];
-            ldsm_x4(a, sQ_u + at(la, j, b, 16 * ks + (lane >> 4) * 8));
+            ldsm_x4(a, a_u ^ (ks << 5));
 #pragma unroll
             for (int cp = 0; cp < MP / 16; ++cp) {
               uint32_t bf[4];
-              const int kb = min(16 * cp + (lane & 7) + (lane >> 4) * 8, m - 1);
-              ldsm_x4(bf, sAL_u + at(kb, j, b, 16 * ks + ((lane >> 3) & 1) * 8));
+              ldsm_x4(bf, b_u[cp] ^ (ks << 5));
               Mma<T>::run(s[2 * cp], a, bf);
               Mma<T>::run(s[2 * cp + 1], a, bf + 2);
             }
@@ -366,6 +382,10 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
               pa[kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
             }
             uint32_t out[8][2];
+            uint32_t y_u[MP / 16];
+#pragma unroll
+            for (int kk = 0; kk < MP / 16; ++kk)
+              y_u[kk] = sV_u + rowx(min(16 * kk + (lane & 15), m - 1), j, b, lane >> 4);
 #pragma unroll
             for (int np = 0; np < 4; ++np) {
               if (np >= ksteps) continue;
@@ -373,8 +393,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
 #pragma unroll
               for (int kk = 0; kk < MP / 16; ++kk) {
                 uint32_t bf[4];
-                const int kb = min(16 * kk + (lane & 15), m - 1);
-                ldsm_x4_trans(bf, sV_u + at(kb, j, b, 16 * np + (lane >> 4) * 8));
+                ldsm_x4_trans(bf, y_u[kk] ^ (np << 5));
                 Mma<T>::run(o[0], pa[kk], bf);
                 Mma<T>::run(o[1], pa[kk], bf + 2);
               }
@@ -388,11 +407,10 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             __syncwarp();
             {
               const int l = l0 + st_row;
-              const uint32_t row_u = sQ_u + (uint32_t)((l * b + j) * kRowBytes);
-              const int x = (j & 7) ^ (l & 7);
+              const uint32_t row_u = sQ_u + rowx(l, j, b, st_nt);
 #pragma unroll
               for (int np = 0; np < 4; ++np)
-                stsm_x4(l < m ? row_u + (uint32_t)(((2 * np + st_nt) ^ x) << 4) : dump_u, out[2 * np][0],
+                stsm_x4(l < m ? row_u ^ (np << 5) : dump_u, out[2 * np][0],
                         out[2 * np][1], out[2 * np + 1][0], out[2 * np + 1][1]);
             }
             __syncwarp();
@@ -410,8 +428,8 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
         }
         if (last) {
           // the m rows (l, j) of Y are complete: this warp copies them out, 16 bytes per lane
-          for (int idx = lane; idx < m * 8; idx += 32) {
-            const int l = idx >> 3, ch = idx & 7;
+          const int ch = lane & 7;
+          for (int l = lane >> 3; l < m; l += 4) {
             if (ch * 8 >= d) continue;
             const uint4 v = *reinterpret_cast<const uint4*>(sQ + at(l, j, b, ch * 8));
             TIn* gp = Y + head_base + (size_t)(l * b + j) * row_stride + ch * 8;
@@ -475,21 +493,23 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
               pa[ls][2] = movm_trans(tp[ls][1][2 * kt]);       // rows k 0-7,  cols l 8-15
               pa[ls][3] = movm_trans(tp[ls][1][2 * kt + 1]);   // rows k 8-15, cols l 8-15
             }
+            uint32_t q_u[MP / 16];
+#pragma unroll
+            for (int ls = 0; ls < MP / 16; ++ls)
+              q_u[ls] = sQ_u + rowx(min(16 * ls + (lane & 15), m - 1), j, b, lane >> 4);
             const int kr = 16 * kt + st_row;                   // alpha_R row (kr, j) this lane addresses
-            const uint32_t row_u = sAR_u + (uint32_t)((kr * b + j) * kRowBytes);
-            const int x = (j & 7) ^ (kr & 7);
+            const uint32_t row_u = sAR_u + rowx(kr, j, b, st_nt);
 #pragma unroll
             for (int np = 0; np < ksteps; ++np) {
               float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
               for (int ls = 0; ls < MP / 16; ++ls) {
                 uint32_t bf[4];   // B[kk = l][n = v] = Q(l,j)[v], read transposed; two 8-column tiles
-                const int lb = min(16 * ls + (lane & 15), m - 1);
-                ldsm_x4_trans(bf, sQ_u + at(lb, j, b, 16 * np + (lane >> 4) * 8));
+                ldsm_x4_trans(bf, q_u[ls] ^ (np << 5));
                 Mma<T>::run(o[0], pa[ls], bf);
                 Mma<T>::run(o[1], pa[ls], bf + 2);
               }
-              stsm_x4(kr < m ? row_u + (uint32_t)(((2 * np + st_nt) ^ x) << 4) : dump_u,
+              stsm_x4(kr < m ? row_u ^ (np << 5) : dump_u,
                       Mma<T>::pack(o[0][0] * ic[0], o[0][1] * ic[0]), Mma<T>::pack(o[0][2] * ic[1], o[0][3] * ic[1]),
                       Mma<T>::pack(o[1][0] * ic[0], o[1][1] * ic[0]), Mma<T>::pack(o[1][2] * ic[1], o[1][3] * ic[1]));
             }
