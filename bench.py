@@ -253,12 +253,12 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="C5", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--workload", default="C5", choices=sorted(wl.WORKLOADS) + sorted(wl.EXTRA_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the other configurations, SDPA context and the CPU baseline")
     args = ap.parse_args()
-    w = wl.WORKLOADS[args.workload]
+    w = {**wl.WORKLOADS, **wl.EXTRA_WORKLOADS}[args.workload]
     if args.impl == "reference":
         run_reference(args, w)
         return

@@ -88,6 +88,15 @@ WORKLOADS = {
                    "long sequence"),
 }
 
+# Shapes of the paper's short-sequence experiments (Sec. 5) with blocks that are not 16 x 16:
+# selectable in bench.py by name, not part of the configuration list the bench reports on.
+EXTRA_WORKLOADS = {
+    "S1": Workload("S1", 64, 12, 210, 64, 14, 2, "f16", 8, 1.0, 5,
+                   "ViT-B sequence (197 padded to 15 blocks of 14), two rounds"),
+    "S2": Workload("S2", 32, 12, 384, 64, 24, 1, "f16", 8, 1.0, 6,
+                   "RoBERTa sequence 384 as 16 blocks of 24, one round"),
+}
+
 
 # --------------------------------------------------------------------------- rounding
 def round_to_dtype(x: np.ndarray, dtype: str) -> np.ndarray:
