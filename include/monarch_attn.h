@@ -100,7 +100,8 @@ int monarch_attn_fwd_host(const void* Q_host, const void* K_host, const void* V_
  * half-step has that number for each row anyway and writes it out:
  *   row_lse: DEVICE pointer, [batch][heads][N] floats (natural logarithm), row b l + j of a head;
  *   f of a head = sum of its N entries (the caller reduces; 4-byte aligned).
- * `path`: MA_PATH_AUTO, MA_PATH_TENSOR (second-generation kernel) or MA_PATH_GENERIC.  Y, workspace
+ * `path`: MA_PATH_AUTO, MA_PATH_TENSOR (second-generation kernel), MA_PATH_FUSED_SMALL or
+ * MA_PATH_GENERIC.  Y, workspace
  * and everything else as monarch_attn_fwd_ex.  Asynchronous on `stream`. */
 int monarch_attn_fwd_objective(const void* Q, const void* K, const void* V, void* Y, int batch,
                                int heads, int N, int d, int b, int T, int dtype,
@@ -132,8 +133,10 @@ int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, 
  * n_valid must satisfy N - b < n_valid <= N (less than one block of padding, so that every key
  * block keeps a valid key; anything else is MA_ERR_SHAPE).  n_valid == N is the unpadded pass.
  * Runs on the general fused kernel (MA_PATH_FUSED_SMALL) where that supports the shape and dtype,
- * else on the generic kernels (any dtype, m need not equal b); a workspace sized for
- * monarch_attn_fwd_ex with path MA_PATH_GENERIC serves both.  Asynchronous on `stream`. */
+ * on the second-generation tensor kernel (MA_PATH_TENSOR) for f16/bf16 with d = 64 and
+ * m = b in {64, 128}, else on the generic kernels (any dtype, m need not equal b).  Workspace: the
+ * larger of monarch_attn_workspace_bytes() for MA_PATH_TENSOR and MA_PATH_GENERIC serves all three
+ * (a return of 0 means that path does not apply).  Asynchronous on `stream`. */
 int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y, int batch,
                             int heads, int N, int d, int b, int T, int dtype, float softmax_scale,
                             int n_valid, void* workspace, size_t workspace_bytes, void* stream);

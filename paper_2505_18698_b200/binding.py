@@ -217,7 +217,8 @@ def monarch_attn_fwd_padded(Q, K, V, b, T, n_valid, softmax_scale=None, workspac
     if Y is None:
         Y = torch.empty_like(Q)
     if workspace is None:
-        need = lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_GENERIC)
+        need = max(lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_TENSOR),
+                   lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_GENERIC))
         workspace = torch.empty(max(int(need), 256), dtype=torch.uint8, device=Q.device)
     _check(lib.monarch_attn_fwd_padded(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                        batch, heads, N, d, b, T, code, float(softmax_scale),

@@ -163,7 +163,7 @@ static int resolve_path(const Problem& p, int path) {
 }
 
 // Path choice of the entry points that only the second-generation tensor kernel, the general fused
-// kernel (layout and padding, no extra outputs: `with_fused_small`) and the generic kernels serve:
+// kernel (`with_fused_small`) and the generic kernels serve:
 // AUTO, TENSOR, FUSED_SMALL or GENERIC; -1 if none applies.
 static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused_small = false) {
   if (path == MA_PATH_AUTO || path == MA_PATH_TENSOR) {
@@ -230,7 +230,7 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
     return rc;
   }
   if (resolved == MA_PATH_FUSED_SMALL) {
-    int rc = fsmall::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.m, p.T, p.dtype, scale, p.n_valid, p.H, st);
+    int rc = fsmall::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.m, p.T, p.dtype, scale, p.n_valid, p.H, p.lse, st);
     if (rc == MA_OK) g_last_launches = 1;
     return rc;
   }
@@ -241,7 +241,7 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   else
     rc = tp::launch(Q, K, V, Y, p.BH, p.N, p.b, p.T, p.dtype, scale, ws, st, &launches,
                     resolved == MA_PATH_TENSOR ? 0 : (resolved == MA_PATH_TENSOR_PHASED ? 1 : 2),
-                    ws_armed, p.H, p.lse);
+                    ws_armed, p.H, p.lse, p.n_valid < p.N ? p.n_valid : 0);
   if (rc == MA_OK) g_last_launches = launches;
   return rc;
 }
@@ -299,9 +299,12 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
   rc = check_ptrs(Q, K, V, Y, p);
   if (rc != MA_OK) return rc;
   if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
-  const int r = fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)
-                    ? MA_PATH_FUSED_SMALL
-                    : (generic_supported(p) ? MA_PATH_GENERIC : -1);
+  // fused kernel for short sequences; the second-generation tensor kernel where a tile row owns a
+  // whole key block (b = 64, 128: the mask touches the last block's tiles only); else generic
+  int r = -1;
+  if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) r = MA_PATH_FUSED_SMALL;
+  else if (resolve_path(p, MA_PATH_AUTO) == MA_PATH_TENSOR && p.b != 32) r = MA_PATH_TENSOR;
+  else if (generic_supported(p)) r = MA_PATH_GENERIC;
   if (r < 0) return MA_ERR_UNSUPPORTED;
   p.n_valid = n_valid;
   return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);
@@ -319,7 +322,7 @@ int monarch_attn_fwd_objective(const void* Q, const void* K, const void* V, void
   if (!row_lse) return MA_ERR_NULL;
   if (((uintptr_t)row_lse & 3) != 0) return MA_ERR_ALIGN;
   if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
-  const int r = resolve_tensor_or_generic(p, path);
+  const int r = resolve_tensor_or_generic(p, path, true);
   if (r < 0) return MA_ERR_UNSUPPORTED;
   p.lse = row_lse;
   return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);

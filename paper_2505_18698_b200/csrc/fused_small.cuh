@@ -78,7 +78,7 @@ template <typename TIn, int BP, int MP>
 __global__ void __launch_bounds__(kThreads, (BP == 16 && MP == 16) ? 2 : 1)
 monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
                     TIn* __restrict__ Y, int N, int d, int b, int m, int T_steps, float scale,
-                    int n_valid, int H) {
+                    int n_valid, int H, float* __restrict__ lse) {
   typedef __half T;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -369,7 +369,12 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
                 s[nt][2 * hh + e] = p;
                 sum += p;
               }
-            inv_s[hh] = 1.f / quad_sum(sum);
+            sum = quad_sum(sum);
+            inv_s[hh] = 1.f / sum;
+            // log-sum-exp of row b l + j of the final L half-step: summed over a head's rows it is
+            // the objective (Eq. 6) at the returned matrix
+            if (last && lse != nullptr && t == 0 && l0 + g + 8 * hh < m)
+              lse[(size_t)h_idx * N + (size_t)(l0 + g + 8 * hh) * b + j] = (mx + log2f(sum)) * kLn2;
           }
           if (last) {
             // Y(l,j) = sum_k L[j,k,l] y(k,j)   (A = weights rows l, B = y rows (k,j) transposed)
@@ -529,30 +534,30 @@ inline bool supported(int N, int d, int b, int m, int dtype, int T) {
 
 template <typename TIn, int BP, int MP>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
-                    int m, int T, float scale, int n_valid, int H, cudaStream_t st) {
+                    int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st) {
   auto kern = monarch_fused_small<TIn, BP, MP>;
   const size_t smem = smem_bytes(N, T);
   if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
     return 7;
   kern<<<BH, kThreads, smem, st>>>((const TIn*)Q, (const TIn*)K, (const TIn*)V, (TIn*)Y, N, d, b, m, T,
-                                   scale, n_valid, H);
+                                   scale, n_valid, H, lse);
   return cudaGetLastError() == cudaSuccess ? 0 : 7;
 }
 
 template <typename TIn>
 inline int launch_d(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
-                    int m, int T, float scale, int n_valid, int H, cudaStream_t st) {
-  if (b <= 16 && m <= 16) return launch_t<TIn, 16, 16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
-  if (b <= 16) return launch_t<TIn, 16, 32>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
-  if (m <= 16) return launch_t<TIn, 32, 16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
-  return launch_t<TIn, 32, 32>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
+                    int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st) {
+  if (b <= 16 && m <= 16) return launch_t<TIn, 16, 16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
+  if (b <= 16) return launch_t<TIn, 16, 32>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
+  if (m <= 16) return launch_t<TIn, 32, 16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
+  return launch_t<TIn, 32, 32>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
 }
 
 inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
-                  int m, int T, int dtype, float scale, int n_valid, int H, cudaStream_t st) {
-  if (dtype == 1) return launch_d<__half>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
-  return launch_d<__nv_bfloat16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, st);
+                  int m, int T, int dtype, float scale, int n_valid, int H, float* lse, cudaStream_t st) {
+  if (dtype == 1) return launch_d<__half>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
+  return launch_d<__nv_bfloat16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
 }
 
 }  // namespace fsmall

@@ -509,6 +509,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         }
         f = P.scale * inv_c * kLog2e;
         float2 z2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        // Padding mask (App. C.3): in the last key block the columns from `lim` on are keys past
+        // n_valid; they take no part in the maximum and get weight 0.
+        int lim = B;
+        if (EXTRA && SB == B && P.n_valid != 0 && t.idx0 + blk == m - 1) lim = P.n_valid - (m - 1) * SB;
         if constexpr (SB == B) {
           // Every row owns all B columns: 16-column chunks, the load of the next chunk in flight
           // while the current one is worked on (TMEM reads compete with the MMAs' accumulator
@@ -524,6 +528,11 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             float* nxt = (cc & 1) ? b0 : b1;
             tmem_ld_wait();
             tmem_ld16(tS + 16 * ((cc + 1) % NC16), nxt);     // wraps to the first chunk of pass 2
+            if (EXTRA && lim < B) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                if (16 * cc + i >= lim) cur[i] = -INFINITY;
+            }
 #pragma unroll
             for (int i = 0; i < 8; ++i) m4[i & 3] = max3(m4[i & 3], cur[2 * i], cur[2 * i + 1]);
           }
@@ -539,9 +548,17 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             if (cc + 1 < NC16) tmem_ld16(tS + 16 * (cc + 1), nxt);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-              const float2 x = make_float2(cur[2 * i], cur[2 * i + 1]);
+              float2 x = make_float2(cur[2 * i], cur[2 * i + 1]);
+              if (EXTRA && lim < B) {      // masked keys: score 0 (any finite value), weight 0 below
+                if (16 * cc + 2 * i >= lim) x.x = 0.f;
+                if (16 * cc + 2 * i + 1 >= lim) x.y = 0.f;
+              }
               const float2 zz = ffma2(x, f2, off2);
-              const float2 pp = exp2_pair(zz, i);
+              float2 pp = exp2_pair(zz, i);
+              if (EXTRA && lim < B) {
+                if (16 * cc + 2 * i >= lim) pp.x = 0.f;
+                if (16 * cc + 2 * i + 1 >= lim) pp.y = 0.f;
+              }
               z2[i & 1] = ffma2(pp, x, z2[i & 1]);
               a2[i & 1] = fadd2(a2[i & 1], pp);
               cur[2 * i] = pp.x;
@@ -842,7 +859,7 @@ inline cudaError_t launch_kernel_x(const Params& P, int grid, cudaStream_t st) {
 }
 template <typename T, int B, int SB>
 inline cudaError_t launch_kernel(const Params& P, int grid, cudaStream_t st) {
-  if (P.H != 0 || P.lse != nullptr || P.trace != nullptr)
+  if (P.H != 0 || P.lse != nullptr || P.trace != nullptr || P.n_valid != 0)
     return launch_kernel_x<T, B, SB, true>(P, grid, st);
   return launch_kernel_x<T, B, SB, false>(P, grid, st);
 }

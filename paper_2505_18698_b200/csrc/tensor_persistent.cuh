@@ -74,6 +74,7 @@ struct Params {
   long long* trace;    // optional: clock64 stamps [4 CTAs][64 tiles][8 events] (profiling aid)
   int m, BH, T;
   int H;               // 0: Q, K, V, Y are [batch][heads][N][d]; heads: [batch][N][heads][d]
+  int n_valid;         // 0: no padding; else keys b k + i >= n_valid are masked (second generation, SB == B)
   int tiles_per_head, tiles_per_phase;
   int g_begin, g_end;  // tile range of this launch
   int check_deps;
@@ -721,8 +722,11 @@ cudaError_t launch_decoupled(const Params& P, int grid, cudaStream_t st);
 template <typename T, int B, int SB>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int T_steps,
                     int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
-                    bool ws_armed, int H, float* lse) {
-  if ((H != 0 || lse != nullptr) && mode != 0) return 4;   // second-generation kernel only   // only the second-generation kernel reads [batch][N][heads][d]
+                    bool ws_armed, int H, float* lse, int n_valid) {
+  // other layout, row log-sum-exp and the padding mask: second-generation kernel only; the mask
+  // only where a tile row owns a whole key block
+  if ((H != 0 || lse != nullptr || n_valid != 0) && mode != 0) return 4;
+  if (n_valid != 0 && SB != B) return 4;
   const Ws w = ws_layout(ws, BH, N);
   int* counters = (int*)((char*)ws + w.bytes);
   const int m = N / SB;            // = SB on this path
@@ -755,7 +759,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   P.aL = (uint8_t*)w.aL; P.aR = (uint8_t*)w.aR; P.y = (uint8_t*)w.y; P.out = (uint8_t*)Y;
   P.cL = w.cL; P.cR = w.cR; P.status = w.status; P.counters = counters;
   P.trace = trace_buffer();
-  P.m = m; P.BH = BH; P.T = T_steps; P.H = H; P.lse = lse;
+  P.m = m; P.BH = BH; P.T = T_steps; P.H = H; P.lse = lse; P.n_valid = n_valid;
   P.tiles_per_head = m / (kRows / SB);
   P.tiles_per_phase = BH * P.tiles_per_head;
   P.scale = scale;
@@ -801,8 +805,8 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
 
 inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int b, int T,
                   int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
-                  bool ws_armed, int H = 0, float* lse = nullptr) {
-#define MA_TP_ARGS Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed, H, lse
+                  bool ws_armed, int H = 0, float* lse = nullptr, int n_valid = 0) {
+#define MA_TP_ARGS Q, K, V, Y, BH, N, T, dtype, scale, ws, st, launches, mode, ws_armed, H, lse, n_valid
   if (dtype == 1) {
     if (b == 128) return launch_t<__half, 128, 128>(MA_TP_ARGS);
     if (b == 64) return launch_t<__half, 64, 64>(MA_TP_ARGS);

@@ -227,6 +227,20 @@ def test_general_fused_kernel_many_heads_and_agreement_with_the_special_case():
         assert float((a - b_).norm() / b_.norm()) <= 2e-3
 
 
+@pytest.mark.parametrize("name", ["S1", "S2"])
+def test_general_fused_kernel_on_the_profiled_short_workloads(name):
+    """The two extra workloads bench.py can time, at full size, every head against the oracle."""
+    w = wl.EXTRA_WORKLOADS[name]
+    Q, K, V = wl.make_workload_inputs(w)
+    Qd, Kd, Vd = (binding.to_device(x, w.dtype) for x in (Q, K, V))
+    Y = binding.monarch_attn_fwd(Qd, Kd, Vd, w.b, w.T).float().cpu().numpy().astype(np.float64)
+    assert binding.monarch_attn_last_launch_count() == 1
+    ref = mo.monarch_attention(Q, K, V, w.b, w.T)
+    err = (np.linalg.norm((Y - ref).reshape(w.BH, -1), axis=1)
+           / np.linalg.norm(ref.reshape(w.BH, -1), axis=1))
+    assert np.isfinite(Y).all() and err.max() <= TOL[w.dtype], err.max()
+
+
 def test_general_fused_kernel_is_the_default_where_it_applies():
     """AUTO: 16-bit inputs with small blocks take the one-launch kernel, with or without padding
     and in either layout; fp32 inputs and sequences too long for shared memory do not."""
@@ -379,6 +393,8 @@ def test_bounded_wait_runs_out_and_reports_timeout():
     (1000, 32, 64, 2, "bf16"),   # N' = 1024
     (380, 24, 64, 1, "f32"),     # m = 16 != b
     (61, 8, 16, 2, "f32"), (64, 8, 16, 2, "f32"),   # ragged and exact
+    (4040, 64, 64, 2, "bf16"), (4033, 64, 64, 1, "f16"), (4095, 64, 64, 3, "bf16"),   # tensor kernel, N' = 4096
+    (16300, 128, 64, 1, "f16"), (16257, 128, 64, 2, "bf16"),                          # N' = 16384
 ])
 def test_padded_sequences_match_masked_oracle(n_valid, b, d, T, dtype):
     """Post-padded inputs with the key mask of App. C.3: valid rows match the oracle's masked
@@ -389,6 +405,8 @@ def test_padded_sequences_match_masked_oracle(n_valid, b, d, T, dtype):
     V[:, :, n_valid:] = wl.round_to_dtype(np.float32(-50.0), dtype)
     Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))
     Y = binding.monarch_attn_fwd_padded(Qd, Kd, Vd, b, T, n_valid).float().cpu().numpy().astype(np.float64)
+    if b >= 64 and dtype != "f32":      # one persistent launch on the tensor kernel
+        assert binding.monarch_attn_last_launch_count() == 1
     ref = mo.monarch_attention(Q, K, V, b, T, n_valid=n_valid)
     assert np.isfinite(Y[:, :, :n_valid]).all()
     err = rel_err(Y[:, :, :n_valid], ref[:, :, :n_valid])
@@ -448,6 +466,9 @@ def test_batch_seq_head_layout_matches_oracle(N, b, d, T, dtype, batch, heads, p
     (4096, 64, 64, "bf16", binding.MA_PATH_TENSOR, 2e-3),
     (16384, 128, 64, "f16", binding.MA_PATH_TENSOR, 2e-3),
     (1024, 32, 64, "bf16", binding.MA_PATH_TENSOR, 2e-3),
+    (256, 16, 64, "f16", binding.MA_PATH_FUSED_SMALL, 1e-3),
+    (210, 14, 64, "bf16", binding.MA_PATH_FUSED_SMALL, 2e-3),
+    (384, 24, 48, "f16", binding.MA_PATH_AUTO, 1e-3),
 ])
 def test_objective_value_matches_oracle_and_ascends(N, b, d, dtype, path, tol):
     """row_lse summed over a head is f(M^(T)) of Eq. 6 at the returned matrix (oracle: the dense

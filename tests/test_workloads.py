@@ -17,6 +17,14 @@ def test_registry_matches_the_five_configs():
     assert w["C4"].algorithmic_flops() == 19327352832
 
 
+def test_extra_workloads_are_the_short_irregular_shapes():
+    e = wl.EXTRA_WORKLOADS
+    assert not set(e) & set(wl.WORKLOADS)
+    assert (e["S1"].N, e["S1"].b, e["S1"].m, e["S1"].T) == (210, 14, 15, 2)      # 197 tokens padded
+    assert (e["S2"].N, e["S2"].b, e["S2"].m, e["S2"].T) == (384, 24, 16, 1)
+    assert all(w.N == w.m * w.b and w.d == 64 and w.dtype == "f16" for w in e.values())
+
+
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
 def test_inputs_are_seeded_and_representable(dtype):
     a = wl.make_qkv(2, 3, 32, 8, dtype, rank=4, s=2.0, seed=5)
