@@ -275,6 +275,36 @@ def test_general_fused_kernel_is_the_default_where_it_applies():
     assert e.value.code == 4
 
 
+def test_general_fused_kernel_properties_and_output_canaries():
+    """Constant V comes back, zero Q gives the mean of V, stress logits stay finite and convex, the
+    padded variant writes nothing outside Y, on blocks that do not fill a fragment (N = 210, 15 x 14)
+    and on wide blocks (N = 384, 12 x 32)."""
+    for (N, b, dtype) in [(210, 14, "f16"), (384, 32, "bf16")]:
+        Q, K, V = wl.make_qkv(2, 2, N, 64, dtype, 4, 1.0, seed=3)
+        c = wl.round_to_dtype(np.linspace(-2, 2, 64, dtype=np.float32), dtype)
+        Vc = np.broadcast_to(c, V.shape).copy()
+        Y = gpu_forward(Q, K, Vc, dtype, b, 2, binding.MA_PATH_FUSED_SMALL)
+        assert np.abs(Y - Vc).max() <= 2e-2
+        Y = gpu_forward(np.zeros_like(Q), K, V, dtype, b, 2, binding.MA_PATH_FUSED_SMALL)
+        assert np.abs(Y - V.astype(np.float64).mean(axis=2, keepdims=True)).max() <= 1e-2
+        rng = np.random.Generator(np.random.Philox(78))
+        W = rng.standard_normal((8, 64), dtype=np.float32)
+        C = rng.standard_normal((1, 1, N, 8), dtype=np.float32)
+        Qs = wl.round_to_dtype(rng.standard_normal((1, 1, N, 64), dtype=np.float32) + 2.0 * C @ W, dtype)
+        Ks = wl.round_to_dtype(rng.standard_normal((1, 1, N, 64), dtype=np.float32) + 2.0 * C @ W, dtype)
+        Y = gpu_forward(Qs, Ks, V[:1, :1], dtype, b, 3, binding.MA_PATH_FUSED_SMALL)
+        assert np.isfinite(Y).all() and np.abs(Y).max() <= np.abs(V[:1, :1]).max() * 1.02
+        Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))
+        n, pad = Qd.numel(), 4096
+        buf = torch.full((n + 2 * pad,), 7.0, dtype=Qd.dtype, device="cuda")
+        Yv = buf[pad:pad + n].view_as(Qd)
+        binding.monarch_attn_fwd_padded(Qd, Kd, Vd, b, 2, N - 3, Y=Yv)
+        assert binding.monarch_attn_last_launch_count() == 1
+        torch.cuda.synchronize()
+        assert bool((buf[:pad] == 7.0).all()) and bool((buf[pad + n:] == 7.0).all())
+        assert bool(torch.isfinite(Yv.float()).all())
+
+
 # ------------------------------------------------------------------ properties at any size
 @pytest.mark.parametrize("path", [binding.MA_PATH_GENERIC, binding.MA_PATH_AUTO])
 def test_constant_v_and_zero_q(path):
