@@ -56,9 +56,12 @@ typedef enum {
   MA_PATH_FUSED = 5,   /* one CTA per (batch, head), everything in shared memory, one launch:
                           f16/bf16, N = 256, m = b = 16, d = 64 only; kept for comparison (AUTO
                           takes MA_PATH_FUSED_SMALL for this shape too) */
-  MA_PATH_FUSED_SMALL = 7 /* the same idea for any block shape: f16/bf16, m and b <= 32 (m need not
+  MA_PATH_FUSED_SMALL = 7, /* the same idea for any block shape: f16/bf16, m and b <= 32 (m need not
                              equal b), d <= 64 a multiple of 8, N <= 580 for T = 1 and <= 440 for
                              T > 1 (the states of a head must fit shared memory); f16 arithmetic */
+  MA_PATH_TILE_MMA = 8    /* warp-MMA kernels, one launch per half-step, f16 states in the workspace:
+                             f16/bf16, m and b <= 128 (m need not equal b), d <= 128 a multiple of
+                             8; the 16-bit path of the shapes no other tensor-core kernel takes */
 } ma_path;
 
 /* T-step MonarchAttention forward (Eq. 7-10 then Eq. 4) with scale = 1/sqrt(d).
@@ -100,8 +103,8 @@ int monarch_attn_fwd_host(const void* Q_host, const void* K_host, const void* V_
  * half-step has that number for each row anyway and writes it out:
  *   row_lse: DEVICE pointer, [batch][heads][N] floats (natural logarithm), row b l + j of a head;
  *   f of a head = sum of its N entries (the caller reduces; 4-byte aligned).
- * `path`: MA_PATH_AUTO, MA_PATH_TENSOR (second-generation kernel), MA_PATH_FUSED_SMALL or
- * MA_PATH_GENERIC.  Y, workspace
+ * `path`: MA_PATH_AUTO, MA_PATH_TENSOR (second-generation kernel), MA_PATH_FUSED_SMALL,
+ * MA_PATH_TILE_MMA or MA_PATH_GENERIC.  Y, workspace
  * and everything else as monarch_attn_fwd_ex.  Asynchronous on `stream`. */
 int monarch_attn_fwd_objective(const void* Q, const void* K, const void* V, void* Y, int batch,
                                int heads, int N, int d, int b, int T, int dtype,
@@ -113,7 +116,7 @@ int monarch_attn_fwd_objective(const void* Q, const void* K, const void* V, void
  * addressing changes.  Q, K, V, Y: DEVICE pointers to contiguous [batch][N][heads][d] arrays of
  * `dtype`, 16-byte aligned, Y not overlapping an input.  `path`: MA_PATH_AUTO, MA_PATH_TENSOR (the
  * second-generation kernel: the head becomes a column offset in the TMA tensor maps),
- * MA_PATH_FUSED_SMALL or MA_PATH_GENERIC; other paths give MA_ERR_UNSUPPORTED.  Workspace as for monarch_attn_fwd_ex with
+ * MA_PATH_FUSED_SMALL, MA_PATH_TILE_MMA or MA_PATH_GENERIC; other paths give MA_ERR_UNSUPPORTED.  Workspace as for monarch_attn_fwd_ex with
  * the same path (monarch_attn_workspace_bytes does not depend on the layout).  Everything else as
  * monarch_attn_fwd_ex.  Asynchronous on `stream`. */
 int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, int batch, int N,
@@ -134,7 +137,8 @@ int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, 
  * block keeps a valid key; anything else is MA_ERR_SHAPE).  n_valid == N is the unpadded pass.
  * Runs on the general fused kernel (MA_PATH_FUSED_SMALL) where that supports the shape and dtype,
  * on the second-generation tensor kernel (MA_PATH_TENSOR) for f16/bf16 with d = 64 and
- * m = b in {64, 128}, else on the generic kernels (any dtype, m need not equal b).  Workspace: the
+ * m = b in {64, 128}, on the warp-MMA tile kernels (MA_PATH_TILE_MMA) for other 16-bit shapes they
+ * support, else on the generic kernels (any dtype, m need not equal b).  Workspace: the
  * larger of monarch_attn_workspace_bytes() for MA_PATH_TENSOR and MA_PATH_GENERIC serves all three
  * (a return of 0 means that path does not apply).  Asynchronous on `stream`. */
 int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y, int batch,

@@ -22,6 +22,7 @@ MA_PATH_AUTO, MA_PATH_GENERIC, MA_PATH_TENSOR, MA_PATH_TENSOR_PHASED, MA_PATH_TE
 MA_PATH_FUSED = 5
 MA_PATH_TENSOR_CHAINED = 6
 MA_PATH_FUSED_SMALL = 7
+MA_PATH_TILE_MMA = 8
 MA_OK = 0
 
 _TORCH_TO_CODE = {torch.float32: MA_F32, torch.float16: MA_F16, torch.bfloat16: MA_BF16}

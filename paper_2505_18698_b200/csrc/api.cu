@@ -14,6 +14,7 @@
 #include "tensor_decoupled.cuh"
 #include "fused_n256.cuh"
 #include "fused_small.cuh"
+#include "tile_mma.cuh"
 
 namespace ma {
 
@@ -144,14 +145,17 @@ static int resolve_path(const Problem& p, int path) {
     // bf16 with b = 32 and more than two rounds stays on the fp32-state kernels: on the peaky-logit
     // recipe of that shape the 8-bit mantissa of alpha_R (used twice from T = 3 on) costs 4e-2 on
     // the worst head; up to T = 2 the hi + lo alpha_L of the tensor path keeps it under 1e-2.
-    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) &&
-        !(p.b == 32 && p.dtype == MA_BF16 && p.T > 2))
-      return MA_PATH_TENSOR;
+    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) {
+      if (!(p.b == 32 && p.dtype == MA_BF16 && p.T > 2)) return MA_PATH_TENSOR;
+      if (generic_supported(p)) return MA_PATH_GENERIC;
+    }
     if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
+    if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
     if (generic_supported(p)) return MA_PATH_GENERIC;
     return -1;
   }
   if (path == MA_PATH_GENERIC) return generic_supported(p) ? path : -1;
+  if (path == MA_PATH_TILE_MMA) return tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
   if (path == MA_PATH_FUSED_SMALL)
     return fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T) ? path : -1;
   if (path == MA_PATH_FUSED) return fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
@@ -163,8 +167,8 @@ static int resolve_path(const Problem& p, int path) {
 }
 
 // Path choice of the entry points that only the second-generation tensor kernel, the general fused
-// kernel (`with_fused_small`) and the generic kernels serve:
-// AUTO, TENSOR, FUSED_SMALL or GENERIC; -1 if none applies.
+// kernel (`with_fused_small`), the warp-MMA tile kernels and the generic kernels serve:
+// AUTO, TENSOR, FUSED_SMALL, TILE_MMA or GENERIC; -1 if none applies.
 static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused_small = false) {
   if (path == MA_PATH_AUTO || path == MA_PATH_TENSOR) {
     const int r = resolve_path(p, path);
@@ -175,6 +179,10 @@ static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused
     if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
     if (path == MA_PATH_FUSED_SMALL) return -1;
   }
+  if (path == MA_PATH_AUTO || path == MA_PATH_TILE_MMA) {
+    if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
+    if (path == MA_PATH_TILE_MMA) return -1;
+  }
   if ((path == MA_PATH_AUTO || path == MA_PATH_GENERIC) && generic_supported(p)) return MA_PATH_GENERIC;
   return -1;
 }
@@ -182,6 +190,7 @@ static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused
 static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
   if (resolved == MA_PATH_FUSED || resolved == MA_PATH_FUSED_SMALL) return kStatusBytes;   // no states leave the chip
+  if (resolved == MA_PATH_TILE_MMA) return tile::workspace_bytes(p.BH, p.N, p.d);
   if (resolved == MA_PATH_TENSOR_BASIC) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
   if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_PHASED ||
       resolved == MA_PATH_TENSOR_CHAINED)
@@ -232,6 +241,13 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   if (resolved == MA_PATH_FUSED_SMALL) {
     int rc = fsmall::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.m, p.T, p.dtype, scale, p.n_valid, p.H, p.lse, st);
     if (rc == MA_OK) g_last_launches = 1;
+    return rc;
+  }
+  if (resolved == MA_PATH_TILE_MMA) {
+    tile::Args a{Q, K, V, Y, p.lse, p.BH, p.N, p.d, p.b, p.m, p.T, p.n_valid, p.H, scale};
+    int n = 0;
+    int rc = tile::launch(a, p.dtype, ws, st, &n);
+    if (rc == MA_OK) g_last_launches = n;
     return rc;
   }
   int launches = 0;
@@ -304,6 +320,7 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
   int r = -1;
   if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) r = MA_PATH_FUSED_SMALL;
   else if (resolve_path(p, MA_PATH_AUTO) == MA_PATH_TENSOR && p.b != 32) r = MA_PATH_TENSOR;
+  else if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) r = MA_PATH_TILE_MMA;
   else if (generic_supported(p)) r = MA_PATH_GENERIC;
   if (r < 0) return MA_ERR_UNSUPPORTED;
   p.n_valid = n_valid;

@@ -1,0 +1,551 @@
+// Warp-MMA kernels for 16-bit inputs of any block shape: m, b <= 128 (m need not equal b),
+// d <= 128 (a multiple of 8), f16/bf16, key padding mask (App. C.3), either layout.
+//
+// One launch per half-step, one CTA per tile, one warp per 16 score rows.  This is the path of the
+// shapes that neither the tcgen05 kernel (d = 64, m = b in {32, 64, 128}) nor the fused per-head
+// kernel (states of a head in shared memory) takes: e.g. (b, m) = (32, 64) or (64, 128) at
+// N = 2048 / 8192, d = 72, d = 48 with N = 7680 = 60 blocks of 128.  The states alpha_L, alpha_R, y
+// (Sec. 3 'Implementation') are f16 arrays in the workspace, c_L is fp32.
+//
+// Every array (Q, K, V, the states) is stored in the SAME row order, row n = k*b + i of a head, so
+// alpha_R of the first round is Q itself and the permutation between the half-steps (Eq. 9, 10) is
+// the choice of rows a tile gathers: an R tile copies the b consecutive rows of block k, an L tile
+// the m rows (l, j) that sit b rows apart, into shared memory (rows padded by 16 bytes, so 8-row
+// fragment loads are conflict-free).  Arithmetic is f16 x f16 -> fp32 (mma.sync m16n8k16; bf16
+// inputs are converted on the way in), alpha_R is stored divided by c_R with the weights' columns
+// rescaled by powers of two first, as in the fused kernels.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fused_n256.cuh"
+#include "fused_small.cuh"
+
+namespace ma {
+namespace tile {
+
+using fused::Mma;
+using fused::col_sum;
+using fused::ex2;
+using fused::kLn2;
+using fused::kLog2e;
+using fused::ldsm_x4;
+using fused::ldsm_x4_trans;
+using fused::lg2;
+using fused::quad_max;
+using fused::quad_sum;
+using fsmall::stsm_x4;
+
+typedef __half T;
+constexpr int kMaxSmem = 227 * 1024;
+
+// Shared-memory row pitch for DT 16-column steps: the 16 bytes of padding put 8 consecutive rows
+// in 8 different 16-byte bank groups.
+__host__ __device__ constexpr int pitch_of(int dt) { return dt * 32 + 16; }
+
+__device__ __forceinline__ uint4 load16_as_f16(const __half* p) {
+  return __ldg(reinterpret_cast<const uint4*>(p));
+}
+__device__ __forceinline__ uint4 load16_as_f16(const __nv_bfloat16* p) {
+  return fused::to_f16x8(__ldg(reinterpret_cast<const uint4*>(p)), p);
+}
+
+// Rows of head h in Q, K, V, Y: element offset of row 0 and the stride between rows.
+struct HeadRows {
+  size_t base, stride;
+};
+__device__ __forceinline__ HeadRows head_rows(int h, int N, int d, int H) {
+  HeadRows r;
+  r.base = H == 0 ? (size_t)h * N * d : ((size_t)(h / H) * N * H + (h % H)) * d;
+  r.stride = H == 0 ? (size_t)d : (size_t)H * d;
+  return r;
+}
+
+// Copies `rows` rows of d elements (row r at src + r * stride) into a shared tile, zero-filling
+// the columns d .. 16*DT - 1.
+template <typename TSrc, int DT>
+__device__ __forceinline__ void gather_rows(uint8_t* dst, const TSrc* __restrict__ src, size_t stride,
+                                            int rows, int d) {
+  constexpr int kChunks = DT * 2;
+  for (int idx = threadIdx.x; idx < rows * kChunks; idx += blockDim.x) {
+    const int r = idx / kChunks, ch = idx - r * kChunks;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (ch * 8 < d) v = load16_as_f16(src + (size_t)r * stride + ch * 8);
+    *reinterpret_cast<uint4*>(dst + r * pitch_of(DT) + ch * 16) = v;
+  }
+}
+
+__device__ __forceinline__ uint4 store16_from_f16(uint4 v, __half*) { return v; }
+__device__ __forceinline__ uint4 store16_from_f16(uint4 v, __nv_bfloat16* p) { return fused::from_f16x8(v, p); }
+
+// One warp copies its 16 staged rows (first `rows` of them valid) out: row r to dst + r * stride.
+template <typename TDst, int DT>
+__device__ __forceinline__ void scatter_rows16(TDst* __restrict__ dst, size_t stride, const uint8_t* src,
+                                               int rows, int d, int lane) {
+  const int chunks = d >> 3;
+  for (int idx = lane; idx < rows * chunks; idx += 32) {
+    const int r = idx / chunks, ch = idx - r * chunks;
+    const uint4 v = *reinterpret_cast<const uint4*>(src + r * pitch_of(DT) + ch * 16);
+    TDst* gp = dst + (size_t)r * stride + ch * 8;
+    *reinterpret_cast<uint4*>(gp) = store16_from_f16(v, gp);
+  }
+}
+
+// Tiles are allocated with their row count rounded up to 16: a warp stores whole 16-row fragments,
+// and the rows past the block land in that padding.
+__host__ __device__ constexpr int round16(int x) { return (x + 15) & ~15; }
+inline size_t r_smem_bytes(int b, int dt) { return (size_t)4 * round16(b) * pitch_of(dt); }
+inline size_t l_smem_bytes(int m, int cm, int dt) {
+  const size_t tiles = (size_t)3 * round16(m) * pitch_of(dt);  // Q(l,j), alpha_L(k,j), y(k,j)
+  const size_t p_tile = (size_t)round16(m) * (cm * 2 + 16);    // weights for the transposed product
+  const size_t stats = (size_t)(2 * 8 * cm + cm) * 4;          // column max / sum per warp, c_L
+  return tiles + p_tile + stats;
+}
+
+// ---------------------------------------------------------------------------------------------
+// R half-step for key block k of head h (Eq. 7, 9 -> Eq. 10):
+//   Z_R[j,i] = scale * <aR(k,j), K(k,i)>  (alpha_R arrives divided by c_R), R = softmax_i Z_R,
+//   aL(k,j) = sum_i R[j,i] K(k,i), cL(k,j) = sum_i R log R, (last round) y(k,j) = sum_i R[j,i] V(k,i)
+// CB: b rounded up to 32, 64 or 128; DT: 16-column steps over d (4 or 8).
+template <typename TIn, int CB, int DT>
+__global__ void __launch_bounds__(256)
+r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
+              const __half* __restrict__ aR, __half* __restrict__ aL, __half* __restrict__ y,
+              float* __restrict__ cL, int N, int d, int b, float scale, int n_valid, int H, int first,
+              int last) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  constexpr int kPitch = pitch_of(DT);
+  const int k = blockIdx.x, h = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int rb = round16(b);
+  uint8_t* sA = smem;
+  uint8_t* sK = sA + (size_t)rb * kPitch;
+  uint8_t* sV = sK + (size_t)rb * kPitch;
+  uint8_t* sY = sV + (size_t)rb * kPitch;      // staging of y rows on the last round
+  const HeadRows hr = head_rows(h, N, d, H);
+  const size_t st_rows = ((size_t)h * N + (size_t)k * b) * d;    // block k of the state arrays
+
+  if (first) gather_rows<TIn, DT>(sA, Q + hr.base + (size_t)k * b * hr.stride, hr.stride, b, d);
+  else gather_rows<__half, DT>(sA, aR + st_rows, (size_t)d, b, d);
+  gather_rows<TIn, DT>(sK, K + hr.base + (size_t)k * b * hr.stride, hr.stride, b, d);
+  if (last) gather_rows<TIn, DT>(sV, V + hr.base + (size_t)k * b * hr.stride, hr.stride, b, d);
+  __syncthreads();
+
+  const int j0 = 16 * warp;
+  if (j0 >= b) return;
+  const uint32_t sA_u = (uint32_t)__cvta_generic_to_shared(sA), sK_u = (uint32_t)__cvta_generic_to_shared(sK);
+  const uint32_t sV_u = (uint32_t)__cvta_generic_to_shared(sV), sY_u = (uint32_t)__cvta_generic_to_shared(sY);
+  const float fl = scale * kLog2e;
+  const int ilim = min(b, n_valid - k * b);          // valid key columns of this block
+
+  float s[CB / 8][4];
+#pragma unroll
+  for (int nt = 0; nt < CB / 8; ++nt)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
+  {
+    const uint32_t a_u = sA_u + min(j0 + (lane & 7) + ((lane >> 3) & 1) * 8, b - 1) * kPitch + (lane >> 4) * 16;
+#pragma unroll
+    for (int ks = 0; ks < DT; ++ks) {
+      uint32_t a[4];
+      ldsm_x4(a, a_u + ks * 32);
+#pragma unroll
+      for (int cp = 0; cp < CB / 16; ++cp) {
+        if (16 * cp >= b) continue;
+        uint32_t bf[4];
+        ldsm_x4(bf, sK_u + min(16 * cp + (lane & 7) + (lane >> 4) * 8, b - 1) * kPitch + ((lane >> 3) & 1) * 16 + ks * 32);
+        Mma<T>::run(s[2 * cp], a, bf);
+        Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+      }
+    }
+  }
+  // rows j = j0 + g (c0, c1) and j0 + g + 8 (c2, c3); columns i = 8 nt + 2t, +1
+  float inv_s[2];
+#pragma unroll
+  for (int hh = 0; hh < 2; ++hh) {
+    const int j = j0 + g + 8 * hh;
+    float mx = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < CB / 8; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float z = (8 * nt + 2 * t + e < ilim) ? s[nt][2 * hh + e] * fl : -INFINITY;
+        s[nt][2 * hh + e] = z;
+        mx = fmaxf(mx, z);
+      }
+    mx = quad_max(mx);
+    float sum = 0.f, sz = 0.f;
+#pragma unroll
+    for (int nt = 0; nt < CB / 8; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float z = s[nt][2 * hh + e];
+        const float p = ex2(z - mx);                 // 0 for masked columns
+        s[nt][2 * hh + e] = p;
+        sum += p;
+        if (z > -INFINITY) sz = fmaf(p, z, sz);      // 0 log 0 = 0
+      }
+    sum = quad_sum(sum);
+    sz = quad_sum(sz);
+    inv_s[hh] = 1.f / sum;
+    // c_L = sum R log R (natural log): ln2 * (sum p z / sum - max - log2 sum)
+    if (t == 0 && j < b) cL[(size_t)h * N + (size_t)k * b + j] = kLn2 * (sz * inv_s[hh] - mx - lg2(sum));
+  }
+  uint32_t pa[CB / 16][4];
+#pragma unroll
+  for (int kk = 0; kk < CB / 16; ++kk) {
+    pa[kk][0] = Mma<T>::pack(s[2 * kk][0], s[2 * kk][1]);
+    pa[kk][1] = Mma<T>::pack(s[2 * kk][2], s[2 * kk][3]);
+    pa[kk][2] = Mma<T>::pack(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+    pa[kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+  }
+  // second products, two 8-column tiles of v at a time; results staged in this warp's own 16 rows
+  // of the alpha_R tile (dead: only this warp read them) and of the y staging tile
+  const int st_row = (lane & 7) + ((lane >> 3) & 1) * 8, st_nt = (lane >> 4) & 1;
+  const uint32_t stA_u = sA_u + (j0 + st_row) * kPitch + st_nt * 16;
+  const uint32_t stY_u = sY_u + (j0 + st_row) * kPitch + st_nt * 16;
+  __syncwarp();
+#pragma unroll
+  for (int np = 0; np < DT; ++np) {
+    float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    float yv[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+    for (int kk = 0; kk < CB / 16; ++kk) {
+      if (16 * kk >= b) continue;
+      uint32_t bf[4];
+      const uint32_t off = min(16 * kk + (lane & 15), b - 1) * kPitch + (lane >> 4) * 16 + np * 32;
+      ldsm_x4_trans(bf, sK_u + off);
+      Mma<T>::run(o[0], pa[kk], bf);
+      Mma<T>::run(o[1], pa[kk], bf + 2);
+      if (last) {
+        ldsm_x4_trans(bf, sV_u + off);
+        Mma<T>::run(yv[0], pa[kk], bf);
+        Mma<T>::run(yv[1], pa[kk], bf + 2);
+      }
+    }
+    stsm_x4(stA_u + np * 32, Mma<T>::pack(o[0][0] * inv_s[0], o[0][1] * inv_s[0]),
+            Mma<T>::pack(o[0][2] * inv_s[1], o[0][3] * inv_s[1]),
+            Mma<T>::pack(o[1][0] * inv_s[0], o[1][1] * inv_s[0]),
+            Mma<T>::pack(o[1][2] * inv_s[1], o[1][3] * inv_s[1]));
+    if (last)
+      stsm_x4(stY_u + np * 32, Mma<T>::pack(yv[0][0] * inv_s[0], yv[0][1] * inv_s[0]),
+              Mma<T>::pack(yv[0][2] * inv_s[1], yv[0][3] * inv_s[1]),
+              Mma<T>::pack(yv[1][0] * inv_s[0], yv[1][1] * inv_s[0]),
+              Mma<T>::pack(yv[1][2] * inv_s[1], yv[1][3] * inv_s[1]));
+  }
+  __syncwarp();
+  const int rows = min(16, b - j0);
+  scatter_rows16<__half, DT>(aL + st_rows + (size_t)j0 * d, (size_t)d, sA + (size_t)j0 * kPitch, rows, d, lane);
+  if (last)
+    scatter_rows16<__half, DT>(y + st_rows + (size_t)j0 * d, (size_t)d, sY + (size_t)j0 * kPitch, rows, d, lane);
+}
+
+// ---------------------------------------------------------------------------------------------
+// L half-step for in-block position j of head h (Eq. 8, 10 -> Eq. 9 or Eq. 4):
+//   Z_L[l,k] = scale * <Q(l,j), aL(k,j)> - cL(k,j), L = softmax_k Z_L
+//   not final: aR(k,j) = sum_l L[l,k] Q(l,j) / cR(k,j), cR(k,j) = sum_l L[l,k]
+//   final:     Y(l,j) = sum_k L[l,k] y(k,j); optionally the row's log-sum-exp (Eq. 6)
+// CM: m rounded up to 32, 64 or 128.
+template <typename TIn, int CM, int DT>
+__global__ void __launch_bounds__(256)
+l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const float* __restrict__ cL,
+              const __half* __restrict__ y, __half* __restrict__ aR, TIn* __restrict__ Y,
+              float* __restrict__ lse, int N, int d, int b, int m, float scale, int H, int last) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  constexpr int kPitch = pitch_of(DT), kPPitch = CM * 2 + 16;
+  const int j = blockIdx.x, h = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int rm = round16(m);
+  uint8_t* sQ = smem;
+  uint8_t* sL = sQ + (size_t)rm * kPitch;
+  uint8_t* sYt = sL + (size_t)rm * kPitch;
+  uint8_t* sP = sYt + (size_t)rm * kPitch;
+  float* sColMax = reinterpret_cast<float*>(sP + (size_t)rm * kPPitch);
+  float* sColSum = sColMax + 8 * CM;
+  float* sC = sColSum + 8 * CM;
+  const HeadRows hr = head_rows(h, N, d, H);
+  const size_t st_rows = ((size_t)h * N + j) * d;              // row (0, j) of the state arrays
+  const size_t st_stride = (size_t)b * d;                      // rows (k, j), (k+1, j) are b rows apart
+
+  gather_rows<TIn, DT>(sQ, Q + hr.base + (size_t)j * hr.stride, (size_t)b * hr.stride, m, d);
+  gather_rows<__half, DT>(sL, aL + st_rows, st_stride, m, d);
+  if (last) gather_rows<__half, DT>(sYt, y + st_rows, st_stride, m, d);
+  for (int kq = threadIdx.x; kq < m; kq += blockDim.x) sC[kq] = cL[(size_t)h * N + (size_t)kq * b + j] * kLog2e;
+  __syncthreads();
+
+  const int l0 = 16 * warp;
+  const bool active = l0 < m;
+  const uint32_t sQ_u = (uint32_t)__cvta_generic_to_shared(sQ), sL_u = (uint32_t)__cvta_generic_to_shared(sL);
+  const uint32_t sY_u = (uint32_t)__cvta_generic_to_shared(sYt), sP_u = (uint32_t)__cvta_generic_to_shared(sP);
+  const float fl = scale * kLog2e;
+  const int st_row = (lane & 7) + ((lane >> 3) & 1) * 8, st_nt = (lane >> 4) & 1;
+
+  float s[CM / 8][4];
+  float inv_s[2] = {0.f, 0.f};
+  if (active) {
+#pragma unroll
+    for (int nt = 0; nt < CM / 8; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
+    const uint32_t a_u = sQ_u + min(l0 + (lane & 7) + ((lane >> 3) & 1) * 8, m - 1) * kPitch + (lane >> 4) * 16;
+#pragma unroll
+    for (int ks = 0; ks < DT; ++ks) {
+      uint32_t a[4];
+      ldsm_x4(a, a_u + ks * 32);
+#pragma unroll
+      for (int cp = 0; cp < CM / 16; ++cp) {
+        if (16 * cp >= m) continue;
+        uint32_t bf[4];
+        ldsm_x4(bf, sL_u + min(16 * cp + (lane & 7) + (lane >> 4) * 8, m - 1) * kPitch + ((lane >> 3) & 1) * 16 + ks * 32);
+        Mma<T>::run(s[2 * cp], a, bf);
+        Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+      }
+    }
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      float mx = -INFINITY;
+#pragma unroll
+      for (int nt = 0; nt < CM / 8; ++nt)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int kc = 8 * nt + 2 * t + e;
+          const float z = kc < m ? fmaf(s[nt][2 * hh + e], fl, -sC[kc]) : -INFINITY;
+          s[nt][2 * hh + e] = z;
+          mx = fmaxf(mx, z);
+        }
+      mx = quad_max(mx);
+      float sum = 0.f;
+#pragma unroll
+      for (int nt = 0; nt < CM / 8; ++nt)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float p = ex2(s[nt][2 * hh + e] - mx);
+          s[nt][2 * hh + e] = p;
+          sum += p;
+        }
+      sum = quad_sum(sum);
+      inv_s[hh] = 1.f / sum;
+      const int l = l0 + g + 8 * hh;
+      if (last && lse != nullptr && t == 0 && l < m)
+        lse[(size_t)h * N + (size_t)l * b + j] = (mx + log2f(sum)) * kLn2;
+    }
+  }
+
+  if (last) {
+    if (!active) return;
+    // Y(l,j) = sum_k L[l,k] y(k,j): A = weights rows l, B = y rows (k,j) read transposed
+    uint32_t pa[CM / 16][4];
+#pragma unroll
+    for (int kk = 0; kk < CM / 16; ++kk) {
+      pa[kk][0] = Mma<T>::pack(s[2 * kk][0], s[2 * kk][1]);
+      pa[kk][1] = Mma<T>::pack(s[2 * kk][2], s[2 * kk][3]);
+      pa[kk][2] = Mma<T>::pack(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+      pa[kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+    }
+    // staged in this warp's own rows of the Q tile (only this warp read them)
+    const uint32_t st_u = sQ_u + (l0 + st_row) * kPitch + st_nt * 16;
+    __syncwarp();
+#pragma unroll
+    for (int np = 0; np < DT; ++np) {
+      float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+      for (int kk = 0; kk < CM / 16; ++kk) {
+        if (16 * kk >= m) continue;
+        uint32_t bf[4];
+        ldsm_x4_trans(bf, sY_u + min(16 * kk + (lane & 15), m - 1) * kPitch + (lane >> 4) * 16 + np * 32);
+        Mma<T>::run(o[0], pa[kk], bf);
+        Mma<T>::run(o[1], pa[kk], bf + 2);
+      }
+      stsm_x4(st_u + np * 32, Mma<T>::pack(o[0][0] * inv_s[0], o[0][1] * inv_s[0]),
+              Mma<T>::pack(o[0][2] * inv_s[1], o[0][3] * inv_s[1]),
+              Mma<T>::pack(o[1][0] * inv_s[0], o[1][1] * inv_s[0]),
+              Mma<T>::pack(o[1][2] * inv_s[1], o[1][3] * inv_s[1]));
+    }
+    __syncwarp();
+    scatter_rows16<TIn, DT>(Y + hr.base + ((size_t)l0 * b + j) * hr.stride, (size_t)b * hr.stride,
+                            sQ + (size_t)l0 * kPitch, min(16, m - l0), d, lane);
+    return;
+  }
+
+  // ---- not final: alpha_R(k,j) = sum_l L[l,k] Q(l,j) / c_R(k,j).  The contraction runs over the
+  // rows of the weights, which are spread over the warps: the normalised weights go through a
+  // shared tile.  Before rounding to 16 bits every column k is multiplied by a power of two g_k
+  // (the result is invariant) so that its largest weight is near 1 however small c_R is, and c_R
+  // is summed over the weights AS ROUNDED, so that numerator and denominator see the same numbers.
+  if (active) {
+#pragma unroll
+    for (int nt = 0; nt < CM / 8; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float p0 = (l0 + g < m) ? s[nt][e] * inv_s[0] : 0.f;          // rows past the block: 0
+        const float p1 = (l0 + g + 8 < m) ? s[nt][2 + e] * inv_s[1] : 0.f;
+        s[nt][e] = p0;
+        s[nt][2 + e] = p1;
+        float cm = fmaxf(p0, p1);
+        cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 4));
+        cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 8));
+        cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 16));
+        if (g == 0) sColMax[warp * CM + 8 * nt + 2 * t + e] = cm;
+      }
+  }
+  __syncthreads();
+  const int row_warps = (m + 15) >> 4;       // warps that hold weight rows
+  if (active) {
+    const uint32_t st_u = sP_u + (l0 + st_row) * kPPitch + st_nt * 16;
+#pragma unroll
+    for (int np = 0; np < CM / 16; ++np) {
+      uint32_t u[2][2];
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const int nt = 2 * np + q;
+        float gk[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          float cm = 0.f;
+          for (int w = 0; w < row_warps; ++w) cm = fmaxf(cm, sColMax[w * CM + 8 * nt + 2 * t + e]);
+          gk[e] = cm > 0.f ? __uint_as_float((253u << 23) - (__float_as_uint(cm) & 0x7f800000u)) : 0.f;
+        }
+        u[q][0] = Mma<T>::pack(s[nt][0] * gk[0], s[nt][1] * gk[1]);
+        u[q][1] = Mma<T>::pack(s[nt][2] * gk[0], s[nt][3] * gk[1]);
+        const float2 f0 = Mma<T>::unpack(u[q][0]), f1 = Mma<T>::unpack(u[q][1]);
+        const float c0 = col_sum(f0.x + f1.x), c1 = col_sum(f0.y + f1.y);
+        if (g == 0) {
+          sColSum[warp * CM + 8 * nt + 2 * t] = c0;
+          sColSum[warp * CM + 8 * nt + 2 * t + 1] = c1;
+        }
+      }
+      stsm_x4(st_u + np * 32, u[0][0], u[0][1], u[1][0], u[1][1]);
+    }
+  }
+  __syncthreads();
+  // warp kt forms rows k = 16 kt .. 16 kt + 15 of alpha_R
+  const int k0 = 16 * warp;
+  if (k0 >= m) return;
+  float ic[2];
+#pragma unroll
+  for (int hh = 0; hh < 2; ++hh) {
+    const int kq = min(k0 + g + 8 * hh, CM - 1);
+    float cr = 0.f;
+    for (int w = 0; w < row_warps; ++w) cr += sColSum[w * CM + kq];
+    ic[hh] = cr > 1e-30f ? 1.f / cr : 0.f;     // c_R underflow: alpha_R = 0, a uniform row next
+  }
+  // staged in this warp's rows k of the alpha_L tile (every warp is done reading it)
+  const uint32_t st_u = sL_u + (k0 + st_row) * kPitch + st_nt * 16;
+  // A = weights transposed: element (k, l) from the tile stored [l][k] (its rows l >= m are the
+  // zero rows the owning warp stored, so a partly filled 16-row step contributes nothing)
+  const uint32_t pt_u = sP_u + ((lane & 7) + ((lane >> 4) & 1) * 8) * kPPitch + (k0 + ((lane >> 3) & 1) * 8) * 2;
+#pragma unroll
+  for (int np = 0; np < DT; ++np) {
+    float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+    for (int ls = 0; ls < CM / 16; ++ls) {
+      if (16 * ls >= m) continue;
+      uint32_t a[4], bf[4];
+      ldsm_x4_trans(a, pt_u + 16 * ls * kPPitch);
+      ldsm_x4_trans(bf, sQ_u + min(16 * ls + (lane & 15), m - 1) * kPitch + (lane >> 4) * 16 + np * 32);
+      Mma<T>::run(o[0], a, bf);
+      Mma<T>::run(o[1], a, bf + 2);
+    }
+    stsm_x4(st_u + np * 32, Mma<T>::pack(o[0][0] * ic[0], o[0][1] * ic[0]),
+            Mma<T>::pack(o[0][2] * ic[1], o[0][3] * ic[1]), Mma<T>::pack(o[1][0] * ic[0], o[1][1] * ic[0]),
+            Mma<T>::pack(o[1][2] * ic[1], o[1][3] * ic[1]));
+  }
+  __syncwarp();
+  scatter_rows16<__half, DT>(aR + st_rows + (size_t)k0 * st_stride, st_stride, sL + (size_t)k0 * kPitch,
+                             min(16, m - k0), d, lane);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side: workspace layout and launches.
+inline bool supported(int N, int d, int b, int m, int dtype, int BH) {
+  (void)N;
+  if (dtype != 1 && dtype != 2) return false;
+  if (d % 8 != 0 || d > 128 || b > 128 || m > 128 || BH > 65535) return false;
+  const int dt = d <= 64 ? 4 : 8, cm = m <= 32 ? 32 : (m <= 64 ? 64 : 128);
+  return r_smem_bytes(b, dt) <= (size_t)kMaxSmem && l_smem_bytes(m, cm, dt) <= (size_t)kMaxSmem;
+}
+
+struct Ws {
+  __half *aL, *aR, *y;
+  float* cL;
+  size_t bytes;
+};
+inline Ws ws_layout(void* base, int BH, int N, int d) {
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  Ws w;
+  char* c = (char*)base;
+  size_t off = 256;                                   // status block (unused: no device-side waits)
+  const size_t big = up((size_t)BH * N * d * 2);
+  w.aL = (__half*)(c + off); off += big;
+  w.aR = (__half*)(c + off); off += big;
+  w.y = (__half*)(c + off); off += big;
+  w.cL = (float*)(c + off); off += up((size_t)BH * N * 4);
+  w.bytes = off;
+  return w;
+}
+inline size_t workspace_bytes(int BH, int N, int d) { return ws_layout(nullptr, BH, N, d).bytes; }
+
+struct Args {
+  const void *Q, *K, *V;
+  void* Y;
+  float* lse;
+  int BH, N, d, b, m, T, n_valid, H;
+  float scale;
+};
+
+template <typename TIn, int CB, int DT>
+inline int launch_r(const Args& a, const Ws& w, bool first, bool last, cudaStream_t st) {
+  auto kern = r_tile_kernel<TIn, CB, DT>;
+  const size_t smem = r_smem_bytes(a.b, DT);
+  if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return 7;
+  kern<<<dim3(a.m, a.BH), 32 * ((a.b + 15) / 16), smem, st>>>((const TIn*)a.Q, (const TIn*)a.K, (const TIn*)a.V, w.aR,
+                                                          w.aL, w.y, w.cL, a.N, a.d, a.b, a.scale, a.n_valid,
+                                                          a.H, first ? 1 : 0, last ? 1 : 0);
+  return 0;
+}
+template <typename TIn, int CM, int DT>
+inline int launch_l(const Args& a, const Ws& w, bool last, cudaStream_t st) {
+  auto kern = l_tile_kernel<TIn, CM, DT>;
+  const size_t smem = l_smem_bytes(a.m, CM, DT);
+  if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return 7;
+  kern<<<dim3(a.b, a.BH), 32 * ((a.m + 15) / 16), smem, st>>>((const TIn*)a.Q, w.aL, w.cL, w.y, w.aR, (TIn*)a.Y,
+                                                          last ? a.lse : nullptr, a.N, a.d, a.b, a.m, a.scale,
+                                                          a.H, last ? 1 : 0);
+  return 0;
+}
+
+template <typename TIn, int DT>
+inline int launch_td(const Args& a, void* ws, cudaStream_t st, int* launches) {
+  const Ws w = ws_layout(ws, a.BH, a.N, a.d);
+  int n = 0;
+  for (int t = 1; t <= a.T; ++t) {
+    const bool first = t == 1, last = t == a.T;
+    int rc;
+    if (a.b <= 32) rc = launch_r<TIn, 32, DT>(a, w, first, last, st);
+    else if (a.b <= 64) rc = launch_r<TIn, 64, DT>(a, w, first, last, st);
+    else rc = launch_r<TIn, 128, DT>(a, w, first, last, st);
+    if (rc != 0) return rc;
+    if (a.m <= 32) rc = launch_l<TIn, 32, DT>(a, w, last, st);
+    else if (a.m <= 64) rc = launch_l<TIn, 64, DT>(a, w, last, st);
+    else rc = launch_l<TIn, 128, DT>(a, w, last, st);
+    if (rc != 0) return rc;
+    n += 2;
+  }
+  if (cudaGetLastError() != cudaSuccess) return 7;
+  *launches = n;
+  return 0;
+}
+
+inline int launch(const Args& a, int dtype, void* ws, cudaStream_t st, int* launches) {
+  if (dtype == 1)
+    return a.d <= 64 ? launch_td<__half, 4>(a, ws, st, launches) : launch_td<__half, 8>(a, ws, st, launches);
+  return a.d <= 64 ? launch_td<__nv_bfloat16, 4>(a, ws, st, launches)
+                   : launch_td<__nv_bfloat16, 8>(a, ws, st, launches);
+}
+
+}  // namespace tile
+}  // namespace ma

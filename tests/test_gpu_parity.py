@@ -305,6 +305,58 @@ def test_general_fused_kernel_properties_and_output_canaries():
         assert bool(torch.isfinite(Yv.float()).all())
 
 
+# ------------------------------------------------------------------ warp-MMA tile kernels
+@pytest.mark.parametrize("N,b,d,T,dtype", [
+    (60, 6, 8, 2, "f16"), (210, 14, 64, 2, "f16"),          # tiles smaller than one fragment
+    (256, 16, 72, 3, "f16"),                                # DiT: d = 72 (zero-padded to 128 columns)
+    (384, 48, 64, 1, "f16"), (384, 96, 64, 1, "bf16"), (384, 128, 64, 2, "f16"),   # RoBERTa: m = 8, 4, 3
+    (2048, 32, 64, 1, "bf16"), (2048, 64, 64, 2, "f16"),    # BART: (b, m) = (32, 64) and the reverse
+    (8192, 64, 64, 1, "bf16"),                              # BART: (b, m) = (64, 128)
+    (7680, 128, 48, 2, "f16"),                              # GPS: 60 blocks of 128, d = 48
+    (4096, 64, 128, 2, "f16"), (2000, 100, 40, 2, "bf16"), (1089, 33, 24, 3, "f16"),
+])
+def test_tile_mma_path_matches_oracle(N, b, d, T, dtype):
+    """Any m, b <= 128 and d <= 128 on tensor cores: 2T launches, f16 states in the workspace."""
+    rank, s = (min(8, d), 1.0) if T <= 2 else (min(16, d), 1.5)
+    check(1, 3, N, d, b, T, dtype, rank=rank, s=s, seed=N + T, path=binding.MA_PATH_TILE_MMA)
+    assert binding.monarch_attn_last_launch_count() == 2 * T
+
+
+def test_tile_mma_path_is_the_16_bit_default_where_no_other_tensor_core_kernel_applies():
+    Q, K, V = wl.make_qkv(2, 3, 2048, 64, "bf16", 8, 1.0, seed=4)
+    Qd, Kd, Vd = (binding.to_device(x, "bf16") for x in (Q, K, V))
+    a = binding.monarch_attn_fwd(Qd, Kd, Vd, 32, 2)                    # (b, m) = (32, 64)
+    assert binding.monarch_attn_last_launch_count() == 4
+    e_ = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 32, 2, path=binding.MA_PATH_TILE_MMA)
+    assert torch.equal(a, e_)
+    # other layout and the objective value on the same kernels
+    Qs, Ks, Vs = (x.transpose(1, 2).contiguous() for x in (Qd, Kd, Vd))
+    c = binding.monarch_attn_fwd_bshd(Qs, Ks, Vs, 32, 2)
+    assert binding.monarch_attn_last_launch_count() == 4
+    assert torch.equal(c.transpose(1, 2), a)
+    Y, lse = binding.monarch_attn_fwd_objective(Qd, Kd, Vd, 32, 2)
+    assert binding.monarch_attn_last_launch_count() == 4 and torch.equal(Y, a)
+    scale = 1.0 / np.sqrt(64)
+    f_gpu = lse.double().sum(-1).cpu().numpy()
+    for h in range(3):
+        _, L, R = mo.monarch_attention_head(Q[0, h], K[0, h], V[0, h], 32, 2, return_factors=True)
+        f_ref = mo.objective_factored(L, R, Q[0, h], K[0, h], scale)
+        assert abs(f_gpu[0, h] - f_ref) <= 2e-3 * abs(f_ref)
+    # padding: N = 7600 -> 60 blocks of 128, d = 48
+    Q, K, V = wl.make_qkv(1, 2, 7680, 48, "f16", 8, 1.0, seed=9)
+    K[:, :, 7600:] = 3.0
+    V[:, :, 7600:] = -50.0
+    x = [binding.to_device(t_, "f16") for t_ in (Q, K, V)]
+    Yp = binding.monarch_attn_fwd_padded(*x, 128, 2, 7600).float().cpu().numpy().astype(np.float64)
+    assert binding.monarch_attn_last_launch_count() == 4
+    ref = mo.monarch_attention(Q, K, V, 128, 2, n_valid=7600)
+    assert rel_err(Yp[:, :, :7600], ref[:, :, :7600]) <= TOL["f16"]
+    # fp32 inputs never take a 16-bit path
+    with pytest.raises(binding.MonarchAttnError) as e:
+        binding.monarch_attn_fwd_ex(*(t_.float() for t_ in x), 128, 2, path=binding.MA_PATH_TILE_MMA)
+    assert e.value.code == 4
+
+
 # ------------------------------------------------------------------ properties at any size
 @pytest.mark.parametrize("path", [binding.MA_PATH_GENERIC, binding.MA_PATH_AUTO])
 def test_constant_v_and_zero_q(path):
