@@ -45,13 +45,6 @@ constexpr int kMaxSmem = 227 * 1024;
 // in 8 different 16-byte bank groups.
 __host__ __device__ constexpr int pitch_of(int dt) { return dt * 32 + 16; }
 
-__device__ __forceinline__ uint4 load16_as_f16(const __half* p) {
-  return __ldg(reinterpret_cast<const uint4*>(p));
-}
-__device__ __forceinline__ uint4 load16_as_f16(const __nv_bfloat16* p) {
-  return fused::to_f16x8(__ldg(reinterpret_cast<const uint4*>(p)), p);
-}
-
 // Rows of head h in Q, K, V, Y: element offset of row 0 and the stride between rows.
 struct HeadRows {
   size_t base, stride;
@@ -63,17 +56,39 @@ __device__ __forceinline__ HeadRows head_rows(int h, int N, int d, int H) {
   return r;
 }
 
-// Copies `rows` rows of d elements (row r at src + r * stride) into a shared tile, zero-filling
-// the columns d .. 16*DT - 1.
+// Starts the copy of `rows` rows of d 16-bit elements (row r at src + r * stride) into a shared
+// tile (asynchronous 16-byte copies of the raw values; columns d .. 16*DT - 1 are zero-filled).
+// After gather_wait(), convert_rows() turns bf16 tiles into f16 in place: every thread converts
+// exactly the chunks it copied, so no barrier is needed in between.
 template <typename TSrc, int DT>
 __device__ __forceinline__ void gather_rows(uint8_t* dst, const TSrc* __restrict__ src, size_t stride,
                                             int rows, int d) {
   constexpr int kChunks = DT * 2;
+  const uint32_t dst_u = (uint32_t)__cvta_generic_to_shared(dst);
   for (int idx = threadIdx.x; idx < rows * kChunks; idx += blockDim.x) {
     const int r = idx / kChunks, ch = idx - r * kChunks;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (ch * 8 < d) v = load16_as_f16(src + (size_t)r * stride + ch * 8);
-    *reinterpret_cast<uint4*>(dst + r * pitch_of(DT) + ch * 16) = v;
+    const uint32_t off = r * pitch_of(DT) + ch * 16;
+    if (ch * 8 < d)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_u + off), "l"(src + (size_t)r * stride + ch * 8)
+                   : "memory");
+    else
+      *reinterpret_cast<uint4*>(dst + off) = make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+__device__ __forceinline__ void gather_wait() {
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+template <typename TSrc, int DT>
+__device__ __forceinline__ void convert_rows(uint8_t* dst, int rows, int d) {
+  if (!Mma<TSrc>::is_f16) {
+    constexpr int kChunks = DT * 2;
+    for (int idx = threadIdx.x; idx < rows * kChunks; idx += blockDim.x) {
+      const int r = idx / kChunks, ch = idx - r * kChunks;
+      if (ch * 8 >= d) continue;
+      uint4* p = reinterpret_cast<uint4*>(dst + r * pitch_of(DT) + ch * 16);
+      *p = fused::to_f16x8(*p, (const TSrc*)nullptr);
+    }
   }
 }
 
@@ -131,6 +146,10 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
   else gather_rows<__half, DT>(sA, aR + st_rows, (size_t)d, b, d);
   gather_rows<TIn, DT>(sK, K + hr.base + (size_t)k * b * hr.stride, hr.stride, b, d);
   if (last) gather_rows<TIn, DT>(sV, V + hr.base + (size_t)k * b * hr.stride, hr.stride, b, d);
+  gather_wait();
+  if (first) convert_rows<TIn, DT>(sA, b, d);
+  convert_rows<TIn, DT>(sK, b, d);
+  if (last) convert_rows<TIn, DT>(sV, b, d);
   __syncthreads();
 
   const int j0 = 16 * warp;
@@ -273,6 +292,8 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
   gather_rows<__half, DT>(sL, aL + st_rows, st_stride, m, d);
   if (last) gather_rows<__half, DT>(sYt, y + st_rows, st_stride, m, d);
   for (int kq = threadIdx.x; kq < m; kq += blockDim.x) sC[kq] = cL[(size_t)h * N + (size_t)kq * b + j] * kLog2e;
+  gather_wait();
+  convert_rows<TIn, DT>(sQ, m, d);
   __syncthreads();
 
   const int l0 = 16 * warp;

@@ -95,6 +95,10 @@ EXTRA_WORKLOADS = {
                    "ViT-B sequence (197 padded to 15 blocks of 14), two rounds"),
     "S2": Workload("S2", 32, 12, 384, 64, 24, 1, "f16", 8, 1.0, 6,
                    "RoBERTa sequence 384 as 16 blocks of 24, one round"),
+    "S3": Workload("S3", 2, 16, 8192, 64, 64, 1, "bf16", 8, 1.0, 7,
+                   "BART sequence 8192 as 128 blocks of 64 (m != b), one round"),
+    "S4": Workload("S4", 1, 8, 7680, 48, 128, 2, "f16", 8, 1.0, 8,
+                   "graph transformer: 7600 nodes padded to 60 blocks of 128, d = 48, two rounds"),
 }
 
 

@@ -22,7 +22,9 @@ def test_extra_workloads_are_the_short_irregular_shapes():
     assert not set(e) & set(wl.WORKLOADS)
     assert (e["S1"].N, e["S1"].b, e["S1"].m, e["S1"].T) == (210, 14, 15, 2)      # 197 tokens padded
     assert (e["S2"].N, e["S2"].b, e["S2"].m, e["S2"].T) == (384, 24, 16, 1)
-    assert all(w.N == w.m * w.b and w.d == 64 and w.dtype == "f16" for w in e.values())
+    assert (e["S3"].N, e["S3"].b, e["S3"].m, e["S3"].T) == (8192, 64, 128, 1)
+    assert (e["S4"].N, e["S4"].b, e["S4"].m, e["S4"].d) == (7680, 128, 60, 48)
+    assert all(w.N == w.m * w.b and w.dtype in ("f16", "bf16") for w in e.values())
 
 
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
