@@ -225,7 +225,7 @@ def roofline(w, ms, peaks, which):
     ach = w.algorithmic_bytes() / (ms * 1e-3) / 1e9
     return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(w.name), "of": which,
-            "scope": "one step (one launch on the tensor and fused paths, 2T on the generic path)"}
+            "scope": "one step (one launch on the tcgen05 and fused paths, 2T on the tile and generic paths)"}
 
 
 def sdpa_ms(w, torch, sets, iters=5):

@@ -40,6 +40,7 @@ using fsmall::stsm_x4;
 
 typedef __half T;
 constexpr int kMaxSmem = 227 * 1024;
+constexpr float kMasked = -1e30f;   // logit of a masked column: exp2(kMasked - max) == 0
 
 // Shared-memory row pitch for DT 16-column steps: the 16 bytes of padding put 8 consecutive rows
 // in 8 different 16-byte bank groups.
@@ -64,15 +65,16 @@ template <typename TSrc, int DT>
 __device__ __forceinline__ void gather_rows(uint8_t* dst, const TSrc* __restrict__ src, size_t stride,
                                             int rows, int d) {
   constexpr int kChunks = DT * 2;
-  const uint32_t dst_u = (uint32_t)__cvta_generic_to_shared(dst);
-  for (int idx = threadIdx.x; idx < rows * kChunks; idx += blockDim.x) {
-    const int r = idx / kChunks, ch = idx - r * kChunks;
-    const uint32_t off = r * pitch_of(DT) + ch * 16;
-    if (ch * 8 < d)
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_u + off), "l"(src + (size_t)r * stride + ch * 8)
-                   : "memory");
-    else
-      *reinterpret_cast<uint4*>(dst + off) = make_uint4(0u, 0u, 0u, 0u);
+  // a thread keeps its 16-byte column and walks down the rows (blockDim.x is a multiple of 32)
+  const int ch = threadIdx.x % kChunks, rstep = blockDim.x / kChunks;
+  uint32_t dst_u = (uint32_t)__cvta_generic_to_shared(dst) + (threadIdx.x / kChunks) * pitch_of(DT) + ch * 16;
+  if (ch * 8 < d) {
+    const TSrc* p = src + (size_t)(threadIdx.x / kChunks) * stride + ch * 8;
+    for (int r = threadIdx.x / kChunks; r < rows; r += rstep, p += (size_t)rstep * stride, dst_u += rstep * pitch_of(DT))
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_u), "l"(p) : "memory");
+  } else {
+    for (int r = threadIdx.x / kChunks; r < rows; r += rstep)
+      *reinterpret_cast<uint4*>(dst + r * pitch_of(DT) + ch * 16) = make_uint4(0u, 0u, 0u, 0u);
   }
 }
 __device__ __forceinline__ void gather_wait() {
@@ -83,12 +85,12 @@ template <typename TSrc, int DT>
 __device__ __forceinline__ void convert_rows(uint8_t* dst, int rows, int d) {
   if (!Mma<TSrc>::is_f16) {
     constexpr int kChunks = DT * 2;
-    for (int idx = threadIdx.x; idx < rows * kChunks; idx += blockDim.x) {
-      const int r = idx / kChunks, ch = idx - r * kChunks;
-      if (ch * 8 >= d) continue;
-      uint4* p = reinterpret_cast<uint4*>(dst + r * pitch_of(DT) + ch * 16);
-      *p = fused::to_f16x8(*p, (const TSrc*)nullptr);
-    }
+    const int ch = threadIdx.x % kChunks, rstep = blockDim.x / kChunks;
+    if (ch * 8 < d)
+      for (int r = threadIdx.x / kChunks; r < rows; r += rstep) {
+        uint4* p = reinterpret_cast<uint4*>(dst + r * pitch_of(DT) + ch * 16);
+        *p = fused::to_f16x8(*p, (const TSrc*)nullptr);
+      }
   }
 }
 
@@ -99,9 +101,10 @@ __device__ __forceinline__ uint4 store16_from_f16(uint4 v, __nv_bfloat16* p) { r
 template <typename TDst, int DT>
 __device__ __forceinline__ void scatter_rows16(TDst* __restrict__ dst, size_t stride, const uint8_t* src,
                                                int rows, int d, int lane) {
-  const int chunks = d >> 3;
-  for (int idx = lane; idx < rows * chunks; idx += 32) {
-    const int r = idx / chunks, ch = idx - r * chunks;
+  constexpr int kChunks = DT * 2;              // a lane keeps its 16-byte column and walks down the rows
+  const int ch = lane % kChunks;
+  if (ch * 8 >= d) return;
+  for (int r = lane / kChunks; r < rows; r += 32 / kChunks) {
     const uint4 v = *reinterpret_cast<const uint4*>(src + r * pitch_of(DT) + ch * 16);
     TDst* gp = dst + (size_t)r * stride + ch * 8;
     *reinterpret_cast<uint4*>(gp) = store16_from_f16(v, gp);
@@ -166,6 +169,10 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
     for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
   {
     const uint32_t a_u = sA_u + min(j0 + (lane & 7) + ((lane >> 3) & 1) * 8, b - 1) * kPitch + (lane >> 4) * 16;
+    uint32_t b_u[CB / 16];
+#pragma unroll
+    for (int cp = 0; cp < CB / 16; ++cp)
+      b_u[cp] = sK_u + min(16 * cp + (lane & 7) + (lane >> 4) * 8, b - 1) * kPitch + ((lane >> 3) & 1) * 16;
 #pragma unroll
     for (int ks = 0; ks < DT; ++ks) {
       uint32_t a[4];
@@ -174,7 +181,7 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
       for (int cp = 0; cp < CB / 16; ++cp) {
         if (16 * cp >= b) continue;
         uint32_t bf[4];
-        ldsm_x4(bf, sK_u + min(16 * cp + (lane & 7) + (lane >> 4) * 8, b - 1) * kPitch + ((lane >> 3) & 1) * 16 + ks * 32);
+        ldsm_x4(bf, b_u[cp] + ks * 32);
         Mma<T>::run(s[2 * cp], a, bf);
         Mma<T>::run(s[2 * cp + 1], a, bf + 2);
       }
@@ -185,12 +192,14 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
 #pragma unroll
   for (int hh = 0; hh < 2; ++hh) {
     const int j = j0 + g + 8 * hh;
-    float mx = -INFINITY;
+    // masked columns (past the block, or past n_valid: App. C.3) get a huge negative FINITE
+    // logit: their weight is exactly 0 and 0 * z stays 0 in the entropy sum (0 log 0 = 0)
+    float mx = kMasked;
 #pragma unroll
     for (int nt = 0; nt < CB / 8; ++nt)
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        const float z = (8 * nt + 2 * t + e < ilim) ? s[nt][2 * hh + e] * fl : -INFINITY;
+        const float z = (8 * nt + 2 * t + e < ilim) ? s[nt][2 * hh + e] * fl : kMasked;
         s[nt][2 * hh + e] = z;
         mx = fmaxf(mx, z);
       }
@@ -204,7 +213,7 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
         const float p = ex2(z - mx);                 // 0 for masked columns
         s[nt][2 * hh + e] = p;
         sum += p;
-        if (z > -INFINITY) sz = fmaf(p, z, sz);      // 0 log 0 = 0
+        sz = fmaf(p, z, sz);
       }
     sum = quad_sum(sum);
     sz = quad_sum(sz);
@@ -226,6 +235,9 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
   const uint32_t stA_u = sA_u + (j0 + st_row) * kPitch + st_nt * 16;
   const uint32_t stY_u = sY_u + (j0 + st_row) * kPitch + st_nt * 16;
   __syncwarp();
+  uint32_t v_off[CB / 16];
+#pragma unroll
+  for (int kk = 0; kk < CB / 16; ++kk) v_off[kk] = min(16 * kk + (lane & 15), b - 1) * kPitch + (lane >> 4) * 16;
 #pragma unroll
   for (int np = 0; np < DT; ++np) {
     float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -234,7 +246,7 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
     for (int kk = 0; kk < CB / 16; ++kk) {
       if (16 * kk >= b) continue;
       uint32_t bf[4];
-      const uint32_t off = min(16 * kk + (lane & 15), b - 1) * kPitch + (lane >> 4) * 16 + np * 32;
+      const uint32_t off = v_off[kk] + np * 32;
       ldsm_x4_trans(bf, sK_u + off);
       Mma<T>::run(o[0], pa[kk], bf);
       Mma<T>::run(o[1], pa[kk], bf + 2);
@@ -311,6 +323,10 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
 #pragma unroll
       for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
     const uint32_t a_u = sQ_u + min(l0 + (lane & 7) + ((lane >> 3) & 1) * 8, m - 1) * kPitch + (lane >> 4) * 16;
+    uint32_t b_u[CM / 16];
+#pragma unroll
+    for (int cp = 0; cp < CM / 16; ++cp)
+      b_u[cp] = sL_u + min(16 * cp + (lane & 7) + (lane >> 4) * 8, m - 1) * kPitch + ((lane >> 3) & 1) * 16;
 #pragma unroll
     for (int ks = 0; ks < DT; ++ks) {
       uint32_t a[4];
@@ -319,20 +335,20 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
       for (int cp = 0; cp < CM / 16; ++cp) {
         if (16 * cp >= m) continue;
         uint32_t bf[4];
-        ldsm_x4(bf, sL_u + min(16 * cp + (lane & 7) + (lane >> 4) * 8, m - 1) * kPitch + ((lane >> 3) & 1) * 16 + ks * 32);
+        ldsm_x4(bf, b_u[cp] + ks * 32);
         Mma<T>::run(s[2 * cp], a, bf);
         Mma<T>::run(s[2 * cp + 1], a, bf + 2);
       }
     }
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
-      float mx = -INFINITY;
+      float mx = kMasked;
 #pragma unroll
       for (int nt = 0; nt < CM / 8; ++nt)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const int kc = 8 * nt + 2 * t + e;
-          const float z = kc < m ? fmaf(s[nt][2 * hh + e], fl, -sC[kc]) : -INFINITY;
+          const float z = kc < m ? fmaf(s[nt][2 * hh + e], fl, -sC[kc]) : kMasked;
           s[nt][2 * hh + e] = z;
           mx = fmaxf(mx, z);
         }
