@@ -88,7 +88,11 @@ int monarch_attn_fwd_ex(const void* Q, const void* K, const void* V, void* Y,
 
 /* End-to-end variant: Q, K, V, Y are HOST pointers (pinned memory gives asynchronous copies).
  * Copies Q, K, V to device staging buffers owned by the library, runs monarch_attn_fwd, copies Y
- * back, all on `stream`; does not synchronise.  Grows the staging buffers on demand. */
+ * back; does not synchronise.  The (batch, head) units are independent (Sec. 3), so the call is
+ * cut into four chunks of units (measured best of 1-8 on C2 and C5): a chunk's kernels and the copy of its result run on two
+ * streams owned by the library while the next chunk's inputs come in on `stream` (fork and join by
+ * events, so work queued on `stream` after the call still sees Y_host complete).  Grows the staging buffers on
+ * demand. */
 int monarch_attn_fwd_host(const void* Q_host, const void* K_host, const void* V_host, void* Y_host,
                           int batch, int heads, int N, int d, int b, int T,
                           int dtype, void* stream);
@@ -190,12 +194,14 @@ int monarch_attn_last_launch_count(void);
  * the buffer stays owned by the caller. */
 int monarch_attn_set_trace_buffer(void* device_buffer, size_t bytes);
 
-/* Test knobs of the persistent tensor path (process-wide; not for production use).
+/* Test and tuning knobs (process-wide; not for production use).  Knobs 1 and 2 belong to the
+ * persistent tensor path:
  *   knob 1: bound, in SM clocks, of every device-side wait (value <= 0 restores the default 2e9);
  *   knob 2: non-zero leaves the first half-step out of later single-launch runs, so that the
  *           dependency waits of the second half-step can never be satisfied.  Together they let a
  *           test watch a wait run out: the kernel ends by itself, results are garbage, and
- *           monarch_attn_device_status reports MA_ERR_TIMEOUT.  Nothing faults or hangs. */
+ *           monarch_attn_device_status reports MA_ERR_TIMEOUT.  Nothing faults or hangs.
+ *   knob 3: number of chunks monarch_attn_fwd_host cuts a call into (1..8, default 4). */
 int monarch_attn_debug_knob(int knob, long long value);
 
 /* Static, NUL-terminated description of an ma_status code. */

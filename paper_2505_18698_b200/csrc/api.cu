@@ -206,7 +206,15 @@ struct DeviceBuffers {
   long long armed_key = -1;   // problem whose status block / counters the workspace is armed for
   void* stage = nullptr;   // Q, K, V, Y staging for the host entry point
   size_t stage_bytes = 0;
+  // host entry point: kernels and the copy back run on streams of their own, so that the compute
+  // and the device-to-host copy of one chunk of heads overlap the host-to-device copies of the
+  // next (PCIe is full duplex)
+  cudaStream_t compute = nullptr, d2h = nullptr;
+  cudaEvent_t chunk_in[8] = {}, chunk_done[8] = {};
+  cudaEvent_t all_back = nullptr;
 };
+constexpr int kHostChunks = 8;
+static int g_host_chunks = 4;   // chunks a host call is cut into (<= kHostChunks)
 static DeviceBuffers g_dev[kMaxDevices];
 
 static int grow(void** ptr, size_t* have, size_t need) {
@@ -399,16 +407,45 @@ int monarch_attn_fwd_host(const void* Qh, const void* Kh, const void* Vh, void* 
   if (rc != MA_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   char* s = (char*)B.stage;
-  size_t bytes = (size_t)p.BH * p.N * p.d * esize(p.dtype);
-  if (cudaMemcpyAsync(s, Qh, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(s + one, Kh, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(s + 2 * one, Vh, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+  if (!B.all_back) {
+    if (cudaStreamCreateWithFlags(&B.compute, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&B.d2h, cudaStreamNonBlocking) != cudaSuccess)
+      return MA_ERR_CUDA;
+    for (int c = 0; c < kHostChunks; ++c)
+      if (cudaEventCreateWithFlags(&B.chunk_in[c], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&B.chunk_done[c], cudaEventDisableTiming) != cudaSuccess)
+        return MA_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&B.all_back, cudaEventDisableTiming) != cudaSuccess) return MA_ERR_CUDA;
+  }
+  // (batch, head) units are independent (Sec. 3: every equation is per head), so the call is cut
+  // into chunks of units: copy in on `stream`, compute on the library's compute stream, copy back
+  // on its copy-back stream, chained by events.
+  const size_t unit = (size_t)p.N * p.d * esize(p.dtype);
+  const int chunks = (unit % 16 == 0 && p.BH >= g_host_chunks) ? g_host_chunks : 1;
+  int launches = 0;
+  for (int c = 0; c < chunks; ++c) {
+    const int u0 = (int)((long long)p.BH * c / chunks), u1 = (int)((long long)p.BH * (c + 1) / chunks);
+    const size_t off = (size_t)u0 * unit, len = (size_t)(u1 - u0) * unit;
+    if (cudaMemcpyAsync(s + off, (const char*)Qh + off, len, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(s + one + off, (const char*)Kh + off, len, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(s + 2 * one + off, (const char*)Vh + off, len, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return MA_ERR_CUDA;
+    if (cudaEventRecord(B.chunk_in[c], st) != cudaSuccess ||
+        cudaStreamWaitEvent(B.compute, B.chunk_in[c], 0) != cudaSuccess)
+      return MA_ERR_CUDA;
+    rc = monarch_attn_fwd(s + off, s + one + off, s + 2 * one + off, s + 3 * one + off, 1, u1 - u0, N, d, b,
+                          T, dtype, (void*)B.compute);
+    if (rc != MA_OK) return rc;
+    launches += g_last_launches;
+    if (cudaEventRecord(B.chunk_done[c], B.compute) != cudaSuccess ||
+        cudaStreamWaitEvent(B.d2h, B.chunk_done[c], 0) != cudaSuccess ||
+        cudaMemcpyAsync((char*)Yh + off, s + 3 * one + off, len, cudaMemcpyDeviceToHost, B.d2h) != cudaSuccess)
+      return MA_ERR_CUDA;
+  }
+  // the caller's stream is done when the last result is back
+  if (cudaEventRecord(B.all_back, B.d2h) != cudaSuccess || cudaStreamWaitEvent(st, B.all_back, 0) != cudaSuccess)
     return MA_ERR_CUDA;
-  rc = monarch_attn_fwd(s, s + one, s + 2 * one, s + 3 * one, batch, heads, N, d, b, T, dtype,
-                        stream);
-  if (rc != MA_OK) return rc;
-  if (cudaMemcpyAsync(Yh, s + 3 * one, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-    return MA_ERR_CUDA;
+  g_last_launches = launches;
   return MA_OK;
 }
 
@@ -474,6 +511,8 @@ int monarch_attn_debug_knob(int knob, long long value) {
     tp::knobs().wait_cycles = value > 0 ? value : tensor::kWaitCycles;
   } else if (knob == 2) {
     tp::knobs().skip_first_half_step = value != 0;
+  } else if (knob == 3) {
+    g_host_chunks = value < 1 ? 1 : (value > kHostChunks ? kHostChunks : (int)value);
   } else {
     return MA_ERR_SHAPE;
   }

@@ -429,6 +429,26 @@ def test_host_entry_point_matches_device_entry_point():
     assert torch.equal(Yd.cpu(), Yh)
 
 
+def test_host_entry_point_chunking_does_not_change_results():
+    """The host call is cut into chunks of (batch, head) units on three streams; any chunk count
+    gives the bits of the device call, the launch count is the sum over chunks, and work queued
+    on the caller's stream after the call sees the result."""
+    Q, K, V = wl.make_qkv(3, 5, 256, 64, "f16", 8, 1.0, seed=14)       # 15 units: ragged chunks
+    hs = [torch.from_numpy(x).to(torch.float16).pin_memory() for x in (Q, K, V)]
+    ref = binding.monarch_attn_fwd(*(h.cuda() for h in hs), 16, 2).cpu()
+    try:
+        for chunks in (1, 2, 4, 7):
+            binding.monarch_attn_debug_knob(3, chunks)
+            Yh = torch.zeros_like(hs[0]).pin_memory()
+            binding.monarch_attn_fwd_host(hs[0], hs[1], hs[2], Yh, 16, 2)
+            assert binding.monarch_attn_last_launch_count() == chunks
+            dev_copy = Yh.cuda(non_blocking=True)          # ordered after the call on the same stream
+            torch.cuda.synchronize()
+            assert torch.equal(Yh, ref) and torch.equal(dev_copy.cpu(), ref)
+    finally:
+        binding.monarch_attn_debug_knob(3, 4)
+
+
 def test_unsupported_and_error_paths_on_device():
     x = torch.zeros(1, 1, 256, 64, device="cuda")
     with pytest.raises(binding.MonarchAttnError) as e:
