@@ -46,7 +46,8 @@ using fused::quad_max;
 using fused::quad_sum;
 
 constexpr int kThreads = 256, kWarps = 8, kRowBytes = 128, kMaxSmem = 227 * 1024;
-constexpr int kDumpBytes = kThreads * 16;   // where stmatrix rows past the end of a block go
+// where stmatrix rows past the end of a block go: 16 bytes per thread
+inline size_t dump_bytes(int threads) { return (size_t)threads * 16; }
 
 // Four 8x8 16-bit matrices from accumulator-layout registers; lane L gives the address of row L & 7
 // of matrix L >> 3.
@@ -69,13 +70,13 @@ __device__ __forceinline__ uint32_t rowx(int k, int i, int b, int c) {
   return (uint32_t)((k * b + i) * kRowBytes + ((c ^ (i & 7) ^ (k & 7)) << 4));
 }
 
-inline size_t smem_bytes(int N, int T) {
-  return (size_t)(T == 1 ? 3 : 4) * N * kRowBytes + (((size_t)N * 4 + 15) & ~(size_t)15) + kDumpBytes + 1024;
+inline size_t smem_bytes(int N, int T, int threads = kThreads) {
+  return (size_t)(T == 1 ? 3 : 4) * N * kRowBytes + (((size_t)N * 4 + 15) & ~(size_t)15) + dump_bytes(threads) + 1024;
 }
 
 // BP, MP: b and m rounded up to 16 or 32.
 template <typename TIn, int BP, int MP>
-__global__ void __launch_bounds__(kThreads, (BP == 16 && MP == 16) ? 2 : 1)
+__global__ void __launch_bounds__((BP == 16 && MP == 16) ? 2 * kThreads : kThreads, 1)
 monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
                     TIn* __restrict__ Y, int N, int d, int b, int m, int T_steps, float scale,
                     int n_valid, int H, float* __restrict__ lse) {
@@ -98,6 +99,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   const uint32_t sK_u = sQ_u + tile, sV_u = sK_u + tile;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nw = blockDim.x >> 5;    // 8 warps, or 16 where only one CTA fits an SM (16 x 16 blocks)
   const int g = lane >> 2, t = lane & 3;
   const int h_idx = blockIdx.x;
   // Contractions over d always run over the 64 padded columns (zeros beyond d: the inputs are
@@ -141,7 +143,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
     else asm volatile("cp.async.wait_group 3;" ::: "memory");
   };
   int my_tiles = 0;                  // blocks this warp owns in an R half-step (at most 4)
-  for (int k = warp; k < m; k += kWarps) {
+  for (int k = warp; k < m; k += nw) {
     load_block(Q, 0, k);
     load_block(K, 1, k);
     if (T_steps == 1) load_block(V, 2, k);
@@ -153,7 +155,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   for (int step = 1; step <= T_steps; ++step) {
     const bool first = step == 1, last = step == T_steps;
     if (last && !first) {   // alpha_L of the round before is dead: V takes its buffer
-      for (int k = warp; k < m; k += kWarps) {
+      for (int k = warp; k < m; k += nw) {
         load_block(V, 2, k);
         asm volatile("cp.async.commit_group;" ::: "memory");
       }
@@ -163,7 +165,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
     {
       const uint32_t sA_u = first ? sQ_u : sV_u + tile;   // alpha_R (= Q rows while L is the identity)
       int it = 0;
-      for (int k = warp; k < m; k += kWarps, ++it) {
+      for (int k = warp; k < m; k += nw, ++it) {
         if (first || last) {          // block k may still be on its way
           wait_pending(my_tiles - 1 - it);
           if (first) {
@@ -305,7 +307,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
     {
       const uint32_t sAL_u = last ? sK_u : sV_u;      // alpha_L of earlier rounds shares V's buffer
       const uint32_t sAR_u = sV_u + tile;
-      for (int j = warp; j < b; j += kWarps) {
+      for (int j = warp; j < b; j += nw) {
         float c[MP / 8][2];
 #pragma unroll
         for (int nt = 0; nt < MP / 8; ++nt)
@@ -536,11 +538,16 @@ template <typename TIn, int BP, int MP>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
                     int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st) {
   auto kern = monarch_fused_small<TIn, BP, MP>;
-  const size_t smem = smem_bytes(N, T);
+  // The 16 x 16 kernel is compiled for 128 registers: two CTAs of 8 warps per SM where shared memory
+  // lets two fit, else one CTA of 16 warps (each warp then owns at most one tile per half-step).
+  int threads = kThreads;
+  if (BP == 16 && MP == 16 && 2 * (smem_bytes(N, T) + 1024) > (size_t)228 * 1024 && (m > 8 || b > 8))
+    threads = 2 * kThreads;
+  const size_t smem = smem_bytes(N, T, threads);
   if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
     return 7;
-  kern<<<BH, kThreads, smem, st>>>((const TIn*)Q, (const TIn*)K, (const TIn*)V, (TIn*)Y, N, d, b, m, T,
+  kern<<<BH, threads, smem, st>>>((const TIn*)Q, (const TIn*)K, (const TIn*)V, (TIn*)Y, N, d, b, m, T,
                                    scale, n_valid, H, lse);
   return cudaGetLastError() == cudaSuccess ? 0 : 7;
 }
