@@ -76,7 +76,7 @@ inline size_t smem_bytes(int N, int T, int threads = kThreads) {
 
 // BP, MP: b and m rounded up to 16 or 32.
 template <typename TIn, int BP, int MP>
-__global__ void __launch_bounds__((BP == 16 && MP == 16) ? 2 * kThreads : kThreads, 1)
+__global__ void __launch_bounds__((BP == 16 || MP == 16) ? 2 * kThreads : kThreads, 1)
 monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
                     TIn* __restrict__ Y, int N, int d, int b, int m, int T_steps, float scale,
                     int n_valid, int H, float* __restrict__ lse) {
@@ -175,7 +175,10 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
           if (last) convert_block(2, k);
           __syncwarp();
         }
-        uint32_t outL[BP / 16][8][2], outY[BP / 16][8][2];
+        // phase 1: scores and softmax of every 16-row tile of the block; the weights stay in
+        // registers as A fragments
+        uint32_t pa[BP / 16][BP / 16][4];
+        float inv_s[BP / 16][2];
 #pragma unroll
         for (int rt = 0; rt < BP / 16; ++rt) {
           const int j0 = 16 * rt;
@@ -204,7 +207,6 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             }
           }
           // rows j = j0 + g (c0, c1) and j0 + g + 8 (c2, c3); columns i = 8 nt + 2t, +1
-          float inv_s[2];
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             const int j = j0 + g + 8 * hh;
@@ -233,69 +235,58 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
               }
             sum = quad_sum(sum);
             sz = quad_sum(sz);
-            inv_s[hh] = 1.f / sum;
+            inv_s[rt][hh] = 1.f / sum;
             // c_L = sum R log R (natural log): ln2 * (sum p z / sum - max - log2 sum)
-            if (t == 0 && j < b) sCL[k * b + j] = kLn2 * (sz * inv_s[hh] - mx - lg2(sum));
+            if (t == 0 && j < b) sCL[k * b + j] = kLn2 * (sz * inv_s[rt][hh] - mx - lg2(sum));
           }
-          uint32_t pa[BP / 16][4];
 #pragma unroll
           for (int kk = 0; kk < BP / 16; ++kk) {
-            pa[kk][0] = Mma<T>::pack(s[2 * kk][0], s[2 * kk][1]);
-            pa[kk][1] = Mma<T>::pack(s[2 * kk][2], s[2 * kk][3]);
-            pa[kk][2] = Mma<T>::pack(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-            pa[kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+            pa[rt][kk][0] = Mma<T>::pack(s[2 * kk][0], s[2 * kk][1]);
+            pa[rt][kk][1] = Mma<T>::pack(s[2 * kk][2], s[2 * kk][3]);
+            pa[rt][kk][2] = Mma<T>::pack(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+            pa[rt][kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
           }
-          uint32_t v_off[BP / 16];    // rows (k, i) of K and V as the second product's B operand
+        }
+        // phase 2: second products, one 16-column slab of v at a time for all row tiles.  This warp
+        // alone reads block k of K and V, and every score is formed: on the last round the slab of
+        // alpha_L / y goes straight over the slab of K / V it was computed from.
+        const uint32_t dstL_u = last ? sK_u : sV_u;     // alpha_L of earlier rounds shares V's buffer
+        uint32_t v_off[BP / 16];    // rows (k, i) of K and V as the second product's B operand
 #pragma unroll
-          for (int kk = 0; kk < BP / 16; ++kk) v_off[kk] = rowx(k, min(16 * kk + (lane & 15), b - 1), b, lane >> 4);
+        for (int kk = 0; kk < BP / 16; ++kk) v_off[kk] = rowx(k, min(16 * kk + (lane & 15), b - 1), b, lane >> 4);
 #pragma unroll
-          for (int np = 0; np < 4; ++np) {     // two 8-column tiles of v per transposing ldmatrix
-            if (np >= ksteps) {
-              outL[rt][2 * np][0] = outL[rt][2 * np][1] = 0u;
-              outL[rt][2 * np + 1][0] = outL[rt][2 * np + 1][1] = 0u;
-              outY[rt][2 * np][0] = outY[rt][2 * np][1] = 0u;
-              outY[rt][2 * np + 1][0] = outY[rt][2 * np + 1][1] = 0u;
-              continue;
-            }
+        for (int np = 0; np < ksteps; ++np) {   // two 8-column tiles of v per transposing ldmatrix
+          uint32_t bk[BP / 16][4], bv[BP / 16][4];
+#pragma unroll
+          for (int kk = 0; kk < BP / 16; ++kk) {
+            ldsm_x4_trans(bk[kk], (sK_u + v_off[kk]) ^ (np << 5));
+            if (last) ldsm_x4_trans(bv[kk], (sV_u + v_off[kk]) ^ (np << 5));
+          }
+          __syncwarp();
+#pragma unroll
+          for (int rt = 0; rt < BP / 16; ++rt) {
+            if (16 * rt >= b) continue;
             float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
             float y[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
             for (int kk = 0; kk < BP / 16; ++kk) {
-              uint32_t bf[4];
-              ldsm_x4_trans(bf, (sK_u + v_off[kk]) ^ (np << 5));
-              Mma<T>::run(o[0], pa[kk], bf);
-              Mma<T>::run(o[1], pa[kk], bf + 2);
+              Mma<T>::run(o[0], pa[rt][kk], bk[kk]);
+              Mma<T>::run(o[1], pa[rt][kk], bk[kk] + 2);
               if (last) {
-                ldsm_x4_trans(bf, (sV_u + v_off[kk]) ^ (np << 5));
-                Mma<T>::run(y[0], pa[kk], bf);
-                Mma<T>::run(y[1], pa[kk], bf + 2);
+                Mma<T>::run(y[0], pa[rt][kk], bv[kk]);
+                Mma<T>::run(y[1], pa[rt][kk], bv[kk] + 2);
               }
             }
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              outL[rt][2 * np + q][0] = Mma<T>::pack(o[q][0] * inv_s[0], o[q][1] * inv_s[0]);
-              outL[rt][2 * np + q][1] = Mma<T>::pack(o[q][2] * inv_s[1], o[q][3] * inv_s[1]);
-              outY[rt][2 * np + q][0] = Mma<T>::pack(y[q][0] * inv_s[0], y[q][1] * inv_s[0]);
-              outY[rt][2 * np + q][1] = Mma<T>::pack(y[q][2] * inv_s[1], y[q][3] * inv_s[1]);
-            }
-          }
-        }
-        // this warp alone reads block k of K and V: on the last round the results take their place
-        __syncwarp();
-        const uint32_t dstL_u = last ? sK_u : sV_u;     // alpha_L of earlier rounds shares V's buffer
-#pragma unroll
-        for (int rt = 0; rt < BP / 16; ++rt) {
-          if (16 * rt >= b) continue;
-          const int j = 16 * rt + st_row;
-          const uint32_t row_u = rowx(k, j, b, st_nt);
-#pragma unroll
-          for (int np = 0; np < 4; ++np) {
-            const uint32_t off = row_u ^ (np << 5);
-            stsm_x4(j < b ? dstL_u + off : dump_u, outL[rt][2 * np][0], outL[rt][2 * np][1],
-                    outL[rt][2 * np + 1][0], outL[rt][2 * np + 1][1]);
+            const int j = 16 * rt + st_row;
+            const uint32_t off = rowx(k, j, b, st_nt) ^ (np << 5);
+            const float i0 = inv_s[rt][0], i1 = inv_s[rt][1];
+            stsm_x4(j < b ? dstL_u + off : dump_u, Mma<T>::pack(o[0][0] * i0, o[0][1] * i0),
+                    Mma<T>::pack(o[0][2] * i1, o[0][3] * i1), Mma<T>::pack(o[1][0] * i0, o[1][1] * i0),
+                    Mma<T>::pack(o[1][2] * i1, o[1][3] * i1));
             if (last)
-              stsm_x4(j < b ? sV_u + off : dump_u, outY[rt][2 * np][0], outY[rt][2 * np][1],
-                      outY[rt][2 * np + 1][0], outY[rt][2 * np + 1][1]);
+              stsm_x4(j < b ? sV_u + off : dump_u, Mma<T>::pack(y[0][0] * i0, y[0][1] * i0),
+                      Mma<T>::pack(y[0][2] * i1, y[0][3] * i1), Mma<T>::pack(y[1][0] * i0, y[1][1] * i0),
+                      Mma<T>::pack(y[1][2] * i1, y[1][3] * i1));
           }
         }
       }
@@ -388,14 +379,17 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
               pa[kk][2] = Mma<T>::pack(s[2 * kk + 1][0], s[2 * kk + 1][1]);
               pa[kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
             }
-            uint32_t out[8][2];
             uint32_t y_u[MP / 16];
 #pragma unroll
             for (int kk = 0; kk < MP / 16; ++kk)
               y_u[kk] = sV_u + rowx(min(16 * kk + (lane & 15), m - 1), j, b, lane >> 4);
+            // only this warp reads the rows (l, j) of Q, and for this row tile it has (they were the
+            // A operand of the scores): Y takes their place, slab by slab
+            const int l = l0 + st_row;
+            const uint32_t row_u = sQ_u + rowx(l, j, b, st_nt);
+            __syncwarp();
 #pragma unroll
-            for (int np = 0; np < 4; ++np) {
-              if (np >= ksteps) continue;
+            for (int np = 0; np < ksteps; ++np) {
               float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
               for (int kk = 0; kk < MP / 16; ++kk) {
@@ -404,21 +398,10 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
                 Mma<T>::run(o[0], pa[kk], bf);
                 Mma<T>::run(o[1], pa[kk], bf + 2);
               }
-#pragma unroll
-              for (int q = 0; q < 2; ++q) {
-                out[2 * np + q][0] = Mma<T>::pack(o[q][0] * inv_s[0], o[q][1] * inv_s[0]);
-                out[2 * np + q][1] = Mma<T>::pack(o[q][2] * inv_s[1], o[q][3] * inv_s[1]);
-              }
-            }
-            // only this warp reads the rows (l, j) of Q, and it has: Y takes their place
-            __syncwarp();
-            {
-              const int l = l0 + st_row;
-              const uint32_t row_u = sQ_u + rowx(l, j, b, st_nt);
-#pragma unroll
-              for (int np = 0; np < 4; ++np)
-                stsm_x4(l < m ? row_u ^ (np << 5) : dump_u, out[2 * np][0],
-                        out[2 * np][1], out[2 * np + 1][0], out[2 * np + 1][1]);
+              stsm_x4(l < m ? row_u ^ (np << 5) : dump_u, Mma<T>::pack(o[0][0] * inv_s[0], o[0][1] * inv_s[0]),
+                      Mma<T>::pack(o[0][2] * inv_s[1], o[0][3] * inv_s[1]),
+                      Mma<T>::pack(o[1][0] * inv_s[0], o[1][1] * inv_s[0]),
+                      Mma<T>::pack(o[1][2] * inv_s[1], o[1][3] * inv_s[1]));
             }
             __syncwarp();
           } else {
@@ -541,7 +524,8 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   // The 16 x 16 kernel is compiled for 128 registers: two CTAs of 8 warps per SM where shared memory
   // lets two fit, else one CTA of 16 warps (each warp then owns at most one tile per half-step).
   int threads = kThreads;
-  if (BP == 16 && MP == 16 && 2 * (smem_bytes(N, T) + 1024) > (size_t)228 * 1024 && (m > 8 || b > 8))
+  if ((BP == 16 || MP == 16) && 2 * (smem_bytes(N, T) + 1024) > (size_t)228 * 1024 && (m > 8 || b > 8) &&
+      smem_bytes(N, T, 2 * kThreads) <= (size_t)kMaxSmem)
     threads = 2 * kThreads;
   const size_t smem = smem_bytes(N, T, threads);
   if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
