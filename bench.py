@@ -210,7 +210,8 @@ def time_e2e(w, steps, warmup, torch, binding, dist=None):
 
 # DRAM bytes of ONE launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
 # ncu; see the summaries under profiles/ named for each kernel and workload).
-NCU_TRAFFIC_BYTES = {"C5": 185.5e6 + 31.7e6, "C4": 174.9e6 + 20.7e6, "C3": 132.7e6 + 42.5e6, "C2": 75.6e6 + 4.4e6}
+NCU_TRAFFIC_BYTES = {"C5": 185.5e6 + 31.7e6, "C4": 174.9e6 + 20.7e6, "C3": 132.7e6 + 42.5e6, "C2": 75.5e6 + 4.0e6,
+                     "S1": 62.0e6 + 2.4e6, "S3": (100.7e6 + 31.8e6) + (101.8e6 + 13.0e6)}   # S3: both launches of a step
 
 
 def roofline(w, ms, peaks, which):
