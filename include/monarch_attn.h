@@ -59,9 +59,10 @@ typedef enum {
   MA_PATH_FUSED_SMALL = 7, /* the same idea for any block shape: f16/bf16, m and b <= 32 (m need not
                              equal b), d <= 64 a multiple of 8, N <= 580 for T = 1 and <= 440 for
                              T > 1 (the states of a head must fit shared memory); f16 arithmetic */
-  MA_PATH_TILE_MMA = 8    /* warp-MMA kernels, one launch per half-step, f16 states in the workspace:
-                             f16/bf16, m and b <= 128 (m need not equal b), d <= 128 a multiple of
-                             8; the 16-bit path of the shapes no other tensor-core kernel takes */
+  MA_PATH_TILE_MMA = 8    /* warp-MMA kernels, one launch per half-step, f16 states in the workspace
+                             (hi + lo pairs of f16 from T = 3 on): f16/bf16, m and b <= 128 (m need
+                             not equal b), d <= 128 a multiple of 8; the 16-bit path of the shapes no
+                             other tensor-core kernel takes */
 } ma_path;
 
 /* T-step MonarchAttention forward (Eq. 7-10 then Eq. 4) with scale = 1/sqrt(d).

@@ -142,13 +142,12 @@ static int resolve_path(const Problem& p, int path) {
     // stores, per-warp pipelined loads), so AUTO never picks MA_PATH_FUSED.
     if (p.b <= 16 && p.m <= 16 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T))
       return MA_PATH_FUSED_SMALL;
-    // bf16 with b = 32 and more than two rounds stays on the fp32-state kernels: on the peaky-logit
-    // recipe of that shape the 8-bit mantissa of alpha_R (used twice from T = 3 on) costs 4e-2 on
-    // the worst head; up to T = 2 the hi + lo alpha_L of the tensor path keeps it under 1e-2.
-    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) {
-      if (!(p.b == 32 && p.dtype == MA_BF16 && p.T > 2)) return MA_PATH_TENSOR;
-      if (generic_supported(p)) return MA_PATH_GENERIC;
-    }
+    // bf16 with b = 32 and more than two rounds leaves the tcgen05 path: on the peaky-logit recipe of
+    // that shape the 8-bit mantissa of alpha_R (used twice from T = 3 on) costs 4e-2 on the worst
+    // head; up to T = 2 the hi + lo alpha_L of that path keeps it under 1e-2.  The tile kernels keep
+    // both states as hi + lo pairs of f16 from T = 3 on (4e-3 on the same inputs).
+    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) && !(p.b == 32 && p.dtype == MA_BF16 && p.T > 2))
+      return MA_PATH_TENSOR;
     if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
     if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
     if (generic_supported(p)) return MA_PATH_GENERIC;
@@ -190,7 +189,7 @@ static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused
 static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
   if (resolved == MA_PATH_FUSED || resolved == MA_PATH_FUSED_SMALL) return kStatusBytes;   // no states leave the chip
-  if (resolved == MA_PATH_TILE_MMA) return tile::workspace_bytes(p.BH, p.N, p.d);
+  if (resolved == MA_PATH_TILE_MMA) return tile::workspace_bytes(p.BH, p.N, p.d, p.T);
   if (resolved == MA_PATH_TENSOR_BASIC) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
   if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_PHASED ||
       resolved == MA_PATH_TENSOR_CHAINED)

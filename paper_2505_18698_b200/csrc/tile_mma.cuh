@@ -114,9 +114,21 @@ __device__ __forceinline__ void scatter_rows16(TDst* __restrict__ dst, size_t st
 // Tiles are allocated with their row count rounded up to 16: a warp stores whole 16-row fragments,
 // and the rows past the block land in that padding.
 __host__ __device__ constexpr int round16(int x) { return (x + 15) & ~15; }
-inline size_t r_smem_bytes(int b, int dt) { return (size_t)4 * round16(b) * pitch_of(dt); }
-inline size_t l_smem_bytes(int m, int cm, int dt) {
-  const size_t tiles = (size_t)3 * round16(m) * pitch_of(dt);  // Q(l,j), alpha_L(k,j), y(k,j)
+// `hilo`: the states alpha_L and alpha_R are kept as a hi + lo pair of f16 arrays (one more tile).
+// x rounded to f16 (hi) and the f16 rounding of what is left (lo): hi + lo carries 22 bits of x.
+template <bool HILO>
+__device__ __forceinline__ void split_hilo(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  hi = Mma<T>::pack(x0, x1);
+  lo = 0u;
+  if (HILO) {
+    const float2 h = Mma<T>::unpack(hi);
+    lo = Mma<T>::pack(x0 - h.x, x1 - h.y);
+  }
+}
+
+inline size_t r_smem_bytes(int b, int dt, bool hilo) { return (size_t)(hilo ? 5 : 4) * round16(b) * pitch_of(dt); }
+inline size_t l_smem_bytes(int m, int cm, int dt, bool hilo) {
+  const size_t tiles = (size_t)(hilo ? 4 : 3) * round16(m) * pitch_of(dt);  // Q(l,j), alpha_L(k,j) (+ lo), y(k,j)
   const size_t p_tile = (size_t)round16(m) * (cm * 2 + 16);    // weights for the transposed product
   const size_t stats = (size_t)(2 * 8 * cm + cm) * 4;          // column max / sum per warp, c_L
   return tiles + p_tile + stats;
@@ -127,10 +139,11 @@ inline size_t l_smem_bytes(int m, int cm, int dt) {
 //   Z_R[j,i] = scale * <aR(k,j), K(k,i)>  (alpha_R arrives divided by c_R), R = softmax_i Z_R,
 //   aL(k,j) = sum_i R[j,i] K(k,i), cL(k,j) = sum_i R log R, (last round) y(k,j) = sum_i R[j,i] V(k,i)
 // CB: b rounded up to 32, 64 or 128; DT: 16-column steps over d (4 or 8).
-template <typename TIn, int CB, int DT>
+template <typename TIn, int CB, int DT, bool HILO>
 __global__ void __launch_bounds__(256)
 r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
               const __half* __restrict__ aR, __half* __restrict__ aL, __half* __restrict__ y,
+              const __half* __restrict__ aR_lo, __half* __restrict__ aL_lo,
               float* __restrict__ cL, int N, int d, int b, float scale, int n_valid, int H, int first,
               int last) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -142,11 +155,14 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
   uint8_t* sK = sA + (size_t)rb * kPitch;
   uint8_t* sV = sK + (size_t)rb * kPitch;
   uint8_t* sY = sV + (size_t)rb * kPitch;      // staging of y rows on the last round
+  uint8_t* sAlo = sY + (size_t)rb * kPitch;    // low halves of alpha_R in, of alpha_L out (hi + lo states)
+  constexpr bool hilo = HILO;
   const HeadRows hr = head_rows(h, N, d, H);
   const size_t st_rows = ((size_t)h * N + (size_t)k * b) * d;    // block k of the state arrays
 
   if (first) gather_rows<TIn, DT>(sA, Q + hr.base + (size_t)k * b * hr.stride, hr.stride, b, d);
   else gather_rows<__half, DT>(sA, aR + st_rows, (size_t)d, b, d);
+  if (!first && hilo) gather_rows<__half, DT>(sAlo, aR_lo + st_rows, (size_t)d, b, d);
   gather_rows<TIn, DT>(sK, K + hr.base + (size_t)k * b * hr.stride, hr.stride, b, d);
   if (last) gather_rows<TIn, DT>(sV, V + hr.base + (size_t)k * b * hr.stride, hr.stride, b, d);
   gather_wait();
@@ -184,6 +200,22 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
         ldsm_x4(bf, b_u[cp] + ks * 32);
         Mma<T>::run(s[2 * cp], a, bf);
         Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+      }
+    }
+    if (!first && hilo) {      // + <alpha_R lo, K>
+      const uint32_t alo_u = a_u - sA_u + (uint32_t)__cvta_generic_to_shared(sAlo);
+#pragma unroll
+      for (int ks = 0; ks < DT; ++ks) {
+        uint32_t a[4];
+        ldsm_x4(a, alo_u + ks * 32);
+#pragma unroll
+        for (int cp = 0; cp < CB / 16; ++cp) {
+          if (16 * cp >= b) continue;
+          uint32_t bf[4];
+          ldsm_x4(bf, b_u[cp] + ks * 32);
+          Mma<T>::run(s[2 * cp], a, bf);
+          Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+        }
       }
     }
   }
@@ -234,6 +266,7 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
   const int st_row = (lane & 7) + ((lane >> 3) & 1) * 8, st_nt = (lane >> 4) & 1;
   const uint32_t stA_u = sA_u + (j0 + st_row) * kPitch + st_nt * 16;
   const uint32_t stY_u = sY_u + (j0 + st_row) * kPitch + st_nt * 16;
+  const uint32_t stLo_u = (uint32_t)__cvta_generic_to_shared(sAlo) + (j0 + st_row) * kPitch + st_nt * 16;
   __syncwarp();
   uint32_t v_off[CB / 16];
 #pragma unroll
@@ -256,10 +289,13 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
         Mma<T>::run(yv[1], pa[kk], bf + 2);
       }
     }
-    stsm_x4(stA_u + np * 32, Mma<T>::pack(o[0][0] * inv_s[0], o[0][1] * inv_s[0]),
-            Mma<T>::pack(o[0][2] * inv_s[1], o[0][3] * inv_s[1]),
-            Mma<T>::pack(o[1][0] * inv_s[0], o[1][1] * inv_s[0]),
-            Mma<T>::pack(o[1][2] * inv_s[1], o[1][3] * inv_s[1]));
+    uint32_t hi[4], lo[4];
+    split_hilo<HILO>(o[0][0] * inv_s[0], o[0][1] * inv_s[0], hi[0], lo[0]);
+    split_hilo<HILO>(o[0][2] * inv_s[1], o[0][3] * inv_s[1], hi[1], lo[1]);
+    split_hilo<HILO>(o[1][0] * inv_s[0], o[1][1] * inv_s[0], hi[2], lo[2]);
+    split_hilo<HILO>(o[1][2] * inv_s[1], o[1][3] * inv_s[1], hi[3], lo[3]);
+    stsm_x4(stA_u + np * 32, hi[0], hi[1], hi[2], hi[3]);
+    if (hilo) stsm_x4(stLo_u + np * 32, lo[0], lo[1], lo[2], lo[3]);
     if (last)
       stsm_x4(stY_u + np * 32, Mma<T>::pack(yv[0][0] * inv_s[0], yv[0][1] * inv_s[0]),
               Mma<T>::pack(yv[0][2] * inv_s[1], yv[0][3] * inv_s[1]),
@@ -269,6 +305,8 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
   __syncwarp();
   const int rows = min(16, b - j0);
   scatter_rows16<__half, DT>(aL + st_rows + (size_t)j0 * d, (size_t)d, sA + (size_t)j0 * kPitch, rows, d, lane);
+  if (hilo)
+    scatter_rows16<__half, DT>(aL_lo + st_rows + (size_t)j0 * d, (size_t)d, sAlo + (size_t)j0 * kPitch, rows, d, lane);
   if (last)
     scatter_rows16<__half, DT>(y + st_rows + (size_t)j0 * d, (size_t)d, sY + (size_t)j0 * kPitch, rows, d, lane);
 }
@@ -279,11 +317,12 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
 //   not final: aR(k,j) = sum_l L[l,k] Q(l,j) / cR(k,j), cR(k,j) = sum_l L[l,k]
 //   final:     Y(l,j) = sum_k L[l,k] y(k,j); optionally the row's log-sum-exp (Eq. 6)
 // CM: m rounded up to 32, 64 or 128.
-template <typename TIn, int CM, int DT>
+template <typename TIn, int CM, int DT, bool HILO>
 __global__ void __launch_bounds__(256)
 l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const float* __restrict__ cL,
-              const __half* __restrict__ y, __half* __restrict__ aR, TIn* __restrict__ Y,
-              float* __restrict__ lse, int N, int d, int b, int m, float scale, int H, int last) {
+              const __half* __restrict__ y, __half* __restrict__ aR, const __half* __restrict__ aL_lo,
+              __half* __restrict__ aR_lo, TIn* __restrict__ Y, float* __restrict__ lse, int N, int d, int b,
+              int m, float scale, int H, int last) {
   extern __shared__ __align__(128) uint8_t smem[];
   constexpr int kPitch = pitch_of(DT), kPPitch = CM * 2 + 16;
   const int j = blockIdx.x, h = blockIdx.y;
@@ -292,7 +331,9 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
   uint8_t* sQ = smem;
   uint8_t* sL = sQ + (size_t)rm * kPitch;
   uint8_t* sYt = sL + (size_t)rm * kPitch;
-  uint8_t* sP = sYt + (size_t)rm * kPitch;
+  constexpr bool hilo = HILO;
+  uint8_t* sLlo = sYt + (size_t)rm * kPitch;   // low halves of alpha_L in, of alpha_R out (hi + lo states)
+  uint8_t* sP = sLlo + (hilo ? (size_t)rm * kPitch : 0);
   float* sColMax = reinterpret_cast<float*>(sP + (size_t)rm * kPPitch);
   float* sColSum = sColMax + 8 * CM;
   float* sC = sColSum + 8 * CM;
@@ -302,6 +343,7 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
 
   gather_rows<TIn, DT>(sQ, Q + hr.base + (size_t)j * hr.stride, (size_t)b * hr.stride, m, d);
   gather_rows<__half, DT>(sL, aL + st_rows, st_stride, m, d);
+  if (hilo) gather_rows<__half, DT>(sLlo, aL_lo + st_rows, st_stride, m, d);
   if (last) gather_rows<__half, DT>(sYt, y + st_rows, st_stride, m, d);
   for (int kq = threadIdx.x; kq < m; kq += blockDim.x) sC[kq] = cL[(size_t)h * N + (size_t)kq * b + j] * kLog2e;
   gather_wait();
@@ -338,6 +380,11 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
         ldsm_x4(bf, b_u[cp] + ks * 32);
         Mma<T>::run(s[2 * cp], a, bf);
         Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+        if (hilo) {      // + <Q, alpha_L lo>
+          ldsm_x4(bf, b_u[cp] - sL_u + (uint32_t)__cvta_generic_to_shared(sLlo) + ks * 32);
+          Mma<T>::run(s[2 * cp], a, bf);
+          Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+        }
       }
     }
 #pragma unroll
@@ -485,13 +532,20 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
       Mma<T>::run(o[0], a, bf);
       Mma<T>::run(o[1], a, bf + 2);
     }
-    stsm_x4(st_u + np * 32, Mma<T>::pack(o[0][0] * ic[0], o[0][1] * ic[0]),
-            Mma<T>::pack(o[0][2] * ic[1], o[0][3] * ic[1]), Mma<T>::pack(o[1][0] * ic[0], o[1][1] * ic[0]),
-            Mma<T>::pack(o[1][2] * ic[1], o[1][3] * ic[1]));
+    uint32_t hi[4], lo[4];
+    split_hilo<HILO>(o[0][0] * ic[0], o[0][1] * ic[0], hi[0], lo[0]);
+    split_hilo<HILO>(o[0][2] * ic[1], o[0][3] * ic[1], hi[1], lo[1]);
+    split_hilo<HILO>(o[1][0] * ic[0], o[1][1] * ic[0], hi[2], lo[2]);
+    split_hilo<HILO>(o[1][2] * ic[1], o[1][3] * ic[1], hi[3], lo[3]);
+    stsm_x4(st_u + np * 32, hi[0], hi[1], hi[2], hi[3]);
+    if (hilo) stsm_x4(st_u - sL_u + (uint32_t)__cvta_generic_to_shared(sLlo) + np * 32, lo[0], lo[1], lo[2], lo[3]);
   }
   __syncwarp();
   scatter_rows16<__half, DT>(aR + st_rows + (size_t)k0 * st_stride, st_stride, sL + (size_t)k0 * kPitch,
                              min(16, m - k0), d, lane);
+  if (hilo)
+    scatter_rows16<__half, DT>(aR_lo + st_rows + (size_t)k0 * st_stride, st_stride, sLlo + (size_t)k0 * kPitch,
+                               min(16, m - k0), d, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -501,15 +555,19 @@ inline bool supported(int N, int d, int b, int m, int dtype, int BH) {
   if (dtype != 1 && dtype != 2) return false;
   if (d % 8 != 0 || d > 128 || b > 128 || m > 128 || BH > 65535) return false;
   const int dt = d <= 64 ? 4 : 8, cm = m <= 32 ? 32 : (m <= 64 ? 64 : 128);
-  return r_smem_bytes(b, dt) <= (size_t)kMaxSmem && l_smem_bytes(m, cm, dt) <= (size_t)kMaxSmem;
+  return r_smem_bytes(b, dt, true) <= (size_t)kMaxSmem && l_smem_bytes(m, cm, dt, true) <= (size_t)kMaxSmem;
 }
+// From the third round on the states alpha_L and alpha_R are hi + lo pairs of f16 arrays: they feed
+// logits of size ~100, and with peaky logits their 2^-11 rounding, fed back round after round,
+// costs more than 1e-2 on the worst head from T = 3 on (measured; 2 rounds stay at 3e-3).
+inline bool uses_hilo(int T) { return T >= 3; }
 
 struct Ws {
-  __half *aL, *aR, *y;
+  __half *aL, *aR, *y, *aL_lo, *aR_lo;
   float* cL;
   size_t bytes;
 };
-inline Ws ws_layout(void* base, int BH, int N, int d) {
+inline Ws ws_layout(void* base, int BH, int N, int d, bool hilo) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
   Ws w;
   char* c = (char*)base;
@@ -519,10 +577,15 @@ inline Ws ws_layout(void* base, int BH, int N, int d) {
   w.aR = (__half*)(c + off); off += big;
   w.y = (__half*)(c + off); off += big;
   w.cL = (float*)(c + off); off += up((size_t)BH * N * 4);
+  w.aL_lo = w.aR_lo = nullptr;
+  if (hilo) {
+    w.aL_lo = (__half*)(c + off); off += big;
+    w.aR_lo = (__half*)(c + off); off += big;
+  }
   w.bytes = off;
   return w;
 }
-inline size_t workspace_bytes(int BH, int N, int d) { return ws_layout(nullptr, BH, N, d).bytes; }
+inline size_t workspace_bytes(int BH, int N, int d, int T) { return ws_layout(nullptr, BH, N, d, uses_hilo(T)).bytes; }
 
 struct Args {
   const void *Q, *K, *V;
@@ -532,43 +595,43 @@ struct Args {
   float scale;
 };
 
-template <typename TIn, int CB, int DT>
+template <typename TIn, int CB, int DT, bool HILO>
 inline int launch_r(const Args& a, const Ws& w, bool first, bool last, cudaStream_t st) {
-  auto kern = r_tile_kernel<TIn, CB, DT>;
-  const size_t smem = r_smem_bytes(a.b, DT);
+  auto kern = r_tile_kernel<TIn, CB, DT, HILO>;
+  const size_t smem = r_smem_bytes(a.b, DT, HILO);
   if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return 7;
   kern<<<dim3(a.m, a.BH), 32 * ((a.b + 15) / 16), smem, st>>>((const TIn*)a.Q, (const TIn*)a.K, (const TIn*)a.V, w.aR,
-                                                          w.aL, w.y, w.cL, a.N, a.d, a.b, a.scale, a.n_valid,
+                                                          w.aL, w.y, w.aR_lo, w.aL_lo, w.cL, a.N, a.d, a.b, a.scale, a.n_valid,
                                                           a.H, first ? 1 : 0, last ? 1 : 0);
   return 0;
 }
-template <typename TIn, int CM, int DT>
+template <typename TIn, int CM, int DT, bool HILO>
 inline int launch_l(const Args& a, const Ws& w, bool last, cudaStream_t st) {
-  auto kern = l_tile_kernel<TIn, CM, DT>;
-  const size_t smem = l_smem_bytes(a.m, CM, DT);
+  auto kern = l_tile_kernel<TIn, CM, DT, HILO>;
+  const size_t smem = l_smem_bytes(a.m, CM, DT, HILO);
   if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return 7;
-  kern<<<dim3(a.b, a.BH), 32 * ((a.m + 15) / 16), smem, st>>>((const TIn*)a.Q, w.aL, w.cL, w.y, w.aR, (TIn*)a.Y,
+  kern<<<dim3(a.b, a.BH), 32 * ((a.m + 15) / 16), smem, st>>>((const TIn*)a.Q, w.aL, w.cL, w.y, w.aR, w.aL_lo, w.aR_lo, (TIn*)a.Y,
                                                           last ? a.lse : nullptr, a.N, a.d, a.b, a.m, a.scale,
                                                           a.H, last ? 1 : 0);
   return 0;
 }
 
-template <typename TIn, int DT>
+template <typename TIn, int DT, bool HILO>
 inline int launch_td(const Args& a, void* ws, cudaStream_t st, int* launches) {
-  const Ws w = ws_layout(ws, a.BH, a.N, a.d);
+  const Ws w = ws_layout(ws, a.BH, a.N, a.d, HILO);
   int n = 0;
   for (int t = 1; t <= a.T; ++t) {
     const bool first = t == 1, last = t == a.T;
     int rc;
-    if (a.b <= 32) rc = launch_r<TIn, 32, DT>(a, w, first, last, st);
-    else if (a.b <= 64) rc = launch_r<TIn, 64, DT>(a, w, first, last, st);
-    else rc = launch_r<TIn, 128, DT>(a, w, first, last, st);
+    if (a.b <= 32) rc = launch_r<TIn, 32, DT, HILO>(a, w, first, last, st);
+    else if (a.b <= 64) rc = launch_r<TIn, 64, DT, HILO>(a, w, first, last, st);
+    else rc = launch_r<TIn, 128, DT, HILO>(a, w, first, last, st);
     if (rc != 0) return rc;
-    if (a.m <= 32) rc = launch_l<TIn, 32, DT>(a, w, last, st);
-    else if (a.m <= 64) rc = launch_l<TIn, 64, DT>(a, w, last, st);
-    else rc = launch_l<TIn, 128, DT>(a, w, last, st);
+    if (a.m <= 32) rc = launch_l<TIn, 32, DT, HILO>(a, w, last, st);
+    else if (a.m <= 64) rc = launch_l<TIn, 64, DT, HILO>(a, w, last, st);
+    else rc = launch_l<TIn, 128, DT, HILO>(a, w, last, st);
     if (rc != 0) return rc;
     n += 2;
   }
@@ -577,11 +640,15 @@ inline int launch_td(const Args& a, void* ws, cudaStream_t st, int* launches) {
   return 0;
 }
 
+template <typename TIn, bool HILO>
+inline int launch_h(const Args& a, void* ws, cudaStream_t st, int* launches) {
+  return a.d <= 64 ? launch_td<TIn, 4, HILO>(a, ws, st, launches) : launch_td<TIn, 8, HILO>(a, ws, st, launches);
+}
 inline int launch(const Args& a, int dtype, void* ws, cudaStream_t st, int* launches) {
   if (dtype == 1)
-    return a.d <= 64 ? launch_td<__half, 4>(a, ws, st, launches) : launch_td<__half, 8>(a, ws, st, launches);
-  return a.d <= 64 ? launch_td<__nv_bfloat16, 4>(a, ws, st, launches)
-                   : launch_td<__nv_bfloat16, 8>(a, ws, st, launches);
+    return uses_hilo(a.T) ? launch_h<__half, true>(a, ws, st, launches) : launch_h<__half, false>(a, ws, st, launches);
+  return uses_hilo(a.T) ? launch_h<__nv_bfloat16, true>(a, ws, st, launches)
+                        : launch_h<__nv_bfloat16, false>(a, ws, st, launches);
 }
 
 }  // namespace tile

@@ -132,12 +132,16 @@ def test_bf16_block_32_keeps_alpha_l_as_hi_lo_pair(T):
     assert need_bf16 - need_f16 == 2 * 12 * w.N * w.d * 2
 
 
-def test_auto_keeps_bf16_block_32_with_three_rounds_on_fp32_states():
-    """From T = 3 on, bf16 alpha_R costs 4e-2 on the worst head of this recipe on the tensor path
-    (hi + lo covers alpha_L only); AUTO must take the fp32-state kernels there."""
+def test_auto_takes_bf16_block_32_with_three_rounds_off_the_tcgen05_path():
+    """From T = 3 on, bf16 alpha_R costs 4e-2 on the worst head of this recipe on the tcgen05 path
+    (hi + lo covers alpha_L only); AUTO must take the tile kernels there, which keep both states as
+    hi + lo pairs of f16 from the third round on (plain f16 states: 1.2e-2 at T = 3, 3.3e-2 at T = 4)."""
     w = wl.WORKLOADS["C3"]
     err = check(2, 12, w.N, w.d, w.b, 3, "bf16", w.rank, w.s, seed=703)
     assert err < 5e-3
+    assert binding.monarch_attn_last_launch_count() == 6
+    err = check(2, 12, w.N, w.d, w.b, 4, "bf16", w.rank, w.s, seed=703, path=binding.MA_PATH_TILE_MMA)
+    assert err < 1e-2
 
 
 def test_tensor_kernel_generations_agree():
