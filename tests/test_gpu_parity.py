@@ -231,14 +231,15 @@ def test_general_fused_kernel_many_heads_and_agreement_with_the_special_case():
         assert float((a - b_).norm() / b_.norm()) <= 2e-3
 
 
-@pytest.mark.parametrize("name", ["S1", "S2"])
-def test_general_fused_kernel_on_the_profiled_short_workloads(name):
-    """The two extra workloads bench.py can time, at full size, every head against the oracle."""
+@pytest.mark.parametrize("name", ["S1", "S2", "S3", "S4"])
+def test_extra_workloads_at_full_size(name):
+    """The extra workloads bench.py can time (fused kernel: S1, S2; tile kernels: S3, S4), at full
+    size, every head against the oracle."""
     w = wl.EXTRA_WORKLOADS[name]
     Q, K, V = wl.make_workload_inputs(w)
     Qd, Kd, Vd = (binding.to_device(x, w.dtype) for x in (Q, K, V))
     Y = binding.monarch_attn_fwd(Qd, Kd, Vd, w.b, w.T).float().cpu().numpy().astype(np.float64)
-    assert binding.monarch_attn_last_launch_count() == 1
+    assert binding.monarch_attn_last_launch_count() == (1 if name in ("S1", "S2") else 2 * w.T)
     ref = mo.monarch_attention(Q, K, V, w.b, w.T)
     err = (np.linalg.norm((Y - ref).reshape(w.BH, -1), axis=1)
            / np.linalg.norm(ref.reshape(w.BH, -1), axis=1))
@@ -324,6 +325,32 @@ def test_tile_mma_path_matches_oracle(N, b, d, T, dtype):
     rank, s = (min(8, d), 1.0) if T <= 2 else (min(16, d), 1.5)
     check(1, 3, N, d, b, T, dtype, rank=rank, s=s, seed=N + T, path=binding.MA_PATH_TILE_MMA)
     assert binding.monarch_attn_last_launch_count() == 2 * T
+
+
+def test_tile_mma_path_is_deterministic_and_stays_inside_its_buffers():
+    Q, K, V = wl.make_qkv(1, 5, 1089, 24, "f16", 8, 1.0, seed=6)          # 33 blocks of 33, d = 24
+    Qd, Kd, Vd = (binding.to_device(x, "f16") for x in (Q, K, V))
+    n, pad = Qd.numel(), 4096
+    for T in (2, 3):                                                        # plain and hi + lo states
+        need = binding.monarch_attn_workspace_bytes(1, 5, 1089, 24, 33, T, Qd.dtype, binding.MA_PATH_TILE_MMA)
+        assert need > 0
+        buf = torch.full((n + 2 * pad,), 7.0, dtype=Qd.dtype, device="cuda")
+        Y = buf[pad:pad + n].view_as(Qd)
+        wsbuf = torch.full((need + 2 * pad,), 0x5A, dtype=torch.uint8, device="cuda")
+        off = (-wsbuf.data_ptr()) % 256 + 256
+        ws = wsbuf[off:off + need]
+        binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 33, T, path=binding.MA_PATH_TILE_MMA, workspace=ws, Y=Y)
+        torch.cuda.synchronize()
+        assert bool((buf[:pad] == 7.0).all()) and bool((buf[pad + n:] == 7.0).all())
+        assert bool((wsbuf[:off] == 0x5A).all()) and bool((wsbuf[off + need:] == 0x5A).all())
+        first = Y.clone()
+        for _ in range(5):
+            binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 33, T, path=binding.MA_PATH_TILE_MMA, workspace=ws, Y=Y)
+            assert torch.equal(Y, first)
+        # a too-small workspace is refused
+        with pytest.raises(binding.MonarchAttnError) as e:
+            binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 33, T, path=binding.MA_PATH_TILE_MMA, workspace=ws[:need - 256])
+        assert e.value.code == 6
 
 
 def test_tile_mma_path_is_the_16_bit_default_where_no_other_tensor_core_kernel_applies():
