@@ -46,6 +46,14 @@ constexpr float kMasked = -1e30f;   // logit of a masked column: exp2(kMasked - 
 // in 8 different 16-byte bank groups.
 __host__ __device__ constexpr int pitch_of(int dt) { return dt * 32 + 16; }
 
+// The half-step kernels of a call are launched with programmatic stream serialisation: the next
+// launch's CTAs may take SM slots as this launch's last CTAs drain, but they touch no memory before
+// every CTA of the launch before them has finished (wait), so the stream order of the data holds.
+__device__ __forceinline__ void grid_dependency_sync() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Rows of head h in Q, K, V, Y: element offset of row 0 and the stride between rows.
 struct HeadRows {
   size_t base, stride;
@@ -148,6 +156,7 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
               int last) {
   extern __shared__ __align__(128) uint8_t smem[];
   constexpr int kPitch = pitch_of(DT);
+  grid_dependency_sync();
   const int k = blockIdx.x, h = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int rb = round16(b);
@@ -325,6 +334,7 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
               int m, float scale, int H, int last) {
   extern __shared__ __align__(128) uint8_t smem[];
   constexpr int kPitch = pitch_of(DT), kPPitch = CM * 2 + 16;
+  grid_dependency_sync();
   const int j = blockIdx.x, h = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int rm = round16(m);
@@ -587,6 +597,21 @@ inline Ws ws_layout(void* base, int BH, int N, int d, bool hilo) {
 }
 inline size_t workspace_bytes(int BH, int N, int d, int T) { return ws_layout(nullptr, BH, N, d, uses_hilo(T)).bytes; }
 
+// Launch configuration with programmatic stream serialisation (see grid_dependency_sync).
+inline cudaLaunchConfig_t serialised_config(dim3 grid, int threads, size_t smem, cudaStream_t st) {
+  static cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cfg;
+}
+
 struct Args {
   const void *Q, *K, *V;
   void* Y;
@@ -601,10 +626,12 @@ inline int launch_r(const Args& a, const Ws& w, bool first, bool last, cudaStrea
   const size_t smem = r_smem_bytes(a.b, DT, HILO);
   if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return 7;
-  kern<<<dim3(a.m, a.BH), 32 * ((a.b + 15) / 16), smem, st>>>((const TIn*)a.Q, (const TIn*)a.K, (const TIn*)a.V, w.aR,
-                                                          w.aL, w.y, w.aR_lo, w.aL_lo, w.cL, a.N, a.d, a.b, a.scale, a.n_valid,
-                                                          a.H, first ? 1 : 0, last ? 1 : 0);
-  return 0;
+  cudaLaunchConfig_t cfg = serialised_config(dim3(a.m, a.BH), 32 * ((a.b + 15) / 16), smem, st);
+  return cudaLaunchKernelEx(&cfg, kern, (const TIn*)a.Q, (const TIn*)a.K, (const TIn*)a.V, (const __half*)w.aR,
+                            w.aL, w.y, (const __half*)w.aR_lo, w.aL_lo, w.cL, a.N, a.d, a.b, a.scale, a.n_valid,
+                            a.H, first ? 1 : 0, last ? 1 : 0) == cudaSuccess
+             ? 0
+             : 7;
 }
 template <typename TIn, int CM, int DT, bool HILO>
 inline int launch_l(const Args& a, const Ws& w, bool last, cudaStream_t st) {
@@ -612,10 +639,13 @@ inline int launch_l(const Args& a, const Ws& w, bool last, cudaStream_t st) {
   const size_t smem = l_smem_bytes(a.m, CM, DT, HILO);
   if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return 7;
-  kern<<<dim3(a.b, a.BH), 32 * ((a.m + 15) / 16), smem, st>>>((const TIn*)a.Q, w.aL, w.cL, w.y, w.aR, w.aL_lo, w.aR_lo, (TIn*)a.Y,
-                                                          last ? a.lse : nullptr, a.N, a.d, a.b, a.m, a.scale,
-                                                          a.H, last ? 1 : 0);
-  return 0;
+  cudaLaunchConfig_t cfg = serialised_config(dim3(a.b, a.BH), 32 * ((a.m + 15) / 16), smem, st);
+  return cudaLaunchKernelEx(&cfg, kern, (const TIn*)a.Q, (const __half*)w.aL, (const float*)w.cL,
+                            (const __half*)w.y, w.aR, (const __half*)w.aL_lo, w.aR_lo, (TIn*)a.Y,
+                            last ? a.lse : (float*)nullptr, a.N, a.d, a.b, a.m, a.scale, a.H, last ? 1 : 0) ==
+                 cudaSuccess
+             ? 0
+             : 7;
 }
 
 template <typename TIn, int DT, bool HILO>
