@@ -73,6 +73,24 @@ static GenericWs generic_layout(const Problem& p, void* base) {
   return w;
 }
 
+// Launch with programmatic stream serialisation (the kernels wait for the launch before them
+// themselves: generic::grid_dependency_sync).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_serialised(void (*kern)(KArgs...), dim3 grid, int threads, size_t smem,
+                                     cudaStream_t st, Args... args) {
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 template <typename TIn>
 static int launch_generic_t(const Problem& p, const TIn* Q, const TIn* K, const TIn* V, TIn* Y,
                             float scale, const GenericWs& w, cudaStream_t st) {
@@ -90,9 +108,10 @@ static int launch_generic_t(const Problem& p, const TIn* Q, const TIn* K, const 
   do {                                                                                         \
     if (set_smem((const void*)r_step_kernel<TIn, FIRST, WITHV>, rs) != cudaSuccess)            \
       return MA_ERR_CUDA;                                                                      \
-    r_step_kernel<TIn, FIRST, WITHV><<<gr, kThreads, rs, st>>>(Q, K, V, w.aR, w.cR, w.aL,     \
-                                                                w.cL, w.y, p.N, p.d, p.b, p.m, \
-                                                                scale, p.n_valid, p.H);        \
+    if (launch_serialised(r_step_kernel<TIn, FIRST, WITHV>, gr, kThreads, rs, st, Q, K, V, w.aR, \
+                          w.cR, w.aL, w.cL, w.y, p.N, p.d, p.b, p.m, scale, p.n_valid,          \
+                          p.H) != cudaSuccess)                                                  \
+      return MA_ERR_CUDA;                                                                       \
   } while (0)
     if (first && last) MA_LAUNCH_R(true, true);
     else if (first) MA_LAUNCH_R(true, false);
@@ -103,12 +122,14 @@ static int launch_generic_t(const Problem& p, const TIn* Q, const TIn* K, const 
     size_t ls = l_step_smem_floats(p.m, p.d, last) * 4;
     if (last) {
       if (set_smem((const void*)l_step_kernel<TIn, true>, ls) != cudaSuccess) return MA_ERR_CUDA;
-      l_step_kernel<TIn, true><<<gl, kThreads, ls, st>>>(Q, w.aL, w.cL, w.y, w.aR, w.cR, Y, p.N,
-                                                         p.d, p.b, p.m, scale, p.H, p.lse);
+      if (launch_serialised(l_step_kernel<TIn, true>, gl, kThreads, ls, st, Q, w.aL, w.cL, w.y, w.aR, w.cR, Y,
+                            p.N, p.d, p.b, p.m, scale, p.H, p.lse) != cudaSuccess)
+        return MA_ERR_CUDA;
     } else {
       if (set_smem((const void*)l_step_kernel<TIn, false>, ls) != cudaSuccess) return MA_ERR_CUDA;
-      l_step_kernel<TIn, false><<<gl, kThreads, ls, st>>>(Q, w.aL, w.cL, w.y, w.aR, w.cR, Y, p.N,
-                                                          p.d, p.b, p.m, scale, p.H, nullptr);
+      if (launch_serialised(l_step_kernel<TIn, false>, gl, kThreads, ls, st, Q, w.aL, w.cL, w.y, w.aR, w.cR, Y,
+                            p.N, p.d, p.b, p.m, scale, p.H, (float*)nullptr) != cudaSuccess)
+        return MA_ERR_CUDA;
     }
     ++launches;
   }

@@ -30,6 +30,14 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// The half-step kernels are launched with programmatic stream serialisation: the next launch's
+// CTAs may take SM slots while this launch's last CTAs drain, but they touch no memory before every
+// CTA of the launch before them has finished.
+__device__ __forceinline__ void grid_dependency_sync() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 
@@ -61,6 +69,7 @@ r_step_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
               float* __restrict__ aL, float* __restrict__ cL, float* __restrict__ y,
               int N, int d, int b, int m, float scale, int n_valid, int H) {
   extern __shared__ float smem[];
+  grid_dependency_sync();
   const int k = blockIdx.x, h = blockIdx.y;
   const int dp = d + 1;
   float* Ks = smem;                                  // [b][d+1]
@@ -143,6 +152,7 @@ l_step_kernel(const TIn* __restrict__ Q, const float* __restrict__ aL, const flo
               TIn* __restrict__ Y, int N, int d, int b, int m, float scale, int H,
               float* __restrict__ row_lse) {
   extern __shared__ float smem[];
+  grid_dependency_sync();
   const int j = blockIdx.x, h = blockIdx.y;
   const int dp = d + 1, mp = m + 1;
   float* As = smem;                                  // aL[j]: [m][d+1]
