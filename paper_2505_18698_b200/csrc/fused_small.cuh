@@ -82,6 +82,8 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
                     int n_valid, int H, float* __restrict__ lse) {
   typedef __half T;
   extern __shared__ uint8_t smem_raw[];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int tile = N * kRowBytes;
   uint8_t* sQ = smem;
@@ -531,9 +533,23 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
     return 7;
-  kern<<<BH, threads, smem, st>>>((const TIn*)Q, (const TIn*)K, (const TIn*)V, (TIn*)Y, N, d, b, m, T,
-                                   scale, n_valid, H, lse);
-  return cudaGetLastError() == cudaSuccess ? 0 : 7;
+  // programmatic stream serialisation: when calls follow one another on a stream, the CTAs of the
+  // next call take SM slots while the last wave of this one drains (they touch no memory before
+  // this launch has finished: the kernel starts with griddepcontrol.wait)
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(BH);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, (const TIn*)Q, (const TIn*)K, (const TIn*)V, (TIn*)Y, N, d, b, m, T, scale,
+                            n_valid, H, lse) == cudaSuccess
+             ? 0
+             : 7;
 }
 
 template <typename TIn>
