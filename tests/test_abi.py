@@ -40,6 +40,45 @@ def test_workspace_query(lib):
     assert wb(1, 1, 256, 64, 16, 1, binding.MA_F32, binding.MA_PATH_TENSOR) == 0   # fp32 has no tensor path
 
 
+def test_binding_constants_match_the_header():
+    import os
+    import re
+    here = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    text = open(os.path.join(here, "include", "monarch_attn.h")).read()
+    enums = {name: int(val) for name, val in re.findall(r"\b(MA_[A-Z0-9_]+)\s*=\s*(\d+)", text)}
+    assert len(enums) >= 20
+    for name, val in enums.items():
+        if hasattr(binding, name):
+            assert getattr(binding, name) == val, name
+    for name in ("MA_PATH_AUTO", "MA_PATH_GENERIC", "MA_PATH_TENSOR", "MA_PATH_FUSED", "MA_PATH_FUSED_SMALL",
+                 "MA_PATH_TILE_MMA", "MA_F32", "MA_F16", "MA_BF16"):
+        assert name in enums and hasattr(binding, name), name
+    assert len({v for k, v in enums.items() if k.startswith("MA_PATH_")}) == \
+        len([k for k in enums if k.startswith("MA_PATH_")])
+
+
+def test_workspace_query_of_the_fused_and_tile_paths(lib):
+    wb = lib.monarch_attn_workspace_bytes
+    F16, BF16 = binding.MA_F16, binding.MA_BF16
+    # fused per-head kernel: only a status block; shapes outside its limits are refused
+    assert wb(64, 12, 210, 64, 14, 2, F16, binding.MA_PATH_FUSED_SMALL) == 256
+    assert wb(1, 1, 480, 64, 24, 2, F16, binding.MA_PATH_FUSED_SMALL) == 0       # 4 tiles do not fit
+    assert wb(1, 1, 480, 64, 24, 1, F16, binding.MA_PATH_FUSED_SMALL) == 256
+    assert wb(1, 1, 480, 64, 12, 1, F16, binding.MA_PATH_FUSED_SMALL) == 0       # m = 40 > 32
+    assert wb(1, 1, 210, 64, 14, 2, binding.MA_F32, binding.MA_PATH_FUSED_SMALL) == 0
+    # tile kernels: three f16 states + c_L, two more states from the third round on
+    n = 2 * 16 * 8192 * 64
+    w2 = wb(2, 16, 8192, 64, 64, 2, BF16, binding.MA_PATH_TILE_MMA)
+    w3 = wb(2, 16, 8192, 64, 64, 3, BF16, binding.MA_PATH_TILE_MMA)
+    assert 3 * 2 * n <= w2 < 3 * 2 * n + 4 * n // 64 + 4096
+    assert w3 - w2 == 2 * 2 * n
+    assert wb(1, 1, 8192, 64, 32, 1, F16, binding.MA_PATH_TILE_MMA) == 0         # m = 256 > 128
+    assert wb(1, 1, 2048, 136, 32, 1, F16, binding.MA_PATH_TILE_MMA) == 0        # d > 128
+    # AUTO: a generic-sized workspace is never smaller than what AUTO needs for 16-bit inputs
+    for (N, d, b, T) in [(210, 64, 14, 2), (8192, 64, 64, 1), (7680, 48, 128, 3), (4096, 64, 64, 2)]:
+        assert 0 < wb(1, 2, N, d, b, T, F16, binding.MA_PATH_AUTO) <= wb(1, 2, N, d, b, T, F16, binding.MA_PATH_GENERIC)
+
+
 def test_host_side_validation_returns_before_any_launch(lib):
     f = lib.monarch_attn_fwd_ex
     p = ctypes.c_void_p
