@@ -526,6 +526,7 @@ def test_bounded_wait_runs_out_and_reports_timeout():
     (1000, 32, 64, 2, "bf16"),   # N' = 1024
     (380, 24, 64, 1, "f32"),     # m = 16 != b
     (61, 8, 16, 2, "f32"), (64, 8, 16, 2, "f32"),   # ragged and exact
+    (250, 16, 64, 2, "f16"), (380, 24, 64, 2, "bf16"), (383, 16, 64, 1, "f16"),   # fused kernel, 16 warps per CTA
     (4040, 64, 64, 2, "bf16"), (4033, 64, 64, 1, "f16"), (4095, 64, 64, 3, "bf16"),   # tensor kernel, N' = 4096
     (16300, 128, 64, 1, "f16"), (16257, 128, 64, 2, "bf16"),                          # N' = 16384
 ])
