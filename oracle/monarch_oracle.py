@@ -32,6 +32,13 @@ Readings taken where the paper is silent:
     beyond ~745.  Such a row gets Z_R = 0 and the event is counted.
   * Padding (App. C.3): with n_valid < N, key columns b*k+i >= n_valid get
     omega = -inf added to Z_R (post-padding).
+  * Batched sequences of different lengths (App. C.3 names the case, gives no
+    formula): a block lying wholly in the padding has no admissible R row
+    (softmax of all -inf).  Reading: such a block is absent from the
+    sequence's problem -- R = 0 there, Z_L = -inf for it as a key block (so
+    the rows of M still sum to one over valid keys), and as a query block it
+    is left out of the sums over l of Eq. 9.  Pin: the valid rows equal those
+    of the same sequence run alone at its own padded length.
 
 Pins (tests/test_oracle_pins.py): the dense Monarch matrix of Eq. 5 and
 M = P^T B; the printed permutation example of App. B; row-stochasticity;
@@ -74,49 +81,95 @@ def _key_mask(m, b, n_valid):
 
 
 # --------------------------------------------------------------------------- updates
-def r_update(L, Qb, Kb, omega=None, stats=None):
-    """Eq. 7 with Eq. 9.  Returns R[k,j,i] and log R[k,j,i]."""
-    aR = np.einsum("jkl,jlv->kjv", L, Qb)                  # alpha_R
-    cR = np.einsum("jkl->kj", L)                           # c_R
-    betaR = np.einsum("kjv,kiv->kji", aR, Kb)              # beta_R
-    zero = cR == 0.0
-    if stats is not None:
-        stats["min_cR"] = min(stats.get("min_cR", np.inf), float(cR.min()))
-        stats["cR_zero_rows"] = stats.get("cR_zero_rows", 0) + int(zero.sum())
-    ZR = np.where(zero[:, :, None], 0.0, betaR / np.where(zero, 1.0, cR)[:, :, None])
-    if omega is not None:
-        ZR = ZR + omega[:, None, :]
-    zmax = ZR.max(axis=2, keepdims=True)
-    lse = zmax + np.log(np.exp(ZR - zmax).sum(axis=2, keepdims=True))
-    logR = ZR - lse
-    R = np.exp(logR)
+# Every contraction below is written per block, as a plain 2-D matrix product over the block's own
+# index pair: "for each key block k" or "for each in-block position j", exactly the batching the
+# equations state.  Nothing is fused or reordered beyond that.
+def _softmax_rows(Z, axis):
+    """softmax and log-softmax along `axis`, max-subtracted; an all -inf slice gives zeros."""
+    zmax = Z.max(axis=axis, keepdims=True)
+    dead = ~np.isfinite(zmax)                       # slice with no admissible entry
+    shifted = Z - np.where(dead, 0.0, zmax)
+    lse = np.log(np.exp(shifted).sum(axis=axis, keepdims=True), where=~dead,
+                 out=np.zeros_like(zmax)) + np.where(dead, 0.0, zmax)
+    logS = np.where(dead, -np.inf, Z - lse)
+    return np.exp(logS), logS
+
+
+def r_update(L, Qb, Kb, omega=None, stats=None, m_live=None):
+    """Eq. 7 with Eq. 9.  Returns R[k,j,i] and log R[k,j,i].
+
+    `m_live` (batched sequences of different lengths, App. C.3): blocks from m_live on lie wholly in
+    the padding; every key of such a block is masked, so it has no admissible R row.  Reading: those
+    blocks are absent from the sequence's problem, as key blocks (R = 0) and as query blocks (no
+    term in the sums over l of Eq. 9); their rows of Q, K are never touched."""
+    b, m, _ = L.shape
+    d = Qb.shape[2]
+    live = m if m_live is None else m_live
+    alpha_R = np.zeros((m, b, d))
+    c_R = np.zeros((m, b))
+    for j in range(b):                              # Eq. 9, position j: [k,l] x [l,v]
+        alpha_R[:live, j, :] = L[j][:live, :live] @ Qb[j][:live]
+        c_R[:live, j] = L[j][:live, :live].sum(axis=1)
+    R = np.zeros((m, b, b))
+    logR = np.full((m, b, b), -np.inf)
+    for k in range(live):                           # Eq. 7, key block k: [j,v] x [v,i]
+        beta_R = alpha_R[k] @ Kb[k].T
+        zero = c_R[k] == 0.0
+        if stats is not None:
+            stats["min_cR"] = min(stats.get("min_cR", np.inf), float(c_R[k].min()))
+            stats["cR_zero_rows"] = stats.get("cR_zero_rows", 0) + int(zero.sum())
+        Z_R = np.where(zero[:, None], 0.0, beta_R / np.where(zero, 1.0, c_R[k])[:, None])
+        if omega is not None:
+            Z_R = Z_R + omega[k][None, :]
+        R[k], logR[k] = _softmax_rows(Z_R, axis=1)
     return R, logR
 
 
-def l_update(R, logR, Qb, Kb):
-    """Eq. 8 with Eq. 10.  Returns L[j,k,l]."""
-    aL = np.einsum("kji,kiv->jkv", R, Kb)                  # alpha_L
-    RlogR = np.where(R > 0.0, R * np.where(R > 0.0, logR, 0.0), 0.0)   # 0 log 0 = 0
-    cL = np.einsum("kji->jk", RlogR)                       # c_L
-    betaL = np.einsum("jkv,jlv->jkl", aL, Qb)              # beta_L
-    ZL = betaL - cL[:, :, None]
-    ZL = ZL - ZL.max(axis=1, keepdims=True)
-    E = np.exp(ZL)
-    return E / E.sum(axis=1, keepdims=True)                # softmax over k
+def l_update(R, logR, Qb, Kb, m_live=None):
+    """Eq. 8 with Eq. 10.  Returns L[j,k,l].
+
+    `m_live`: see r_update.  An absent key block has Z_L = -inf, i.e. L[j,k,:] = 0, so that the
+    rows of M still sum to one over the valid keys; an absent query block has L[j,:,l] = 0."""
+    m, b, _ = R.shape
+    d = Kb.shape[2]
+    live = m if m_live is None else m_live
+    alpha_L = np.zeros((b, m, d))
+    c_L = np.zeros((b, m))
+    for k in range(live):                           # Eq. 10, key block k: [j,i] x [i,v]
+        alpha_L[:, k, :] = R[k] @ Kb[k]
+        RlogR = np.where(R[k] > 0.0, R[k] * np.where(R[k] > 0.0, logR[k], 0.0), 0.0)   # 0 log 0 = 0
+        c_L[:, k] = RlogR.sum(axis=1)
+    L = np.zeros((b, m, m))
+    for j in range(b):                              # Eq. 8, position j: [k,v] x [v,l]
+        Z_L = alpha_L[j][:live] @ Qb[j][:live].T - c_L[j][:live, None]
+        L[j][:live, :live], _ = _softmax_rows(Z_L, axis=0)        # over k for every l
+    return L
 
 
-def monarch_multiply(L, R, Vb):
-    """Eq. 4: O[b*l+j,:] = sum_k L[j,k,l] * (sum_i R[k,j,i] Vb[k,i,:])."""
+def monarch_multiply(L, R, Vb, m_live=None):
+    """Eq. 4: O[b*l+j,:] = sum_k L[j,k,l] * (sum_i R[k,j,i] Vb[k,i,:]).  Rows of absent blocks
+    (`m_live`, see r_update) are zero."""
     b, m, _ = L.shape
-    y = np.einsum("kji,kiv->jkv", R, Vb)
-    z = np.einsum("jkl,jkv->ljv", L, y)                    # row b*l+j
-    return z.reshape(m * b, Vb.shape[2])
+    dv = Vb.shape[2]
+    live = m if m_live is None else m_live
+    y = np.zeros((b, m, dv))
+    for k in range(live):                           # first factor, key block k: [j,i] x [i,v]
+        y[:, k, :] = R[k] @ Vb[k]
+    O = np.zeros((m, b, dv))                        # [l, j, v] = row b*l + j
+    for j in range(b):                              # second factor, position j: [l,k] x [k,v]
+        O[:live, j, :] = L[j][:live, :live].T @ y[j][:live]
+    return O.reshape(m * b, dv)
 
 
 # --------------------------------------------------------------------------- one head
 def monarch_attention_head(Q, K, V, b, T, scale=None, n_valid=None,
                            return_factors=False, stats=None, trace=None):
     """One head.  Q, K: (N, d); V: (N, dv); returns O (N, dv) in float64.
+
+    n_valid (App. C.3, post-padding): keys b*k+i >= n_valid are masked.  With less than one block
+    of padding this is the appendix's case.  With more (a sequence of a padded batch), the blocks
+    that lie wholly in the padding are absent from the sequence's problem: see r_update / l_update;
+    rows of O from ceil(n_valid/b)*b on are zero.
 
     `trace`, if a list, receives (name, L.copy(), R.copy()) after every
     half-step (used by the ascent pin)."""
@@ -132,25 +185,34 @@ def monarch_attention_head(Q, K, V, b, T, scale=None, n_valid=None,
     if scale is None:
         scale = 1.0 / np.sqrt(d)
     Qb, Kb, Vb = block_views(Q, K, V, b, scale)
-    omega = None if n_valid is None or n_valid >= N else _key_mask(m, b, n_valid)
+    omega = None
+    m_live = m
+    if n_valid is not None and n_valid < N:
+        if n_valid < 1:
+            raise ValueError("n_valid must be >= 1")
+        omega = _key_mask(m, b, n_valid)
+        m_live = -(-n_valid // b)
 
-    L = np.broadcast_to(np.eye(m), (b, m, m)).copy()       # L^(0)[j,k,l] = delta_kl
+    L = np.zeros((b, m, m))
+    L[:, np.arange(m_live), np.arange(m_live)] = 1.0       # L^(0)[j,k,l] = delta_kl
     R = logR = None
     for _ in range(T):
-        R, logR = r_update(L, Qb, Kb, omega, stats)
+        R, logR = r_update(L, Qb, Kb, omega, stats, m_live)
         if trace is not None:
             trace.append(("R", L.copy(), R.copy()))
-        L = l_update(R, logR, Qb, Kb)
+        L = l_update(R, logR, Qb, Kb, m_live)
         if trace is not None:
             trace.append(("L", L.copy(), R.copy()))
-    O = monarch_multiply(L, R, Vb)
+    O = monarch_multiply(L, R, Vb, m_live)
     if return_factors:
         return O, L, R
     return O
 
 
 def monarch_attention(Q, K, V, b, T, scale=None, n_valid=None):
-    """Batched: Q, K, V of shape (..., N, d); heads are independent (Sec. 2)."""
+    """Batched: Q, K, V of shape (..., N, d); heads are independent (Sec. 2).  n_valid: None, one
+    length for all, or an array of lengths with the shape of the leading axes (or of the first of
+    them: one length per batch entry)."""
     Q = np.asarray(Q)
     lead = Q.shape[:-2]
     N, d = Q.shape[-2:]
@@ -158,17 +220,25 @@ def monarch_attention(Q, K, V, b, T, scale=None, n_valid=None):
     Qf = np.asarray(Q).reshape(-1, N, d)
     Kf = np.asarray(K).reshape(-1, N, d)
     Vf = np.asarray(V).reshape(-1, N, dv)
+    if n_valid is None or np.ndim(n_valid) == 0:
+        nv = [n_valid] * Qf.shape[0]
+    else:
+        nva = np.asarray(n_valid)
+        if nva.shape != lead:                       # one length per batch entry
+            nva = np.broadcast_to(nva.reshape(nva.shape + (1,) * (len(lead) - nva.ndim)), lead)
+        nv = [int(x) for x in nva.reshape(-1)]
     out = np.empty((Qf.shape[0], N, dv), dtype=np.float64)
     for h in range(Qf.shape[0]):
-        out[h] = monarch_attention_head(Qf[h], Kf[h], Vf[h], b, T, scale, n_valid)
+        out[h] = monarch_attention_head(Qf[h], Kf[h], Vf[h], b, T, scale, nv[h])
     return out.reshape(*lead, N, dv)
 
 
 # --------------------------------------------------------------------------- state form
 def monarch_attention_state_form_head(Q, K, V, b, T, scale=None):
-    """The same recursion carried by the states (alpha, c) only, L and R living
-    just inside one half-step (Sec. 3 'Implementation', Fig. 4).  A second
-    statement of the algorithm used as a cross-check of the first."""
+    """The same recursion carried by the states (alpha, c) only (Sec. 3 'Implementation'): the
+    factors live only inside one half-step, a key block at a time (R) or a position at a time (L).
+    A second statement of the algorithm, used as a cross-check of the first: its only state between
+    half-steps is alpha_R, c_R (k-major) or alpha_L, c_L, y (j-major)."""
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
@@ -176,32 +246,40 @@ def monarch_attention_state_form_head(Q, K, V, b, T, scale=None):
     m = N // b
     if scale is None:
         scale = 1.0 / np.sqrt(d)
-    Qb, Kb, Vb = block_views(Q, K, V, b, scale)
-
-    # L^(0) = identity  =>  alpha_R^(1)[k,j,:] = Qb[j,k,:],  c_R^(1) = 1
-    aR = Qb.transpose(1, 0, 2).copy()
-    cR = np.ones((m, b))
-    out = None
+    Qs = scale * Q
+    dv = V.shape[1]
+    # L^(0) = identity  =>  alpha_R^(1)[k,j,:] = Qs[b*k + j],  c_R^(1) = 1
+    alpha_R = Qs.reshape(m, b, d).copy()
+    c_R = np.ones((m, b))
+    O = np.empty((N, dv))
     for t in range(1, T + 1):
-        # alpha_R, c_R -> alpha_L, c_L (and y on the last step)
-        ZR = np.einsum("kjv,kiv->kji", aR, Kb) / cR[:, :, None]
-        ZR = ZR - ZR.max(axis=2, keepdims=True)
-        R = np.exp(ZR)
-        R = R / R.sum(axis=2, keepdims=True)
-        with np.errstate(divide="ignore", invalid="ignore"):
-            cL = np.where(R > 0, R * np.log(R), 0.0).sum(axis=2).T      # [j,k]
-        aL = np.einsum("kji,kiv->jkv", R, Kb)
-        ZL = np.einsum("jkv,jlv->jkl", aL, Qb) - cL[:, :, None]
-        ZL = ZL - ZL.max(axis=1, keepdims=True)
-        Lf = np.exp(ZL)
-        Lf = Lf / Lf.sum(axis=1, keepdims=True)
-        if t < T:
-            aR = np.einsum("jkl,jlv->kjv", Lf, Qb)
-            cR = Lf.sum(axis=2).T
-        else:
-            y = np.einsum("kji,kiv->jkv", R, Vb)
-            out = np.einsum("jkl,jkv->ljv", Lf, y).reshape(N, Vb.shape[2])
-    return out
+        alpha_L = np.empty((b, m, d))
+        c_L = np.empty((b, m))
+        y = np.empty((b, m, dv))
+        for k in range(m):                          # R half-step of key block k
+            Kk = K[b * k:b * (k + 1)]
+            Z = (alpha_R[k] @ Kk.T) / c_R[k][:, None]
+            Z = Z - Z.max(axis=1, keepdims=True)
+            E = np.exp(Z)
+            s = E.sum(axis=1, keepdims=True)
+            Rk = E / s
+            with np.errstate(divide="ignore", invalid="ignore"):
+                c_L[:, k] = np.where(Rk > 0, Rk * (Z - np.log(s)), 0.0).sum(axis=1)
+            alpha_L[:, k, :] = Rk @ Kk
+            if t == T:
+                y[:, k, :] = Rk @ V[b * k:b * (k + 1)]
+        for j in range(b):                          # L half-step of position j
+            Qj = Qs[j::b]                           # rows b*l + j, l = 0..m-1
+            Z = alpha_L[j] @ Qj.T - c_L[j][:, None]          # [k, l]
+            Z = Z - Z.max(axis=0, keepdims=True)
+            E = np.exp(Z)
+            Lj = E / E.sum(axis=0, keepdims=True)
+            if t < T:
+                alpha_R[:, j, :] = Lj @ Qj
+                c_R[:, j] = Lj.sum(axis=1)
+            else:
+                O[j::b] = Lj.T @ y[j]
+    return O
 
 
 # --------------------------------------------------------------------------- dense forms
@@ -250,20 +328,24 @@ def objective_dense(M, Q, K, scale):
 def final_row_lse(R, Q, K, b, scale):
     """Row-wise log-sum-exp of the logits of the L update that follows R (Eq. 8 with Eq. 10):
     lse[b*l + j] = log sum_k exp(Z_L[j,k,l]).  Because that update is the exact maximiser over L
-    (L = softmax_k Z_L, so Z_L - log L is constant in k) and every R[k,j,:] sums to one, the
-    objective of Eq. 6 at (L, R) is the plain sum of these N numbers; the pin is
-    test_objective_equals_sum_of_final_row_lse."""
+    (L = softmax_k Z_L, so Z_L - log L is constant in k) and every R[k,j,:] sums to one, row
+    b*l + j of M contributes exactly lse[b*l + j] to the objective of Eq. 6, and the objective is
+    the plain sum of these N numbers; pins: test_objective_equals_sum_of_final_row_lse (sum) and
+    test_final_row_lse_is_each_rows_own_term_of_the_objective (row by row)."""
     Q = np.asarray(Q, np.float64)
     K = np.asarray(K, np.float64)
     Qb, Kb, _ = block_views(Q, K, K, b, scale)
     m = Q.shape[0] // b
-    logR = np.where(R > 0.0, np.log(np.where(R > 0.0, R, 1.0)), 0.0)
-    aL = np.einsum("kji,kiv->jkv", R, Kb)
-    cL = np.einsum("kji->jk", np.where(R > 0.0, R * logR, 0.0))
-    ZL = np.einsum("jkv,jlv->jkl", aL, Qb) - cL[:, :, None]
-    zmax = ZL.max(axis=1)
-    lse = zmax + np.log(np.exp(ZL - zmax[:, None, :]).sum(axis=1))          # [j, l]
-    return lse.T.reshape(m * b)                                            # row b*l + j
+    lse = np.empty((m, b))                                                  # [l, j] = row b*l + j
+    for j in range(b):
+        alpha_L = np.stack([R[k, j] @ Kb[k] for k in range(m)])            # [k, v]
+        with np.errstate(divide="ignore", invalid="ignore"):
+            c_L = np.array([np.where(R[k, j] > 0, R[k, j] * np.log(R[k, j]), 0.0).sum()
+                            for k in range(m)])
+        Z_L = alpha_L @ Qb[j].T - c_L[:, None]                              # [k, l]
+        zmax = Z_L.max(axis=0)
+        lse[:, j] = zmax + np.log(np.exp(Z_L - zmax[None, :]).sum(axis=0))
+    return lse.reshape(m * b)
 
 
 def objective_factored(L, R, Q, K, scale):

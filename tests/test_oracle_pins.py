@@ -280,3 +280,65 @@ def test_objective_equals_sum_of_final_row_lse(N, b, T):
     lse = mo.final_row_lse(R, Q, K, b, scale)
     assert lse.shape == (N,)
     assert abs(lse.sum() - f_dense) < 1e-9 * max(1.0, abs(f_dense))
+
+
+@pytest.mark.parametrize("N,b,T", [(12, 4, 1), (12, 3, 2), (20, 2, 2), (18, 9, 2), (24, 6, 3)])
+def test_final_row_lse_is_each_rows_own_term_of_the_objective(N, b, T):
+    """Row r of the dense Monarch matrix contributes sum_c M[r,c] S[r,c] - sum_c M[r,c] log M[r,c]
+    to Eq. 6.  Because the final L is the exact maximiser, that term equals the log-sum-exp of row
+    r's L logits.  This pins the ROW ORDER of final_row_lse (row b*l + j), with m != b: a
+    transposed order passes the sum test above but not this one."""
+    rng = np.random.default_rng(N * 17 + b + T)
+    Q, K, V = (rng.standard_normal((N, 5)) * 1.3 for _ in range(3))
+    scale = 0.41
+    _, L, R = mo.monarch_attention_head(Q, K, V, b, T, scale=scale, return_factors=True)
+    M = mo.dense_monarch(L, R)
+    S = scale * Q @ K.T
+    with np.errstate(divide="ignore", invalid="ignore"):
+        ent = -np.where(M > 0, M * np.log(M), 0.0).sum(axis=1)
+    per_row = (M * S).sum(axis=1) + ent
+    lse = mo.final_row_lse(R, Q, K, b, scale)
+    assert np.allclose(lse, per_row, rtol=0, atol=1e-10)
+    if N // b != b:      # the transposed order must be told apart
+        m = N // b
+        assert not np.allclose(lse.reshape(m, b).T.reshape(-1), per_row, atol=1e-6)
+
+
+# ---------------------------------------------------------------- sequences of different lengths
+@pytest.mark.parametrize("N,b,n_valid", [(24, 4, 9), (24, 4, 12), (24, 6, 5), (20, 5, 11), (32, 4, 3)])
+@pytest.mark.parametrize("T", [1, 2, 3])
+def test_sequence_inside_a_longer_padding_equals_the_sequence_alone(N, b, n_valid, T):
+    """App. C.3 names batches padded to a maximum length.  Reading: blocks that lie wholly in the
+    padding are absent from the sequence's problem, so the valid rows must equal those of the same
+    sequence run alone at its own padded length ceil(n_valid/b)*b with the appendix's mask."""
+    rng = np.random.default_rng(N + 7 * n_valid + T)
+    Q, K, V = (rng.standard_normal((N, 4)) * 1.2 for _ in range(3))
+    own = -(-n_valid // b) * b
+    alone = mo.monarch_attention_head(Q[:own], K[:own], V[:own], b, T, scale=0.5,
+                                      n_valid=n_valid if n_valid < own else None)
+    padded, L, R = mo.monarch_attention_head(Q, K, V, b, T, scale=0.5, n_valid=n_valid,
+                                             return_factors=True)
+    assert np.allclose(padded[:n_valid], alone[:n_valid], rtol=0, atol=1e-13)
+    assert np.all(padded[own:] == 0.0)
+    # what is unique about M: no mass on padded keys, unit mass on valid keys for the sequence's rows
+    M = mo.dense_monarch(L, R)
+    assert np.all(M[:, n_valid:] == 0.0)
+    assert np.allclose(M[:own].sum(axis=1), 1.0, atol=1e-13)
+    # garbage (even non-finite values) in the rows past the sequence's own padded length is never read
+    Q2, K2, V2 = Q.copy(), K.copy(), V.copy()
+    K2[own:] = np.nan
+    V2[own:] = np.inf
+    Q2[own:] = -np.inf
+    again = mo.monarch_attention_head(Q2, K2, V2, b, T, scale=0.5, n_valid=n_valid)
+    assert np.array_equal(again[:own], padded[:own])
+
+
+def test_batched_lengths_one_per_batch_entry():
+    rng = np.random.default_rng(5)
+    Q, K, V = (rng.standard_normal((3, 2, 24, 4)) for _ in range(3))
+    lens = np.array([24, 10, 5])
+    O = mo.monarch_attention(Q, K, V, b=4, T=2, n_valid=lens)
+    for e in range(3):
+        for h in range(2):
+            ref = mo.monarch_attention_head(Q[e, h], K[e, h], V[e, h], 4, 2, n_valid=int(lens[e]))
+            assert np.array_equal(O[e, h], ref)
