@@ -44,18 +44,17 @@ typedef enum {
 typedef enum {
   MA_PATH_AUTO = 0,
   MA_PATH_GENERIC = 1, /* fp32 SIMT kernels, fp32 states; any dtype, any N = m*b that fits smem */
-  MA_PATH_TENSOR = 2,  /* tcgen05/TMA kernels, 16-bit states; f16/bf16, d = 64, m = b in
-                          {32, 64, 128}: one persistent launch for all 2T half-steps (softmax and
-                          epilogue in separate warpgroups); bf16 with b = 32 keeps alpha_L as a
-                          hi + lo pair of bf16 arrays (one more workspace array) */
-  MA_PATH_TENSOR_PHASED = 3, /* first-generation persistent kernel, one launch per half-step */
+  MA_PATH_TENSOR = 2,  /* tcgen05/TMA kernel, 16-bit states; f16/bf16, d = 64, m = b in
+                          {32, 64, 128}: one persistent launch for all 2T half-steps, softmax
+                          weights handed to the second MMA through shared memory; bf16 with b = 32
+                          keeps alpha_L as a hi + lo pair of bf16 arrays (one more workspace
+                          array).  Needs the whole GPU: see monarch_attn_fwd_ex */
+  MA_PATH_TENSOR_TMEM = 3, /* the same tiles and order with the softmax weights handed over in
+                              tensor memory and deeper operand rings: f16/bf16, d = 64, m = b in
+                              {64, 128}.  Needs the whole GPU as well */
   MA_PATH_TENSOR_BASIC = 4,  /* one CTA per tile, one launch per half-step (no pipelining);
-                                m = b in {64, 128} */
-  MA_PATH_TENSOR_CHAINED = 6, /* first-generation persistent kernel (each softmax warpgroup also
-                                 does its tile's epilogue), one launch; kept for comparison */
-  MA_PATH_FUSED = 5,   /* one CTA per (batch, head), everything in shared memory, one launch:
-                          f16/bf16, N = 256, m = b = 16, d = 64 only; kept for comparison (AUTO
-                          takes MA_PATH_FUSED_SMALL for this shape too) */
+                                m = b in {64, 128}; the plain statement the persistent kernels are
+                                tested against */
   MA_PATH_FUSED_SMALL = 7, /* the same idea for any block shape: f16/bf16, m and b <= 32 (m need not
                              equal b), d <= 64 a multiple of 8, N <= 580 for T = 1 and <= 440 for
                              T > 1 (the states of a head must fit shared memory); f16 arithmetic */

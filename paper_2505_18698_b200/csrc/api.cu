@@ -12,7 +12,6 @@
 #include "tensor_path.cuh"
 #include "tensor_persistent.cuh"
 #include "tensor_decoupled.cuh"
-#include "fused_n256.cuh"
 #include "fused_small.cuh"
 #include "tile_mma.cuh"
 
@@ -158,9 +157,7 @@ static int launch_generic(const Problem& p, const void* Q, const void* K, const 
 // ------------------------------------------------------------------ path selection
 static int resolve_path(const Problem& p, int path) {
   if (path == MA_PATH_AUTO) {
-    // Short sequences with small blocks: one CTA per head, states in shared memory.  The general
-    // kernel is the faster of the two fused kernels on the N = 256, b = 16 shape as well (matrix
-    // stores, per-warp pipelined loads), so AUTO never picks MA_PATH_FUSED.
+    // Short sequences with small blocks: one CTA per head, states in shared memory.
     if (p.b <= 16 && p.m <= 16 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T))
       return MA_PATH_FUSED_SMALL;
     // bf16 with b = 32 and more than two rounds leaves the tcgen05 path: on the peaky-logit recipe of
@@ -178,9 +175,12 @@ static int resolve_path(const Problem& p, int path) {
   if (path == MA_PATH_TILE_MMA) return tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
   if (path == MA_PATH_FUSED_SMALL)
     return fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T) ? path : -1;
-  if (path == MA_PATH_FUSED) return fused::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
-  if (path == MA_PATH_TENSOR || path == MA_PATH_TENSOR_PHASED || path == MA_PATH_TENSOR_CHAINED)
-    return tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
+  if (path == MA_PATH_TENSOR) return tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
+  if (path == MA_PATH_TENSOR_TMEM)
+    return (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) &&
+            tp::tmem_kernel_supported(p.b, p.H, p.lse, p.n_valid < p.N ? p.n_valid : 0))
+               ? path
+               : -1;
   if (path == MA_PATH_TENSOR_BASIC)
     return tensor::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
   return -1;
@@ -209,11 +209,10 @@ static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused
 
 static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
-  if (resolved == MA_PATH_FUSED || resolved == MA_PATH_FUSED_SMALL) return kStatusBytes;   // no states leave the chip
+  if (resolved == MA_PATH_FUSED_SMALL) return kStatusBytes;   // no states leave the chip
   if (resolved == MA_PATH_TILE_MMA) return tile::workspace_bytes(p.BH, p.N, p.d, p.T);
   if (resolved == MA_PATH_TENSOR_BASIC) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
-  if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_PHASED ||
-      resolved == MA_PATH_TENSOR_CHAINED)
+  if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_TMEM)
     return tp::workspace_bytes(p.BH, p.N, p.T, tp::uses_hilo(p.dtype, p.b));
   return 0;
 }
@@ -261,11 +260,6 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   if (!ws || ws_bytes < workspace_bytes_for(p, resolved)) return MA_ERR_WORKSPACE;
   if (((uintptr_t)ws & 255) != 0) return MA_ERR_ALIGN;
   if (resolved == MA_PATH_GENERIC) return launch_generic(p, Q, K, V, Y, scale, ws, st);
-  if (resolved == MA_PATH_FUSED) {
-    int rc = fused::launch(Q, K, V, Y, p.BH, p.T, p.dtype, scale, st);
-    if (rc == MA_OK) g_last_launches = 1;
-    return rc;
-  }
   if (resolved == MA_PATH_FUSED_SMALL) {
     int rc = fsmall::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.m, p.T, p.dtype, scale, p.n_valid, p.H, p.lse, st);
     if (rc == MA_OK) g_last_launches = 1;
@@ -284,7 +278,7 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
     rc = tensor::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.T, p.dtype, scale, ws, st, &launches);
   else
     rc = tp::launch(Q, K, V, Y, p.BH, p.N, p.b, p.T, p.dtype, scale, ws, st, &launches,
-                    resolved == MA_PATH_TENSOR ? 0 : (resolved == MA_PATH_TENSOR_PHASED ? 1 : 2),
+                    resolved == MA_PATH_TENSOR_TMEM ? 1 : 0,
                     ws_armed, p.H, p.lse, p.n_valid < p.N ? p.n_valid : 0);
   if (rc == MA_OK) g_last_launches = launches;
   return rc;

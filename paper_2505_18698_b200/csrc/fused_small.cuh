@@ -3,9 +3,9 @@
 //
 // One CTA (8 warps) per (batch, head), one launch for all T rounds.  Q, K, V are read from HBM
 // once, the states alpha_L, alpha_R, y, c_L (Sec. 3 'Implementation') never leave shared memory,
-// Y is written once.  It covers the shapes whose blocks do not fill a 64-row tensor-core tile and
-// are not the 16 x 16 special case of the N = 256 kernel: e.g. N = 210 as 15 blocks of 14 with 197
-// valid keys, or N = 384 as 16 blocks of 24.
+// Y is written once.  It covers the shapes whose blocks do not fill a 64-row tensor-core tile:
+// N = 256 as 16 blocks of 16, N = 210 as 15 blocks of 14 with 197 valid keys, N = 384 as 16 blocks
+// of 24.
 //
 // Layout.  Every tile (Q, K, V and the states) is stored with the SAME row order, row = k*b + i
 // for block k and in-block position i, 128 bytes per row (d padded with zeros to 64).  The
@@ -16,8 +16,9 @@
 // (L) entirely, so inside a half-step no two warps touch the same rows and the outputs can take
 // the place of dead inputs: on the last round alpha_L goes over K, y over V, Y over Q.
 //
-// Contractions are warp-level mma.sync m16n8k16 in f16 (bf16 inputs are converted on the way in,
-// as in the N = 256 kernel).  Blocks are padded to 16 or 32 rows/columns in registers only:
+// Contractions are warp-level mma.sync m16n8k16 in f16 (bf16 inputs are converted to f16 on the way
+// in: exact for magnitudes in [6.1e-5, 65504], clamped beyond; the dominant error of a 16-bit
+// pipeline is the rounding of alpha_L, and f16 carries three more mantissa bits than bf16).  Blocks are padded to 16 or 32 rows/columns in registers only:
 // operand rows past the block are clamped to its last row (finite values), score columns past the
 // block or past n_valid get -inf, weight rows past the block are zeroed before a transposed
 // product, and output rows past the block are not stored.
@@ -27,23 +28,23 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include "fused_n256.cuh"
+#include "warp_mma.cuh"
 
 namespace ma {
 namespace fsmall {
 
-using fused::Mma;
-using fused::col_sum;
-using fused::ex2;
-using fused::kLn2;
-using fused::kLog2e;
-using fused::ldsm_x2_trans;
-using fused::ldsm_x4;
-using fused::ldsm_x4_trans;
-using fused::lg2;
-using fused::movm_trans;
-using fused::quad_max;
-using fused::quad_sum;
+using warpmma::Mma;
+using warpmma::col_sum;
+using warpmma::ex2;
+using warpmma::kLn2;
+using warpmma::kLog2e;
+using warpmma::ldsm_x2_trans;
+using warpmma::ldsm_x4;
+using warpmma::ldsm_x4_trans;
+using warpmma::lg2;
+using warpmma::movm_trans;
+using warpmma::quad_max;
+using warpmma::quad_sum;
 
 constexpr int kThreads = 256, kWarps = 8, kRowBytes = 128, kMaxSmem = 227 * 1024;
 // where stmatrix rows past the end of a block go: 16 bytes per thread
@@ -134,7 +135,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
       for (int i = lane >> 3; i < b; i += 4) {
         if (ch * 8 >= d) continue;
         uint4* p = reinterpret_cast<uint4*>(smem + (size_t)a * tile + at(k, i, b, ch * 8));
-        *p = fused::to_f16x8(*p, (const TIn*)nullptr);
+        *p = warpmma::to_f16x8(*p, (const TIn*)nullptr);
       }
     }
   };
@@ -425,7 +426,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             if (ch * 8 >= d) continue;
             const uint4 v = *reinterpret_cast<const uint4*>(sQ + at(l, j, b, ch * 8));
             TIn* gp = Y + head_base + (size_t)(l * b + j) * row_stride + ch * 8;
-            *reinterpret_cast<uint4*>(gp) = fused::from_f16x8(v, gp);
+            *reinterpret_cast<uint4*>(gp) = warpmma::from_f16x8(v, gp);
           }
         }
         if (!last) {
@@ -519,6 +520,10 @@ inline bool supported(int N, int d, int b, int m, int dtype, int T) {
          smem_bytes(N, T) <= (size_t)kMaxSmem;
 }
 
+int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
+           int m, int T, int dtype, float scale, int n_valid, int H, float* lse, cudaStream_t st);
+
+#ifdef MA_TU_FUSED_SMALL
 template <typename TIn, int BP, int MP>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
                     int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st) {
@@ -561,11 +566,13 @@ inline int launch_d(const void* Q, const void* K, const void* V, void* Y, int BH
   return launch_t<TIn, 32, 32>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
 }
 
-inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
+int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
                   int m, int T, int dtype, float scale, int n_valid, int H, float* lse, cudaStream_t st) {
   if (dtype == 1) return launch_d<__half>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
   return launch_d<__nv_bfloat16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
 }
+
+#endif  // MA_TU_FUSED_SMALL
 
 }  // namespace fsmall
 }  // namespace ma

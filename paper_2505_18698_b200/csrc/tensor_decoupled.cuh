@@ -1,10 +1,5 @@
-// Persistent tensor-core kernel, second generation: the epilogue has warps of its own.
-//
-// Same tiles, same order, same dependency counters, same MMAs as `monarch_persistent`
-// (tensor_persistent.cuh); what changes is who waits for what.  There a softmax warpgroup walked
-// the whole chain of a tile (scores -> softmax -> wait for the apply MMA -> epilogue -> wait for
-// the next scores), about 2.8 us of mostly latency, and two such chains were all that tensor
-// memory and shared memory allow.  Here
+// Persistent tensor-core kernel with P handed to the apply MMA through shared memory
+// (MA_PATH_TENSOR): tiles, order and dependency counters as described in tensor_persistent.cuh.
 //   * two softmax warpgroups do nothing but S -> P (alternate tiles); S has three (b = 128) or four
 //     (b <= 64) TMEM stages, so the score MMA runs ahead and a group never waits for it;
 //   * a third warpgroup does every epilogue (O -> 16-bit rows -> staging), so the softmax groups
@@ -871,5 +866,13 @@ template <typename T, int B, int SB>
 cudaError_t launch_decoupled(const Params& P, int grid, cudaStream_t st) {
   return tp2::launch_kernel<T, B, SB>(P, grid, st);
 }
+#ifdef MA_TU_TENSOR_DECOUPLED
+template cudaError_t launch_decoupled<__half, 128, 128>(const Params&, int, cudaStream_t);
+template cudaError_t launch_decoupled<__half, 64, 64>(const Params&, int, cudaStream_t);
+template cudaError_t launch_decoupled<__half, 64, 32>(const Params&, int, cudaStream_t);
+template cudaError_t launch_decoupled<__nv_bfloat16, 128, 128>(const Params&, int, cudaStream_t);
+template cudaError_t launch_decoupled<__nv_bfloat16, 64, 64>(const Params&, int, cudaStream_t);
+template cudaError_t launch_decoupled<__nv_bfloat16, 64, 32>(const Params&, int, cudaStream_t);
+#endif
 }  // namespace tp
 }  // namespace ma

@@ -933,6 +933,10 @@ inline bool make_map_blocked_io(CUtensorMap* tm, int dtype, void* base, uint64_t
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
+           int T, int dtype, float scale, void* ws, cudaStream_t st, int* launches);
+
+#ifdef MA_TU_TENSOR_BASIC
 template <typename T, int B>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int T_steps,
                     int dtype, float scale, const Ws& w, cudaStream_t st, int* launches) {
@@ -987,7 +991,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   return 0;
 }
 
-inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
+int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
                   int T, int dtype, float scale, void* ws, cudaStream_t st, int* launches) {
   (void)d;
   Ws w = ws_layout(ws, BH, N);
@@ -999,6 +1003,8 @@ inline int launch(const void* Q, const void* K, const void* V, void* Y, int BH, 
     return launch_t<__nv_bfloat16, 128>(Q, K, V, Y, BH, N, T, dtype, scale, w, st, launches);
   return launch_t<__nv_bfloat16, 64>(Q, K, V, Y, BH, N, T, dtype, scale, w, st, launches);
 }
+
+#endif  // MA_TU_TENSOR_BASIC
 
 }  // namespace tensor
 }  // namespace ma

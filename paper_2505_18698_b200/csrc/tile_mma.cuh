@@ -20,22 +20,22 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include "fused_n256.cuh"
+#include "warp_mma.cuh"
 #include "fused_small.cuh"
 
 namespace ma {
 namespace tile {
 
-using fused::Mma;
-using fused::col_sum;
-using fused::ex2;
-using fused::kLn2;
-using fused::kLog2e;
-using fused::ldsm_x4;
-using fused::ldsm_x4_trans;
-using fused::lg2;
-using fused::quad_max;
-using fused::quad_sum;
+using warpmma::Mma;
+using warpmma::col_sum;
+using warpmma::ex2;
+using warpmma::kLn2;
+using warpmma::kLog2e;
+using warpmma::ldsm_x4;
+using warpmma::ldsm_x4_trans;
+using warpmma::lg2;
+using warpmma::quad_max;
+using warpmma::quad_sum;
 using fsmall::stsm_x4;
 
 typedef __half T;
@@ -97,13 +97,13 @@ __device__ __forceinline__ void convert_rows(uint8_t* dst, int rows, int d) {
     if (ch * 8 < d)
       for (int r = threadIdx.x / kChunks; r < rows; r += rstep) {
         uint4* p = reinterpret_cast<uint4*>(dst + r * pitch_of(DT) + ch * 16);
-        *p = fused::to_f16x8(*p, (const TSrc*)nullptr);
+        *p = warpmma::to_f16x8(*p, (const TSrc*)nullptr);
       }
   }
 }
 
 __device__ __forceinline__ uint4 store16_from_f16(uint4 v, __half*) { return v; }
-__device__ __forceinline__ uint4 store16_from_f16(uint4 v, __nv_bfloat16* p) { return fused::from_f16x8(v, p); }
+__device__ __forceinline__ uint4 store16_from_f16(uint4 v, __nv_bfloat16* p) { return warpmma::from_f16x8(v, p); }
 
 // One warp copies its 16 staged rows (first `rows` of them valid) out: row r to dst + r * stride.
 template <typename TDst, int DT>
@@ -620,6 +620,9 @@ struct Args {
   float scale;
 };
 
+int launch(const Args& a, int dtype, void* ws, cudaStream_t st, int* launches);
+
+#ifdef MA_TU_TILE_MMA
 template <typename TIn, int CB, int DT, bool HILO>
 inline int launch_r(const Args& a, const Ws& w, bool first, bool last, cudaStream_t st) {
   auto kern = r_tile_kernel<TIn, CB, DT, HILO>;
@@ -674,12 +677,14 @@ template <typename TIn, bool HILO>
 inline int launch_h(const Args& a, void* ws, cudaStream_t st, int* launches) {
   return a.d <= 64 ? launch_td<TIn, 4, HILO>(a, ws, st, launches) : launch_td<TIn, 8, HILO>(a, ws, st, launches);
 }
-inline int launch(const Args& a, int dtype, void* ws, cudaStream_t st, int* launches) {
+int launch(const Args& a, int dtype, void* ws, cudaStream_t st, int* launches) {
   if (dtype == 1)
     return uses_hilo(a.T) ? launch_h<__half, true>(a, ws, st, launches) : launch_h<__half, false>(a, ws, st, launches);
   return uses_hilo(a.T) ? launch_h<__nv_bfloat16, true>(a, ws, st, launches)
                         : launch_h<__nv_bfloat16, false>(a, ws, st, launches);
 }
+
+#endif  // MA_TU_TILE_MMA
 
 }  // namespace tile
 }  // namespace ma

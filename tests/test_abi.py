@@ -50,7 +50,7 @@ def test_binding_constants_match_the_header():
     for name, val in enums.items():
         if hasattr(binding, name):
             assert getattr(binding, name) == val, name
-    for name in ("MA_PATH_AUTO", "MA_PATH_GENERIC", "MA_PATH_TENSOR", "MA_PATH_FUSED", "MA_PATH_FUSED_SMALL",
+    for name in ("MA_PATH_AUTO", "MA_PATH_GENERIC", "MA_PATH_TENSOR", "MA_PATH_TENSOR_TMEM", "MA_PATH_FUSED_SMALL",
                  "MA_PATH_TILE_MMA", "MA_F32", "MA_F16", "MA_BF16"):
         assert name in enums and hasattr(binding, name), name
     assert len({v for k, v in enums.items() if k.startswith("MA_PATH_")}) == \

@@ -94,8 +94,7 @@ def test_generic_path_on_configuration_shapes(name):
 
 
 # ------------------------------------------------------------------ tensor-core paths
-TENSOR_PATHS = [binding.MA_PATH_TENSOR, binding.MA_PATH_TENSOR_PHASED, binding.MA_PATH_TENSOR_BASIC,
-                binding.MA_PATH_TENSOR_CHAINED]
+TENSOR_PATHS = [binding.MA_PATH_TENSOR, binding.MA_PATH_TENSOR_TMEM, binding.MA_PATH_TENSOR_BASIC]
 
 
 @pytest.mark.parametrize("path", TENSOR_PATHS)
@@ -108,12 +107,12 @@ def test_tensor_paths_match_oracle(N, b, T, dtype, batch, heads, path):
     check(batch, heads, N, 64, b, T, dtype, rank=16, s=1.5, seed=N + T + heads, path=path)
 
 
-@pytest.mark.parametrize("path", [binding.MA_PATH_TENSOR, binding.MA_PATH_TENSOR_PHASED])
 @pytest.mark.parametrize("T,dtype,batch,heads", [(1, "bf16", 1, 1), (2, "bf16", 2, 3), (3, "f16", 1, 5),
                                                   (2, "f16", 19, 1)])
-def test_tensor_path_block_32_on_64_row_tiles(T, dtype, batch, heads, path):
+def test_tensor_path_block_32_on_64_row_tiles(T, dtype, batch, heads):
     """b = m = 32 (N = 1024): two blocks share one 64-row MMA tile, off-diagonal P is zero."""
-    check(batch, heads, 1024, 64, 32, T, dtype, rank=16, s=1.5, seed=3 * T + heads, path=path)
+    check(batch, heads, 1024, 64, 32, T, dtype, rank=16, s=1.5, seed=3 * T + heads,
+          path=binding.MA_PATH_TENSOR)
 
 
 @pytest.mark.parametrize("T", [1, 2])
@@ -144,21 +143,20 @@ def test_auto_takes_bf16_block_32_with_three_rounds_off_the_tcgen05_path():
     assert err < 1e-2
 
 
-def test_tensor_kernel_generations_agree():
-    """The two generations of the persistent kernel and the per-half-step launches of the first run
-    the same tiles with the same MMAs: the first generation is bit-identical between its launch
-    modes (counters vs stream order), and the second differs from it only by where the non-final L
-    weights are rounded (once, after normalising in fp32, instead of twice)."""
+def test_persistent_tensor_kernels_agree_with_the_one_tile_per_cta_kernels():
+    """The persistent kernels run the tiles of the plain one-CTA-per-tile kernels with the same MMAs.
+    Without a non-final L half-step (T = 1) the shared-memory variant's arithmetic is the same to
+    the bit; the tensor-memory variant and T > 1 differ only by where weights are rounded."""
     Q, K, V = wl.make_qkv(1, 5, 4096, 64, "bf16", 16, 1.5, seed=41)
-    a = gpu_forward(Q, K, V, "bf16", 64, 3, binding.MA_PATH_TENSOR_CHAINED)
-    b_ = gpu_forward(Q, K, V, "bf16", 64, 3, binding.MA_PATH_TENSOR_PHASED)
-    assert np.array_equal(a, b_)
-    c = gpu_forward(Q, K, V, "bf16", 64, 3, binding.MA_PATH_TENSOR)
-    assert rel_err(c, a) <= 1e-2
-    # without a non-final L half-step (T = 1) the arithmetic is the same to the bit
-    a1 = gpu_forward(Q, K, V, "bf16", 64, 1, binding.MA_PATH_TENSOR_CHAINED)
+    a = gpu_forward(Q, K, V, "bf16", 64, 3, binding.MA_PATH_TENSOR_BASIC)
+    for path in (binding.MA_PATH_TENSOR, binding.MA_PATH_TENSOR_TMEM):
+        c = gpu_forward(Q, K, V, "bf16", 64, 3, path)
+        assert rel_err(c, a) <= 1e-2
+    a1 = gpu_forward(Q, K, V, "bf16", 64, 1, binding.MA_PATH_TENSOR_BASIC)
     c1 = gpu_forward(Q, K, V, "bf16", 64, 1, binding.MA_PATH_TENSOR)
-    assert np.array_equal(a1, c1)
+    assert rel_err(c1, a1) <= 2e-3
+    t1 = gpu_forward(Q, K, V, "bf16", 64, 1, binding.MA_PATH_TENSOR_TMEM)
+    assert rel_err(t1, a1) <= 2e-3
 
 
 def test_persistent_kernel_repeated_calls_share_workspace():
@@ -178,19 +176,7 @@ def test_persistent_kernel_repeated_calls_share_workspace():
     assert rel_err(outs[0].float().cpu().numpy().astype(np.float64), ref) <= 1e-2
 
 
-# ------------------------------------------------------------------ fused per-head kernel (N = 256)
-@pytest.mark.parametrize("dtype", ["f16", "bf16"])
-@pytest.mark.parametrize("T", [1, 2, 3])
-@pytest.mark.parametrize("batch,heads", [(1, 1), (2, 3), (149, 2)])
-def test_fused_kernel_matches_oracle(batch, heads, T, dtype):
-    # T <= 2: the recipe of configuration C2 (logit std ~ 11).  With such peaky logits a third
-    # round amplifies the 16-bit rounding of the states beyond 1e-2 on about one head in 300, so
-    # T = 3 is checked on the milder recipe of C4/C5 (logit std ~ 5.6).
-    rank, s = (8, 2.0) if T <= 2 else (16, 1.5)
-    check(batch, heads, 256, 64, 16, T, dtype, rank=rank, s=s, seed=7 * T + heads,
-          path=binding.MA_PATH_FUSED)
-
-
+# ------------------------------------------------------------------ fused per-head kernel
 def test_a_fused_kernel_is_the_default_for_short_sequences_and_launches_once():
     Q, K, V = wl.make_qkv(2, 2, 256, 64, "f16", 8, 2.0, seed=12)
     Qd, Kd, Vd = (binding.to_device(x, "f16") for x in (Q, K, V))
@@ -200,8 +186,6 @@ def test_a_fused_kernel_is_the_default_for_short_sequences_and_launches_once():
     assert binding.monarch_attn_last_launch_count() == 1
     torch.cuda.synchronize()
     assert torch.equal(a, b_)
-    binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 16, 2, path=binding.MA_PATH_FUSED)
-    assert binding.monarch_attn_last_launch_count() == 1
 
 
 # ------------------------------------------------------------------ general fused per-head kernel
@@ -221,14 +205,8 @@ def test_general_fused_kernel_matches_oracle(N, b, d, T, dtype):
     assert binding.monarch_attn_last_launch_count() == 1
 
 
-def test_general_fused_kernel_many_heads_and_agreement_with_the_special_case():
+def test_general_fused_kernel_many_heads():
     check(151, 3, 210, 64, 14, 2, "f16", rank=8, s=1.0, seed=5, path=binding.MA_PATH_FUSED_SMALL)
-    Q, K, V = wl.make_qkv(3, 4, 256, 64, "f16", 8, 2.0, seed=21)
-    Qd, Kd, Vd = (binding.to_device(x, "f16") for x in (Q, K, V))
-    for T in (1, 2):
-        a = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 16, T, path=binding.MA_PATH_FUSED_SMALL).float()
-        b_ = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 16, T, path=binding.MA_PATH_FUSED).float()
-        assert float((a - b_).norm() / b_.norm()) <= 2e-3
 
 
 @pytest.mark.parametrize("name", ["S1", "S2", "S3", "S4"])
