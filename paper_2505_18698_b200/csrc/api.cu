@@ -157,15 +157,15 @@ static int launch_generic(const Problem& p, const void* Q, const void* K, const 
 // ------------------------------------------------------------------ path selection
 static int resolve_path(const Problem& p, int path) {
   if (path == MA_PATH_AUTO) {
+    // From the third round on, plain 16-bit states are too coarse on peaky logits (they are fed
+    // back round after round: about one head in 300 of the N = 256 recipe exceeds 1e-2 at T = 3).
+    // The fused per-head kernel and the tcgen05 kernels keep such states; the tile kernels switch to
+    // hi + lo pairs from T = 3 on, so they take every 16-bit shape they support then.
+    if (p.T >= 3 && tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
     // Short sequences with small blocks: one CTA per head, states in shared memory.
     if (p.b <= 16 && p.m <= 16 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T))
       return MA_PATH_FUSED_SMALL;
-    // bf16 with b = 32 and more than two rounds leaves the tcgen05 path: on the peaky-logit recipe of
-    // that shape the 8-bit mantissa of alpha_R (used twice from T = 3 on) costs 4e-2 on the worst
-    // head; up to T = 2 the hi + lo alpha_L of that path keeps it under 1e-2.  The tile kernels keep
-    // both states as hi + lo pairs of f16 from T = 3 on (4e-3 on the same inputs).
-    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) && !(p.b == 32 && p.dtype == MA_BF16 && p.T > 2))
-      return MA_PATH_TENSOR;
+    if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TENSOR;
     if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
     if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
     if (generic_supported(p)) return MA_PATH_GENERIC;
@@ -190,20 +190,15 @@ static int resolve_path(const Problem& p, int path) {
 // kernel (`with_fused_small`), the warp-MMA tile kernels and the generic kernels serve:
 // AUTO, TENSOR, FUSED_SMALL, TILE_MMA or GENERIC; -1 if none applies.
 static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused_small = false) {
-  if (path == MA_PATH_AUTO || path == MA_PATH_TENSOR) {
-    const int r = resolve_path(p, path);
-    if (r == MA_PATH_TENSOR) return r;
-    if (path == MA_PATH_TENSOR) return -1;
-  }
-  if (with_fused_small && (path == MA_PATH_AUTO || path == MA_PATH_FUSED_SMALL)) {
-    if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
-    if (path == MA_PATH_FUSED_SMALL) return -1;
-  }
-  if (path == MA_PATH_AUTO || path == MA_PATH_TILE_MMA) {
+  if (path == MA_PATH_AUTO) {
+    const int r = resolve_path(p, MA_PATH_AUTO);
+    if (r != MA_PATH_FUSED_SMALL || with_fused_small) return r;
     if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
-    if (path == MA_PATH_TILE_MMA) return -1;
+    return generic_supported(p) ? MA_PATH_GENERIC : -1;
   }
-  if ((path == MA_PATH_AUTO || path == MA_PATH_GENERIC) && generic_supported(p)) return MA_PATH_GENERIC;
+  if (path == MA_PATH_TENSOR || path == MA_PATH_TILE_MMA || path == MA_PATH_GENERIC ||
+      (path == MA_PATH_FUSED_SMALL && with_fused_small))
+    return resolve_path(p, path);
   return -1;
 }
 

@@ -137,7 +137,7 @@ __device__ __forceinline__ void split_hilo(float x0, float x1, uint32_t& hi, uin
 inline size_t r_smem_bytes(int b, int dt, bool hilo) { return (size_t)(hilo ? 5 : 4) * round16(b) * pitch_of(dt); }
 inline size_t l_smem_bytes(int m, int cm, int dt, bool hilo) {
   const size_t tiles = (size_t)(hilo ? 4 : 3) * round16(m) * pitch_of(dt);  // Q(l,j), alpha_L(k,j) (+ lo), y(k,j)
-  const size_t p_tile = (size_t)round16(m) * (cm * 2 + 16);    // weights for the transposed product
+  const size_t p_tile = (size_t)(hilo ? 2 : 1) * round16(m) * (cm * 2 + 16);   // weights for the transposed product (+ lo)
   const size_t stats = (size_t)(2 * 8 * cm + cm) * 4;          // column max / sum per warp, c_L
   return tiles + p_tile + stats;
 }
@@ -262,13 +262,25 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
     // c_L = sum R log R (natural log): ln2 * (sum p z / sum - max - log2 sum)
     if (t == 0 && j < b) cL[(size_t)h * N + (size_t)k * b + j] = kLn2 * (sz * inv_s[hh] - mx - lg2(sum));
   }
-  uint32_t pa[CB / 16][4];
+  // Weights as A fragments.  With hi + lo states (HILO) the weights are a hi + lo pair as well:
+  // alpha_L feeds logits of size ~100, so the 2^-12 relative rounding of a dominant weight is a
+  // logit error of a few hundredths, and from the third round on that alone costs more than 1e-2
+  // on the worst head of a peaky recipe (measured 2.7e-2; 2e-4 with the pair).
+  uint32_t pa[CB / 16][4], pal[HILO ? CB / 16 : 1][4];
 #pragma unroll
   for (int kk = 0; kk < CB / 16; ++kk) {
     pa[kk][0] = Mma<T>::pack(s[2 * kk][0], s[2 * kk][1]);
     pa[kk][1] = Mma<T>::pack(s[2 * kk][2], s[2 * kk][3]);
     pa[kk][2] = Mma<T>::pack(s[2 * kk + 1][0], s[2 * kk + 1][1]);
     pa[kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+    if (HILO) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 hi = Mma<T>::unpack(pa[kk][q]);
+        const int nt = 2 * kk + (q >> 1), e0 = 2 * (q & 1);
+        pal[kk][q] = Mma<T>::pack(s[nt][e0] - hi.x, s[nt][e0 + 1] - hi.y);
+      }
+    }
   }
   // second products, two 8-column tiles of v at a time; results staged in this warp's own 16 rows
   // of the alpha_R tile (dead: only this warp read them) and of the y staging tile
@@ -292,6 +304,10 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
       ldsm_x4_trans(bf, sK_u + off);
       Mma<T>::run(o[0], pa[kk], bf);
       Mma<T>::run(o[1], pa[kk], bf + 2);
+      if (HILO) {
+        Mma<T>::run(o[0], pal[kk], bf);
+        Mma<T>::run(o[1], pal[kk], bf + 2);
+      }
       if (last) {
         ldsm_x4_trans(bf, sV_u + off);
         Mma<T>::run(yv[0], pa[kk], bf);
@@ -344,7 +360,8 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
   constexpr bool hilo = HILO;
   uint8_t* sLlo = sYt + (size_t)rm * kPitch;   // low halves of alpha_L in, of alpha_R out (hi + lo states)
   uint8_t* sP = sLlo + (hilo ? (size_t)rm * kPitch : 0);
-  float* sColMax = reinterpret_cast<float*>(sP + (size_t)rm * kPPitch);
+  uint8_t* sPlo = sP + (size_t)rm * kPPitch;   // low halves of the non-final weights (hi + lo states)
+  float* sColMax = reinterpret_cast<float*>(sPlo + (hilo ? (size_t)rm * kPPitch : 0));
   float* sColSum = sColMax + 8 * CM;
   float* sC = sColSum + 8 * CM;
   const HeadRows hr = head_rows(h, N, d, H);
@@ -490,7 +507,7 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
     const uint32_t st_u = sP_u + (l0 + st_row) * kPPitch + st_nt * 16;
 #pragma unroll
     for (int np = 0; np < CM / 16; ++np) {
-      uint32_t u[2][2];
+      uint32_t u[2][2], ul[2][2];
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
         const int nt = 2 * np + q;
@@ -501,9 +518,17 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
           for (int w = 0; w < row_warps; ++w) cm = fmaxf(cm, sColMax[w * CM + 8 * nt + 2 * t + e]);
           gk[e] = cm > 0.f ? __uint_as_float((253u << 23) - (__float_as_uint(cm) & 0x7f800000u)) : 0.f;
         }
-        u[q][0] = Mma<T>::pack(s[nt][0] * gk[0], s[nt][1] * gk[1]);
-        u[q][1] = Mma<T>::pack(s[nt][2] * gk[0], s[nt][3] * gk[1]);
-        const float2 f0 = Mma<T>::unpack(u[q][0]), f1 = Mma<T>::unpack(u[q][1]);
+        const float w00 = s[nt][0] * gk[0], w01 = s[nt][1] * gk[1];
+        const float w10 = s[nt][2] * gk[0], w11 = s[nt][3] * gk[1];
+        u[q][0] = Mma<T>::pack(w00, w01);
+        u[q][1] = Mma<T>::pack(w10, w11);
+        float2 f0 = Mma<T>::unpack(u[q][0]), f1 = Mma<T>::unpack(u[q][1]);
+        if (hilo) {      // weights as a hi + lo pair (see r_tile_kernel); c_R sums both halves
+          ul[q][0] = Mma<T>::pack(w00 - f0.x, w01 - f0.y);
+          ul[q][1] = Mma<T>::pack(w10 - f1.x, w11 - f1.y);
+          const float2 g0 = Mma<T>::unpack(ul[q][0]), g1 = Mma<T>::unpack(ul[q][1]);
+          f0.x += g0.x; f0.y += g0.y; f1.x += g1.x; f1.y += g1.y;
+        }
         const float c0 = col_sum(f0.x + f1.x), c1 = col_sum(f0.y + f1.y);
         if (g == 0) {
           sColSum[warp * CM + 8 * nt + 2 * t] = c0;
@@ -511,6 +536,9 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
         }
       }
       stsm_x4(st_u + np * 32, u[0][0], u[0][1], u[1][0], u[1][1]);
+      if (hilo)
+        stsm_x4(st_u - sP_u + (uint32_t)__cvta_generic_to_shared(sPlo) + np * 32, ul[0][0], ul[0][1], ul[1][0],
+                ul[1][1]);
     }
   }
   __syncthreads();
@@ -541,6 +569,11 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
       ldsm_x4_trans(bf, sQ_u + min(16 * ls + (lane & 15), m - 1) * kPitch + (lane >> 4) * 16 + np * 32);
       Mma<T>::run(o[0], a, bf);
       Mma<T>::run(o[1], a, bf + 2);
+      if (hilo) {
+        ldsm_x4_trans(a, pt_u - sP_u + (uint32_t)__cvta_generic_to_shared(sPlo) + 16 * ls * kPPitch);
+        Mma<T>::run(o[0], a, bf);
+        Mma<T>::run(o[1], a, bf + 2);
+      }
     }
     uint32_t hi[4], lo[4];
     split_hilo<HILO>(o[0][0] * ic[0], o[0][1] * ic[0], hi[0], lo[0]);
