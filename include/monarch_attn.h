@@ -149,6 +149,30 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
                             int heads, int N, int d, int b, int T, int dtype, float softmax_scale,
                             int n_valid, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Forward pass on a batch of sequences of different lengths padded to one length N (Appendix C.3
+ * names the case: "batched sequences of different lengths are padded to a maximum length").
+ *
+ * seq_len: DEVICE pointer to `batch` ints, 4-byte aligned; entry e is the number of real rows of
+ * every head of batch entry e (values outside [1, N] are clamped into it).  For each sequence:
+ *   - keys b k + i >= seq_len[e] get the mask of that appendix (minus infinity on Z_R, Eq. 7);
+ *   - a block lying wholly in the padding (k >= ceil(seq_len[e] / b)) has no admissible R row, and
+ *     the appendix gives no formula for it.  The library's reading: such a block is absent from
+ *     the sequence's problem -- no weight as a key block (Z_L = -inf in Eq. 8, so every row of the
+ *     Monarch matrix still sums to one over the valid keys), no term in the sums over l of Eq. 9
+ *     as a query block -- so that rows 0 .. seq_len[e]-1 of Y equal what the same sequence gives
+ *     when run alone at its own padded length ceil(seq_len[e] / b) * b;
+ *   - rows seq_len[e] .. ceil(seq_len[e] / b) * b - 1 of Y carry no meaning, later rows are zero;
+ *     rows of Q, K, V in absent blocks are never read.
+ * Q, K, V, Y: DEVICE pointers, [batch][heads][N][d], rules as monarch_attn_fwd_ex.  Runs on the
+ * general fused kernel (f16/bf16, m and b <= 32, d <= 64, short N: one launch) where that
+ * applies, else on the generic kernels (any dtype, any N = m b); workspace: the larger of
+ * monarch_attn_workspace_bytes() for MA_PATH_FUSED_SMALL and MA_PATH_GENERIC that is not 0.
+ * Asynchronous on `stream`. */
+int monarch_attn_fwd_varlen(const void* Q, const void* K, const void* V, void* Y, int batch,
+                            int heads, int N, int d, int b, int T, int dtype, float softmax_scale,
+                            const int* seq_len, void* workspace, size_t workspace_bytes,
+                            void* stream);
+
 /* The same forward pass for callers that must not allocate device memory.  (The paper has no
  * counterpart: this is a deployment variant of the library, not a step of the method.)
  *
@@ -185,24 +209,6 @@ int monarch_attn_device_status(const void* workspace, void* stream);
 
 /* Number of kernel launches the last successful call on this host thread enqueued. */
 int monarch_attn_last_launch_count(void);
-
-/* Profiling aid for the persistent tensor path.  With a DEVICE buffer of at least 4*64*8 int64
- * set, CTAs 0-3 of later MA_PATH_TENSOR / MA_PATH_TENSOR_PHASED launches write SM-clock stamps
- * [cta][tile][event] for their first 64 tiles; events: 0 operands requested, 1 score MMA issued,
- * 2 softmax group sees the scores, 3 P written, 4 apply MMA issued, 5 softmax group sees O,
- * 6 rows staged, 7 rows stored and signalled.  NULL switches it off (the default).  Process-wide;
- * the buffer stays owned by the caller. */
-int monarch_attn_set_trace_buffer(void* device_buffer, size_t bytes);
-
-/* Test and tuning knobs (process-wide; not for production use).  Knobs 1 and 2 belong to the
- * persistent tensor path:
- *   knob 1: bound, in SM clocks, of every device-side wait (value <= 0 restores the default 2e9);
- *   knob 2: non-zero leaves the first half-step out of later single-launch runs, so that the
- *           dependency waits of the second half-step can never be satisfied.  Together they let a
- *           test watch a wait run out: the kernel ends by itself, results are garbage, and
- *           monarch_attn_device_status reports MA_ERR_TIMEOUT.  Nothing faults or hangs.
- *   knob 3: number of chunks monarch_attn_fwd_host cuts a call into (1..8, default 4). */
-int monarch_attn_debug_knob(int knob, long long value);
 
 /* Static, NUL-terminated description of an ma_status code. */
 const char* monarch_attn_status_string(int status);

@@ -15,7 +15,8 @@ import torch
 
 _PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG_DIR, "libmonarch_attn.so")
-HEADER_PATH = os.path.join(os.path.dirname(_PKG_DIR), "include", "monarch_attn.h")
+INCLUDE_DIR = os.path.join(os.path.dirname(_PKG_DIR), "include")
+HEADER_PATH = os.path.join(INCLUDE_DIR, "monarch_attn.h")
 
 MA_F32, MA_F16, MA_BF16 = 0, 1, 2
 MA_PATH_AUTO, MA_PATH_GENERIC, MA_PATH_TENSOR, MA_PATH_TENSOR_TMEM, MA_PATH_TENSOR_BASIC = 0, 1, 2, 3, 4
@@ -35,11 +36,15 @@ class MonarchAttnError(RuntimeError):
         self.code = code
 
 
-def declared_symbols(header_path: str = HEADER_PATH):
-    """Names of the functions the public header declares."""
-    text = open(header_path).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(monarch_attn_\w+)\s*\(", text)))
+def declared_symbols(header_path: str | None = None):
+    """Names of the functions the headers under include/ declare (or one header's)."""
+    paths = [header_path] if header_path else sorted(
+        os.path.join(INCLUDE_DIR, f) for f in os.listdir(INCLUDE_DIR) if f.endswith(".h"))
+    names = set()
+    for p in paths:
+        text = re.sub(r"/\*.*?\*/", "", open(p).read(), flags=re.S)
+        names.update(re.findall(r"\b(monarch_attn_\w+)\s*\(", text))
+    return sorted(names)
 
 
 def load_library(path: str = LIB_PATH):
@@ -62,6 +67,8 @@ def load_library(path: str = LIB_PATH):
     lib.monarch_attn_fwd_bshd.restype = i
     lib.monarch_attn_fwd_padded.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp, sz, vp]
     lib.monarch_attn_fwd_padded.restype = i
+    lib.monarch_attn_fwd_varlen.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp, vp, sz, vp]
+    lib.monarch_attn_fwd_varlen.restype = i
     lib.monarch_attn_fwd_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
     lib.monarch_attn_fwd_host.restype = i
     lib.monarch_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
@@ -107,6 +114,33 @@ def _shape_of(Q, K, V):
     return tuple(int(x) for x in Q.shape)
 
 
+def _out_like(Y, Q, what="Y"):
+    """A caller-supplied output must match the input exactly: the kernels write Q.numel() elements
+    of Q's dtype through its pointer, on Q's device."""
+    if Y is None:
+        return torch.empty_like(Q)
+    if not isinstance(Y, torch.Tensor) or Y.shape != Q.shape or Y.dtype != Q.dtype:
+        raise ValueError(f"{what} must have the shape and dtype of Q")
+    if not Y.is_contiguous():
+        raise ValueError(f"{what} must be contiguous")
+    if Y.device != Q.device:
+        raise ValueError(f"{what} must be on the same device as Q")
+    return Y
+
+
+def _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code, paths):
+    """A caller-supplied workspace is checked; otherwise the largest any of `paths` needs."""
+    if workspace is not None:
+        if workspace.device != Q.device or workspace.dtype != torch.uint8 or not workspace.is_contiguous():
+            raise ValueError("workspace must be a contiguous uint8 tensor on Q's device")
+        return workspace
+    need = max(int(lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, p)) for p in paths)
+    return torch.zeros(max(need, 256), dtype=torch.uint8, device=Q.device)
+
+
+_ANY_PATH = (MA_PATH_TENSOR, MA_PATH_GENERIC, MA_PATH_TILE_MMA, MA_PATH_FUSED_SMALL)
+
+
 def monarch_attn_workspace_bytes(batch, heads, N, d, b, T, dtype, path=MA_PATH_AUTO) -> int:
     code = _TORCH_TO_CODE[dtype] if isinstance(dtype, torch.dtype) else int(dtype)
     return int(load_library().monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, path))
@@ -119,11 +153,11 @@ def monarch_attn_fwd(Q, K, V, b, T, Y=None, stream=None):
     if not Q.is_cuda:
         raise MonarchAttnError(-2, "monarch_attn_fwd needs CUDA tensors; there is no CPU path")
     batch, heads, N, d = _shape_of(Q, K, V)
-    if Y is None:
-        Y = torch.empty_like(Q)
-    _check(lib.monarch_attn_fwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
-                                batch, heads, N, d, b, T, _TORCH_TO_CODE[Q.dtype],
-                                _stream_ptr(stream)))
+    Y = _out_like(Y, Q)
+    with torch.cuda.device(Q.device):
+        _check(lib.monarch_attn_fwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                    batch, heads, N, d, b, T, _TORCH_TO_CODE[Q.dtype],
+                                    _stream_ptr(stream)))
     return Y
 
 
@@ -138,14 +172,12 @@ def monarch_attn_fwd_ex(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, wo
     code = _TORCH_TO_CODE[Q.dtype]
     if softmax_scale is None:
         softmax_scale = 1.0 / math.sqrt(d)
-    if Y is None:
-        Y = torch.empty_like(Q)
-    if workspace is None:
-        need = lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, path)
-        workspace = torch.empty(max(int(need), 256), dtype=torch.uint8, device=Q.device)
-    _check(lib.monarch_attn_fwd_ex(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
-                                   batch, heads, N, d, b, T, code, float(softmax_scale), int(path),
-                                   workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
+    Y = _out_like(Y, Q)
+    workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code, (path,))
+    with torch.cuda.device(Q.device):
+        _check(lib.monarch_attn_fwd_ex(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                       batch, heads, N, d, b, T, code, float(softmax_scale), int(path),
+                                       workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
     return Y
 
 
@@ -160,17 +192,14 @@ def monarch_attn_fwd_objective(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_A
     code = _TORCH_TO_CODE[Q.dtype]
     if softmax_scale is None:
         softmax_scale = 1.0 / math.sqrt(d)
-    if Y is None:
-        Y = torch.empty_like(Q)
+    Y = _out_like(Y, Q)
     lse = torch.empty((batch, heads, N), dtype=torch.float32, device=Q.device)
-    if workspace is None:
-        need = max(lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_TENSOR),
-                   lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_GENERIC))
-        workspace = torch.zeros(max(int(need), 256), dtype=torch.uint8, device=Q.device)
-    _check(lib.monarch_attn_fwd_objective(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
-                                          batch, heads, N, d, b, T, code, float(softmax_scale),
-                                          int(path), lse.data_ptr(), workspace.data_ptr(),
-                                          workspace.numel(), _stream_ptr(stream)))
+    workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code, _ANY_PATH)
+    with torch.cuda.device(Q.device):
+        _check(lib.monarch_attn_fwd_objective(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                              batch, heads, N, d, b, T, code, float(softmax_scale),
+                                              int(path), lse.data_ptr(), workspace.data_ptr(),
+                                              workspace.numel(), _stream_ptr(stream)))
     return Y, lse
 
 
@@ -189,15 +218,12 @@ def monarch_attn_fwd_bshd(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, 
     code = _TORCH_TO_CODE[Q.dtype]
     if softmax_scale is None:
         softmax_scale = 1.0 / math.sqrt(d)
-    if Y is None:
-        Y = torch.empty_like(Q)
-    if workspace is None:
-        need = max(lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_TENSOR),
-                   lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_GENERIC))
-        workspace = torch.zeros(max(int(need), 256), dtype=torch.uint8, device=Q.device)
-    _check(lib.monarch_attn_fwd_bshd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
-                                     batch, N, heads, d, b, T, code, float(softmax_scale), int(path),
-                                     workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
+    Y = _out_like(Y, Q)
+    workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code, _ANY_PATH)
+    with torch.cuda.device(Q.device):
+        _check(lib.monarch_attn_fwd_bshd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                         batch, N, heads, d, b, T, code, float(softmax_scale), int(path),
+                                         workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
     return Y
 
 
@@ -213,16 +239,39 @@ def monarch_attn_fwd_padded(Q, K, V, b, T, n_valid, softmax_scale=None, workspac
     code = _TORCH_TO_CODE[Q.dtype]
     if softmax_scale is None:
         softmax_scale = 1.0 / math.sqrt(d)
-    if Y is None:
-        Y = torch.empty_like(Q)
-    if workspace is None:
-        need = max(lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_TENSOR),
-                   lib.monarch_attn_workspace_bytes(batch, heads, N, d, b, T, code, MA_PATH_GENERIC))
-        workspace = torch.empty(max(int(need), 256), dtype=torch.uint8, device=Q.device)
-    _check(lib.monarch_attn_fwd_padded(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
-                                       batch, heads, N, d, b, T, code, float(softmax_scale),
-                                       int(n_valid), workspace.data_ptr(), workspace.numel(),
-                                       _stream_ptr(stream)))
+    Y = _out_like(Y, Q)
+    workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code, _ANY_PATH)
+    with torch.cuda.device(Q.device):
+        _check(lib.monarch_attn_fwd_padded(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                           batch, heads, N, d, b, T, code, float(softmax_scale),
+                                           int(n_valid), workspace.data_ptr(), workspace.numel(),
+                                           _stream_ptr(stream)))
+    return Y
+
+
+def monarch_attn_fwd_varlen(Q, K, V, b, T, seq_len, softmax_scale=None, workspace=None, Y=None,
+                            stream=None):
+    """Forward pass on a batch of sequences of different lengths padded to N rows (App. C.3).
+    seq_len: int32 CUDA tensor [batch] with the number of real rows of each batch entry.  Rows
+    below seq_len[e] of Y are the result; rows from ceil(seq_len[e] / b) * b on are zero."""
+    lib = load_library()
+    if not Q.is_cuda:
+        raise MonarchAttnError(-2, "monarch_attn_fwd_varlen needs CUDA tensors; there is no CPU path")
+    batch, heads, N, d = _shape_of(Q, K, V)
+    if not (isinstance(seq_len, torch.Tensor) and seq_len.dtype == torch.int32 and seq_len.is_contiguous()
+            and seq_len.device == Q.device and tuple(seq_len.shape) == (batch,)):
+        raise ValueError("seq_len must be a contiguous int32 tensor of shape [batch] on Q's device")
+    code = _TORCH_TO_CODE[Q.dtype]
+    if softmax_scale is None:
+        softmax_scale = 1.0 / math.sqrt(d)
+    Y = _out_like(Y, Q)
+    workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code,
+                               (MA_PATH_GENERIC, MA_PATH_FUSED_SMALL))
+    with torch.cuda.device(Q.device):
+        _check(lib.monarch_attn_fwd_varlen(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                           batch, heads, N, d, b, T, code, float(softmax_scale),
+                                           seq_len.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                           _stream_ptr(stream)))
     return Y
 
 
@@ -231,8 +280,9 @@ def monarch_attn_fwd_host(Qh, Kh, Vh, Yh, b, T, stream=None):
     `stream`; returns Yh without synchronising."""
     lib = load_library()
     batch, heads, N, d = _shape_of(Qh, Kh, Vh)
-    if Qh.is_cuda or Yh.is_cuda:
+    if Qh.is_cuda or Kh.is_cuda or Vh.is_cuda or Yh.is_cuda:
         raise ValueError("monarch_attn_fwd_host takes host tensors")
+    _out_like(Yh, Qh, "Yh")
     _check(lib.monarch_attn_fwd_host(Qh.data_ptr(), Kh.data_ptr(), Vh.data_ptr(), Yh.data_ptr(),
                                      batch, heads, N, d, b, T, _TORCH_TO_CODE[Qh.dtype],
                                      _stream_ptr(stream)))
@@ -248,12 +298,16 @@ def monarch_attn_fwd_noalloc(Q, K, V, b, T, Y, stream=None):
     wrapper allocates nothing either).  Small problems only (see the header for the limit);
     calls that overlap on the GPU race on the shared scratch."""
     lib = load_library()
-    if not (Q.is_cuda and Y.is_cuda):
+    if not (Q.is_cuda and Y is not None and Y.is_cuda):
         raise MonarchAttnError(-2, "monarch_attn_fwd_noalloc needs CUDA tensors; there is no CPU path")
     batch, heads, N, d = _shape_of(Q, K, V)
-    _check(lib.monarch_attn_fwd_noalloc(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
-                                        batch, heads, N, d, b, T, _TORCH_TO_CODE[Q.dtype],
-                                        _stream_ptr(stream)))
+    if Y is None:
+        raise ValueError("monarch_attn_fwd_noalloc allocates nothing: pass the output tensor Y")
+    _out_like(Y, Q)
+    with torch.cuda.device(Q.device):
+        _check(lib.monarch_attn_fwd_noalloc(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
+                                            batch, heads, N, d, b, T, _TORCH_TO_CODE[Q.dtype],
+                                            _stream_ptr(stream)))
     return Y
 
 

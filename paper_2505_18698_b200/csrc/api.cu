@@ -1,6 +1,7 @@
 // C-ABI boundary of libmonarch_attn: argument validation, workspace layout, path selection and
 // kernel launches.  No torch types; plain device/host pointers and sizes only.
 #include "../../include/monarch_attn.h"
+#include "../../include/monarch_attn_test.h"
 
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -27,6 +28,7 @@ struct Problem {
   int n_valid;   // keys b k + i >= n_valid are masked out (App. C.3); N when there is no padding
   int H;         // 0: [batch][heads][N][d]; heads: [batch][N][heads][d]
   float* lse;    // optional output [batch*heads][N]: row log-sum-exp of the final L half-step
+  const int* seq_len;   // optional DEVICE array [batch]: valid length of every sequence (App. C.3)
 };
 
 static int validate_shape(int batch, int heads, int N, int d, int b, int T, int dtype, Problem* p) {
@@ -34,7 +36,7 @@ static int validate_shape(int batch, int heads, int N, int d, int b, int T, int 
   if (batch <= 0 || heads <= 0 || N <= 0 || d <= 0 || b <= 0 || T < 1) return MA_ERR_SHAPE;
   if (N % b != 0) return MA_ERR_SHAPE;
   if ((long long)batch * heads > 0x7fffffffLL / 2) return MA_ERR_SHAPE;
-  *p = Problem{batch, heads, N, d, b, T, dtype, N / b, batch * heads, N, 0, nullptr};
+  *p = Problem{batch, heads, N, d, b, T, dtype, N / b, batch * heads, N, 0, nullptr, nullptr};
   return MA_OK;
 }
 
@@ -109,7 +111,7 @@ static int launch_generic_t(const Problem& p, const TIn* Q, const TIn* K, const 
       return MA_ERR_CUDA;                                                                      \
     if (launch_serialised(r_step_kernel<TIn, FIRST, WITHV>, gr, kThreads, rs, st, Q, K, V, w.aR, \
                           w.cR, w.aL, w.cL, w.y, p.N, p.d, p.b, p.m, scale, p.n_valid,          \
-                          p.H) != cudaSuccess)                                                  \
+                          p.H, p.seq_len, p.heads) != cudaSuccess)                              \
       return MA_ERR_CUDA;                                                                       \
   } while (0)
     if (first && last) MA_LAUNCH_R(true, true);
@@ -122,12 +124,12 @@ static int launch_generic_t(const Problem& p, const TIn* Q, const TIn* K, const 
     if (last) {
       if (set_smem((const void*)l_step_kernel<TIn, true>, ls) != cudaSuccess) return MA_ERR_CUDA;
       if (launch_serialised(l_step_kernel<TIn, true>, gl, kThreads, ls, st, Q, w.aL, w.cL, w.y, w.aR, w.cR, Y,
-                            p.N, p.d, p.b, p.m, scale, p.H, p.lse) != cudaSuccess)
+                            p.N, p.d, p.b, p.m, scale, p.H, p.lse, p.seq_len, p.heads) != cudaSuccess)
         return MA_ERR_CUDA;
     } else {
       if (set_smem((const void*)l_step_kernel<TIn, false>, ls) != cudaSuccess) return MA_ERR_CUDA;
       if (launch_serialised(l_step_kernel<TIn, false>, gl, kThreads, ls, st, Q, w.aL, w.cL, w.y, w.aR, w.cR, Y,
-                            p.N, p.d, p.b, p.m, scale, p.H, (float*)nullptr) != cudaSuccess)
+                            p.N, p.d, p.b, p.m, scale, p.H, (float*)nullptr, p.seq_len, p.heads) != cudaSuccess)
         return MA_ERR_CUDA;
     }
     ++launches;
@@ -256,7 +258,8 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   if (((uintptr_t)ws & 255) != 0) return MA_ERR_ALIGN;
   if (resolved == MA_PATH_GENERIC) return launch_generic(p, Q, K, V, Y, scale, ws, st);
   if (resolved == MA_PATH_FUSED_SMALL) {
-    int rc = fsmall::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.m, p.T, p.dtype, scale, p.n_valid, p.H, p.lse, st);
+    int rc = fsmall::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.m, p.T, p.dtype, scale, p.n_valid, p.H, p.lse, st,
+                            p.seq_len, p.heads);
     if (rc == MA_OK) g_last_launches = 1;
     return rc;
   }
@@ -335,12 +338,34 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
   // fused kernel for short sequences; the second-generation tensor kernel where a tile row owns a
   // whole key block (b = 64, 128: the mask touches the last block's tiles only); else generic
   int r = -1;
-  if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) r = MA_PATH_FUSED_SMALL;
+  if (p.T <= 2 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) r = MA_PATH_FUSED_SMALL;
   else if (resolve_path(p, MA_PATH_AUTO) == MA_PATH_TENSOR && p.b != 32) r = MA_PATH_TENSOR;
   else if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) r = MA_PATH_TILE_MMA;
   else if (generic_supported(p)) r = MA_PATH_GENERIC;
   if (r < 0) return MA_ERR_UNSUPPORTED;
   p.n_valid = n_valid;
+  return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+int monarch_attn_fwd_varlen(const void* Q, const void* K, const void* V, void* Y, int batch,
+                            int heads, int N, int d, int b, int T, int dtype, float softmax_scale,
+                            const int* seq_len, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+  Problem p;
+  int rc = validate_shape(batch, heads, N, d, b, T, dtype, &p);
+  if (rc != MA_OK) return rc;
+  rc = check_ptrs(Q, K, V, Y, p);
+  if (rc != MA_OK) return rc;
+  if (!seq_len) return MA_ERR_NULL;
+  if (((uintptr_t)seq_len & 3) != 0) return MA_ERR_ALIGN;
+  if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
+  // short 16-bit sequences with up to two rounds: the fused per-head kernel (one launch); else the
+  // generic kernels (fp32 states: also what three or more rounds on peaky logits need)
+  int r = -1;
+  if (p.T <= 2 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) r = MA_PATH_FUSED_SMALL;
+  else if (generic_supported(p)) r = MA_PATH_GENERIC;
+  if (r < 0) return MA_ERR_UNSUPPORTED;
+  p.seq_len = seq_len;
   return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 

@@ -80,11 +80,22 @@ template <typename TIn, int BP, int MP>
 __global__ void __launch_bounds__((BP == 16 || MP == 16) ? 2 * kThreads : kThreads, 1)
 monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
                     TIn* __restrict__ Y, int N, int d, int b, int m, int T_steps, float scale,
-                    int n_valid, int H, float* __restrict__ lse) {
+                    int n_valid, int H, float* __restrict__ lse, const int* __restrict__ seq_len,
+                    int heads) {
   typedef __half T;
   extern __shared__ uint8_t smem_raw[];
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Batched sequences of different lengths (App. C.3): blocks that lie wholly in a sequence's
+  // padding are absent from its problem, which is then exactly the problem with
+  // m = ceil(length / b) blocks and the appendix's mask in the last of them.  Rows are addressed
+  // by (block, position) with the block size b only, so running the smaller problem is a matter
+  // of the block count; the rows of Y past it are zeroed, the rows of Q, K, V past it never read.
+  const int m_alloc = m;
+  if (seq_len != nullptr) {
+    n_valid = min(max(seq_len[blockIdx.x / heads], 1), N);
+    m = (n_valid + b - 1) / b;
+  }
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int tile = N * kRowBytes;
   uint8_t* sQ = smem;
@@ -421,10 +432,12 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
         }
         if (last) {
           // the m rows (l, j) of Y are complete: this warp copies them out, 16 bytes per lane
+          // (rows of blocks that are absent from a shorter sequence's problem: zeros)
           const int ch = lane & 7;
-          for (int l = lane >> 3; l < m; l += 4) {
+          for (int l = lane >> 3; l < m_alloc; l += 4) {
             if (ch * 8 >= d) continue;
-            const uint4 v = *reinterpret_cast<const uint4*>(sQ + at(l, j, b, ch * 8));
+            const uint4 v = l < m ? *reinterpret_cast<const uint4*>(sQ + at(l, j, b, ch * 8))
+                                  : make_uint4(0u, 0u, 0u, 0u);
             TIn* gp = Y + head_base + (size_t)(l * b + j) * row_stride + ch * 8;
             *reinterpret_cast<uint4*>(gp) = warpmma::from_f16x8(v, gp);
           }
@@ -521,12 +534,14 @@ inline bool supported(int N, int d, int b, int m, int dtype, int T) {
 }
 
 int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
-           int m, int T, int dtype, float scale, int n_valid, int H, float* lse, cudaStream_t st);
+           int m, int T, int dtype, float scale, int n_valid, int H, float* lse, cudaStream_t st,
+           const int* seq_len = nullptr, int heads = 1);
 
 #ifdef MA_TU_FUSED_SMALL
 template <typename TIn, int BP, int MP>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
-                    int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st) {
+                    int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st,
+                    const int* seq_len, int heads) {
   auto kern = monarch_fused_small<TIn, BP, MP>;
   // The 16 x 16 kernel is compiled for 128 registers: two CTAs of 8 warps per SM where shared memory
   // lets two fit, else one CTA of 16 warps (each warp then owns at most one tile per half-step).
@@ -552,24 +567,29 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kern, (const TIn*)Q, (const TIn*)K, (const TIn*)V, (TIn*)Y, N, d, b, m, T, scale,
-                            n_valid, H, lse) == cudaSuccess
+                            n_valid, H, lse, seq_len, heads) == cudaSuccess
              ? 0
              : 7;
 }
 
 template <typename TIn>
 inline int launch_d(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
-                    int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st) {
-  if (b <= 16 && m <= 16) return launch_t<TIn, 16, 16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
-  if (b <= 16) return launch_t<TIn, 16, 32>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
-  if (m <= 16) return launch_t<TIn, 32, 16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
-  return launch_t<TIn, 32, 32>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
+                    int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st,
+                    const int* seq_len, int heads) {
+#define MA_FS_ARGS Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st, seq_len, heads
+  if (b <= 16 && m <= 16) return launch_t<TIn, 16, 16>(MA_FS_ARGS);
+  if (b <= 16) return launch_t<TIn, 16, 32>(MA_FS_ARGS);
+  if (m <= 16) return launch_t<TIn, 32, 16>(MA_FS_ARGS);
+  return launch_t<TIn, 32, 32>(MA_FS_ARGS);
+#undef MA_FS_ARGS
 }
 
 int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
-                  int m, int T, int dtype, float scale, int n_valid, int H, float* lse, cudaStream_t st) {
-  if (dtype == 1) return launch_d<__half>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
-  return launch_d<__nv_bfloat16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st);
+           int m, int T, int dtype, float scale, int n_valid, int H, float* lse, cudaStream_t st,
+           const int* seq_len, int heads) {
+  if (dtype == 1)
+    return launch_d<__half>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st, seq_len, heads);
+  return launch_d<__nv_bfloat16>(Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st, seq_len, heads);
 }
 
 #endif  // MA_TU_FUSED_SMALL

@@ -67,11 +67,29 @@ __global__ void __launch_bounds__(kThreads)
 r_step_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
               const float* __restrict__ aR, const float* __restrict__ cR,
               float* __restrict__ aL, float* __restrict__ cL, float* __restrict__ y,
-              int N, int d, int b, int m, float scale, int n_valid, int H) {
+              int N, int d, int b, int m, float scale, int n_valid, int H,
+              const int* __restrict__ seq_len, int heads) {
   extern __shared__ float smem[];
   grid_dependency_sync();
   const int k = blockIdx.x, h = blockIdx.y;
   const int dp = d + 1;
+  // Batched sequences of different lengths (App. C.3): n_valid is per batch entry.  A key block that
+  // lies wholly in the padding is absent from its sequence's problem: alpha_L = y = 0 and
+  // c_L = +inf, so that Z_L = -inf and the block gets no weight in the L half-step.
+  if (seq_len != nullptr) {
+    n_valid = min(max(seq_len[h / heads], 1), N);
+    if (k * b >= n_valid) {
+      const size_t head_off0 = (size_t)h * N * d;
+      for (int e = threadIdx.x; e < b * d; e += kThreads) {
+        const int j = e / d, v = e - j * d;
+        const size_t row = head_off0 + ((size_t)j * m + k) * d;
+        aL[row + v] = 0.f;
+        if (WITH_V) y[row + v] = 0.f;
+      }
+      for (int j = threadIdx.x; j < b; j += kThreads) cL[(size_t)h * N + (size_t)j * m + k] = INFINITY;
+      return;
+    }
+  }
   float* Ks = smem;                                  // [b][d+1]
   float* Vs = Ks + (size_t)b * dp;                   // [b][d+1] if WITH_V
   float* wbuf = Vs + (WITH_V ? (size_t)b * dp : 0);  // per warp: z[b], a[d]
@@ -150,10 +168,14 @@ __global__ void __launch_bounds__(kThreads)
 l_step_kernel(const TIn* __restrict__ Q, const float* __restrict__ aL, const float* __restrict__ cL,
               const float* __restrict__ y, float* __restrict__ aR, float* __restrict__ cR,
               TIn* __restrict__ Y, int N, int d, int b, int m, float scale, int H,
-              float* __restrict__ row_lse) {
+              float* __restrict__ row_lse, const int* __restrict__ seq_len, int heads) {
   extern __shared__ float smem[];
   grid_dependency_sync();
   const int j = blockIdx.x, h = blockIdx.y;
+  // blocks from m_live on lie wholly in the padding of this sequence (App. C.3, batched lengths):
+  // as key blocks they carry c_L = +inf (no weight), as query blocks they are left out of the sums
+  // over l of Eq. 9 and their rows of Y are zero; their rows of Q are never read
+  const int m_live = seq_len != nullptr ? (min(max(seq_len[h / heads], 1), N) + b - 1) / b : m;
   const int dp = d + 1, mp = m + 1;
   float* As = smem;                                  // aL[j]: [m][d+1]
   float* Qs = As + (size_t)m * dp;                   // Qb[j]: [m][d+1]
@@ -169,13 +191,23 @@ l_step_kernel(const TIn* __restrict__ Q, const float* __restrict__ aL, const flo
   for (int e = threadIdx.x; e < m * d; e += kThreads) {
     int r = e / d, v = e - r * d;
     As[r * dp + v] = aLj[e];
-    Qs[r * dp + v] = ld_as_float(Q + io_off(h, r * b + j, N, d, H) + v);
+    Qs[r * dp + v] = r < m_live ? ld_as_float(Q + io_off(h, r * b + j, N, d, H) + v) : 0.f;
     if (FINAL) Xs[r * dp + v] = yj[e];
   }
   for (int k = threadIdx.x; k < m; k += kThreads) cs[k] = cL[(size_t)h * N + (size_t)j * m + k];
   __syncthreads();
 
   for (int l = warp; l < m; l += kWarps) {
+    if (l >= m_live) {                            // absent query block
+      if (FINAL) {
+        TIn* out = Y + io_off(h, l * b + j, N, d, H);
+        for (int v = lane; v < d; v += 32) st_from_float(out + v, 0.f);
+        if (row_lse != nullptr && lane == 0) row_lse[(size_t)h * N + (size_t)l * b + j] = 0.f;
+      } else {
+        for (int k = lane; k < m; k += 32) Xs[l * mp + k] = 0.f;
+      }
+      continue;
+    }
     const float* q = Qs + l * dp;
     float zmax = -INFINITY;
     for (int k = lane; k < m; k += 32) {

@@ -535,8 +535,8 @@ def test_padded_sequences_match_masked_oracle(n_valid, b, d, T, dtype):
     V[:, :, n_valid:] = wl.round_to_dtype(np.float32(-50.0), dtype)
     Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))
     Y = binding.monarch_attn_fwd_padded(Qd, Kd, Vd, b, T, n_valid).float().cpu().numpy().astype(np.float64)
-    if b >= 64 and dtype != "f32":      # one persistent launch on the tensor kernel
-        assert binding.monarch_attn_last_launch_count() == 1
+    if b >= 64 and dtype != "f32":      # one persistent launch on the tensor kernel up to two rounds
+        assert binding.monarch_attn_last_launch_count() == (1 if T <= 2 else 2 * T)
     ref = mo.monarch_attention(Q, K, V, b, T, n_valid=n_valid)
     assert np.isfinite(Y[:, :, :n_valid]).all()
     err = rel_err(Y[:, :, :n_valid], ref[:, :, :n_valid])
@@ -672,3 +672,65 @@ def test_results_are_bit_identical_from_call_to_call(name):
         binding.monarch_attn_fwd(Qd, Kd, Vd, w.b, w.T, Y=Y)
         assert torch.equal(Y, Y0)
     assert binding.monarch_attn_device_status() == 0
+
+
+# ------------------------------------------------------------------ sequences of different lengths
+@pytest.mark.parametrize("N,b,d,T,dtype,lens,launches", [
+    (24, 4, 8, 2, "f32", [24, 17, 9, 3, 12], 4),            # generic kernels, tiny
+    (210, 14, 64, 2, "f16", [197, 210, 120, 29, 14, 1], 1),  # fused per-head kernel: ViT-like batch
+    (384, 24, 64, 1, "bf16", [384, 300, 100, 23], 1),       # fused kernel, m != b
+    (256, 16, 64, 3, "f16", [256, 250, 130, 40], 6),        # three rounds: generic kernels
+    (1024, 32, 64, 2, "bf16", [1024, 700, 333, 64, 31], 4),  # longer than the fused kernel takes
+])
+def test_batched_sequences_of_different_lengths_match_the_oracle(N, b, d, T, dtype, lens, launches):
+    """App. C.3, batches padded to a maximum length: one length per batch entry, including lengths
+    more than a block short of N (key blocks lying wholly in the padding).  Valid rows must match
+    the oracle's reading (each sequence's own problem); rows past a sequence's own padded length
+    are zero; non-finite garbage in the absent blocks of Q, K, V is never read."""
+    batch, heads = len(lens), 3
+    Q, K, V = wl.make_qkv(batch, heads, N, d, dtype, min(8, d), 1.0, seed=N + T)
+    ref = mo.monarch_attention(Q, K, V, b, T, n_valid=np.array(lens))
+    Qg, Kg, Vg = Q.copy(), K.copy(), V.copy()
+    for e, n in enumerate(lens):
+        own = -(-n // b) * b
+        Kg[e, :, n:own] = 7.0          # padding inside the last block: any finite values
+        Vg[e, :, n:own] = -9.0
+        Qg[e, :, own:] = np.nan        # absent blocks: never read
+        Kg[e, :, own:] = np.inf
+        Vg[e, :, own:] = np.nan
+    Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Qg, Kg, Vg))
+    sl = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    Y = binding.monarch_attn_fwd_varlen(Qd, Kd, Vd, b, T, sl)
+    torch.cuda.synchronize()
+    assert binding.monarch_attn_last_launch_count() == launches
+    Y = Y.float().cpu().numpy().astype(np.float64)
+    for e, n in enumerate(lens):
+        own = -(-n // b) * b
+        for h in range(heads):
+            got, want = Y[e, h, :n], ref[e, h, :n]
+            assert np.isfinite(got).all()
+            err = np.linalg.norm(got - want) / np.linalg.norm(want)
+            assert err <= TOL[dtype], (e, h, n, err)
+        assert np.all(Y[e, :, own:] == 0.0)
+    # a full-length batch is the plain forward pass
+    full = torch.full((batch,), N, dtype=torch.int32, device="cuda")
+    Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))
+    a = binding.monarch_attn_fwd_varlen(Qd, Kd, Vd, b, T, full)
+    same_path = binding.MA_PATH_FUSED_SMALL if launches == 1 else binding.MA_PATH_GENERIC
+    assert torch.equal(a, binding.monarch_attn_fwd_ex(Qd, Kd, Vd, b, T, path=same_path))
+
+
+def test_varlen_entry_point_argument_errors():
+    Q, K, V = (torch.zeros(2, 1, 16, 8, device="cuda") for _ in range(3))
+    with pytest.raises(ValueError):
+        binding.monarch_attn_fwd_varlen(Q, K, V, 4, 1, torch.tensor([16, 8], device="cuda"))          # int64
+    with pytest.raises(ValueError):
+        binding.monarch_attn_fwd_varlen(Q, K, V, 4, 1, torch.tensor([16], dtype=torch.int32, device="cuda"))
+    with pytest.raises(ValueError):
+        binding.monarch_attn_fwd_ex(Q, K, V, 4, 1, Y=torch.zeros(2, 1, 16, 4, device="cuda"))          # wrong shape
+    with pytest.raises(ValueError):
+        binding.monarch_attn_fwd_ex(Q, K, V, 4, 1, Y=torch.zeros(2, 1, 16, 8, device="cuda", dtype=torch.float16))
+    # lengths outside [1, N] are clamped into it
+    sl = torch.tensor([99, -5], dtype=torch.int32, device="cuda")
+    Y = binding.monarch_attn_fwd_varlen(Q + 1.0, K, V + 2.0, 4, 1, sl)
+    assert bool(torch.isfinite(Y).all())
