@@ -97,23 +97,52 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- reference arm
-def oracle_sample(w: wl.Workload, budget_s: float):
-    """Times the fp64 oracle, as it stands, on whole heads of the workload until the budget is
-    used; returns (tokens_per_s, heads_done, seconds, threads)."""
+def _oracle_head(args):
+    """One whole head through the fp64 oracle (runs in a worker process, one BLAS thread)."""
     from oracle import monarch_oracle
-    Q, K, V = wl.make_qkv(1, min(w.heads, 16), w.N, w.d, w.dtype, w.rank, w.s, w.seed)
-    monarch_oracle.monarch_attention_head(Q[0, 0, :w.b * 2], K[0, 0, :w.b * 2], V[0, 0, :w.b * 2],
-                                          w.b, 1)   # import/warm-up
-    done, t0 = 0, time.perf_counter()
-    while True:
-        h = done % Q.shape[1]
-        monarch_oracle.monarch_attention_head(Q[0, h], K[0, h], V[0, h], w.b, w.T)
-        done += 1
-        el = time.perf_counter() - t0
-        if el >= budget_s or done >= w.BH:
-            break
+    Q, K, V, b, T = args
+    monarch_oracle.monarch_attention_head(Q, K, V, b, T)
+    return 1
+
+
+def _one_blas_thread():
+    """One BLAS thread per worker process: the host cores are the workers."""
+    try:
+        from threadpoolctl import threadpool_limits
+        threadpool_limits(1)
+    except Exception:
+        pass
+
+
+def host_cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def oracle_sample(w: wl.Workload, budget_s: float):
+    """Times the fp64 oracle, as it stands, on whole heads of the workload, one head per host core
+    at a time (the (batch, head) units are independent), until the budget is used; returns
+    (tokens_per_s, heads_done, seconds, cores).  The rate over the sample is extrapolated to the
+    workload's token count: the sample cycles through the workload's own heads."""
+    import multiprocessing as mp
+    cores = host_cores()
+    n_heads = min(w.heads, max(cores, 4))
+    Q, K, V = wl.make_qkv(1, n_heads, w.N, w.d, w.dtype, w.rank, w.s, w.seed)
+    done = 0
+    with mp.get_context("fork").Pool(cores, initializer=_one_blas_thread) as pool:
+        pool.map(_oracle_head, [(Q[0, 0, :w.b * 2], K[0, 0, :w.b * 2], V[0, 0, :w.b * 2], w.b, 1)] * cores)
+        t0 = time.perf_counter()
+        while True:
+            jobs = [(Q[0, (done + i) % n_heads], K[0, (done + i) % n_heads], V[0, (done + i) % n_heads],
+                     w.b, w.T) for i in range(cores)]
+            done += sum(pool.map(_oracle_head, jobs))
+            el = time.perf_counter() - t0
+            if el >= budget_s:
+                break
     tokens = w.tokens * done / w.BH
-    return tokens / el, done, el, 1
+    return tokens / el, done, el, cores
 
 
 def run_reference(args, w):
@@ -121,20 +150,21 @@ def run_reference(args, w):
     if rank != 0:
         return
     steps, warm = max(1, args.steps), max(0, args.warmup)
-    budget = min(20.0, 150.0 / (steps + warm))
-    vals, heads = [], 0
+    budget = min(15.0, 120.0 / (steps + warm))
+    vals, heads, cores = [], 0, 1
     for i in range(warm + steps):
-        v, heads, _, threads = oracle_sample(w, budget)
+        v, heads, _, cores = oracle_sample(w, budget)
         if i >= warm:
             vals.append(v)
     value = float(np.mean(vals))
-    sample = f"{heads} of {w.BH} (batch, head) units of {w.name} per step, fp64 numpy oracle"
+    sample = (f"{heads} head evaluations of {w.name} (its {w.BH} (batch, head) units in turn) per step on "
+              f"{cores} host cores, fp64 numpy oracle; tokens/s extrapolated from the sample")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": warm, "ms_per_step": 1e3 * w.tokens / value,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "config": workload_config(w, 1),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -142,22 +172,30 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-def workload_config(w, world):
+def workload_config(w, world, strong=False):
     return {"workload": f"{w.name}: batch={w.batch} heads={w.heads} N={w.N} d={w.d} b={w.b} "
                         f"T={w.T} {w.dtype}, rank-{w.rank} component x{w.s}, seed {w.seed}",
-            "per_gpu_batch": w.batch, "global_batch": w.batch * world, "seq_len": w.N,
-            "parallelism": f"(batch,head) units sharded, {world} rank(s), no collective",
+            "per_gpu_batch": w.batch if not strong else None,
+            "global_batch": w.batch * (1 if strong else world), "seq_len": w.N,
+            "parallelism": (f"the configuration's {w.BH} (batch,head) units split over {world} rank(s), "
+                            "no collective" if strong else
+                            f"every rank runs the configuration on its own batch, {world} rank(s), "
+                            "no collective"),
             "l2": "3 rotating input/output sets (>= 3x the call's footprint) so no step re-reads "
                   "data left in the 126 MB L2 by the previous one"}
 
 
 # ----------------------------------------------------------------------------- ours
-def time_config(w, steps, warmup, torch, binding, n_sets=3, dist=None):
-    """Device-timed steps of workload w.  Returns dict with ms_per_step etc."""
+def time_config(w, steps, warmup, torch, binding, n_sets=3, dist=None, units=None):
+    """Device-timed steps of workload w (or, with `units` = (lo, hi), of that slice of its
+    (batch, head) units: strong scaling).  Returns dict with ms_per_step etc."""
     sets = []
     for r in range(n_sets):
-        Q, K, V = wl.make_qkv(w.batch, w.heads, w.N, w.d, w.dtype, w.rank, w.s,
-                              w.seed + 1000 * r + 17 * int(os.environ.get("RANK", "0")))
+        seed = w.seed + 1000 * r + 17 * int(os.environ.get("RANK", "0"))
+        if units is None:
+            Q, K, V = wl.make_qkv(w.batch, w.heads, w.N, w.d, w.dtype, w.rank, w.s, seed)
+        else:      # this rank's units as one batch entry with (hi - lo) heads
+            Q, K, V = wl.make_qkv(1, units[1] - units[0], w.N, w.d, w.dtype, w.rank, w.s, seed)
         Qd, Kd, Vd = (binding.to_device(x, w.dtype) for x in (Q, K, V))
         sets.append((Qd, Kd, Vd, torch.empty_like(Qd)))
     binding.monarch_attn_fwd(sets[0][0], sets[0][1], sets[0][2], w.b, w.T, Y=sets[0][3])  # sizes ws
@@ -182,8 +220,18 @@ def time_config(w, steps, warmup, torch, binding, n_sets=3, dist=None):
     total_ms = evs[0].elapsed_time(evs[-1])
     per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
     assert binding.monarch_attn_device_status() == 0
+    # host time of one call with an idle stream (argument checks, cached tensor maps, launch)
+    host = []
+    for i in range(20):
+        s = sets[i % n_sets]
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        binding.monarch_attn_fwd(s[0], s[1], s[2], w.b, w.T, Y=s[3])
+        host.append((time.perf_counter() - t0) * 1e6)
+    torch.cuda.synchronize()
     return {"total_ms": total_ms, "ms_per_step": total_ms / steps, "min_ms": min(per),
-            "median_ms": statistics.median(per), "launches_per_step": launches, "sets": sets}
+            "median_ms": statistics.median(per), "launches_per_step": launches, "sets": sets,
+            "host_us_per_call": statistics.median(host)}
 
 
 def time_e2e(w, steps, warmup, torch, binding, dist=None):
@@ -208,10 +256,16 @@ def time_e2e(w, steps, warmup, torch, binding, dist=None):
     return e0.elapsed_time(e1) / steps, 3 * nbytes, nbytes
 
 
-# DRAM bytes of ONE launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
-# ncu; see the summaries under profiles/ named for each kernel and workload).
-NCU_TRAFFIC_BYTES = {"C5": 185.5e6 + 31.7e6, "C4": 174.9e6 + 20.7e6, "C3": 132.7e6 + 42.5e6, "C2": 75.5e6 + 4.0e6,
-                     "S1": 62.0e6 + 2.4e6, "S3": (100.7e6 + 31.8e6) + (101.8e6 + 13.0e6)}   # S3: both launches of a step
+def ncu_traffic_bytes(name):
+    """DRAM bytes of ONE step of workload `name` (dram__bytes_read.sum + dram__bytes_write.sum of its
+    kernel launches, from the ncu captures summarised under profiles/): read from
+    profiles/traffic.json, which is written when a capture is summarised; None if not captured."""
+    try:
+        d = json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))
+        e = d["workloads"].get(name)
+        return None if e is None else float(e["dram_read_bytes"]) + float(e["dram_write_bytes"])
+    except Exception:
+        return None
 
 
 def roofline(w, ms, peaks, which):
@@ -221,11 +275,11 @@ def roofline(w, ms, peaks, which):
         ach = w.algorithmic_flops() / (ms * 1e-3) / 1e12
         return {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
                 "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
-                "traffic": NCU_TRAFFIC_BYTES.get(w.name), "of": which + " (sustained)",
+                "traffic": ncu_traffic_bytes(w.name), "of": which + " (sustained)",
                 "scope": "one launch = one step (the tensor path is a single persistent kernel)"}
     ach = w.algorithmic_bytes() / (ms * 1e-3) / 1e9
     return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(w.name), "of": which,
+            "frac": ach / peaks["hbm_gbs"], "traffic": ncu_traffic_bytes(w.name), "of": which,
             "scope": "one step (one launch on the tcgen05 and fused paths, 2T on the tile and generic paths)"}
 
 
@@ -256,6 +310,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="C5", choices=sorted(wl.WORKLOADS) + sorted(wl.EXTRA_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak: every rank runs the whole configuration on its own batch; strong: the "
+                         "configuration's (batch, head) units are split over the ranks")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the other configurations, SDPA context and the CPU baseline")
     args = ap.parse_args()
@@ -282,25 +339,33 @@ def main():
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     peaks, which = load_peaks()
 
+    strong = args.scaling == "strong" and world > 1
+    units = wl.shard_units(w.BH, world, rank) if strong else None
+    if strong and units[1] == units[0]:
+        raise SystemExit(f"--scaling strong: {w.name} has only {w.BH} units for {world} ranks")
     sampler = ClockSampler(local)
     sampler.start()
-    res = time_config(w, steps, warmup, torch, binding, dist=dist)
+    res = time_config(w, steps, warmup, torch, binding, dist=dist, units=units)
     clocks = sampler.stop()
     ms = D.max_over_ranks(res["total_ms"] / steps, device="cuda")
     e2e_ms, h2d, d2h = time_e2e(w, max(3, min(steps, 20)), 3, torch, binding, dist)
     e2e_ms = D.max_over_ranks(e2e_ms, device="cuda")
+    # weak: every rank processed the whole configuration; strong: the ranks shared one
+    job_tokens = w.tokens if strong else world * w.tokens
 
     line = {
-        "metric": METRIC, "value": world * w.tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": job_tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
-        "config": workload_config(w, world),
+        "scaling": "strong" if strong else "weak", "vs_baseline": None, "dtype": w.dtype,
+        "data": "synthetic", "config": workload_config(w, world, strong),
         "clocks": clocks,
         "e2e": {"value": world * w.tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "note": "every rank moves the whole configuration through its own host buffers"},
         "gpu_launches": res["launches_per_step"] * steps,
-        "roofline": roofline(w, ms, peaks, which),
+        "roofline": roofline(w, ms, peaks, which) if not strong else None,
         "min_ms": res["min_ms"], "median_ms": res["median_ms"],
+        "host_us_per_call": res["host_us_per_call"],
     }
 
     if rank == 0 and not args.no_extras and world == 1:
@@ -323,10 +388,11 @@ def main():
             del r
             torch.cuda.empty_cache()
         line["other_configs"] = per
-        v, heads, secs, threads = oracle_sample(w, 12.0)
+        v, heads, secs, threads = oracle_sample(w, 3.0)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                "sample": f"{heads} of {w.BH} (batch, head) units of {w.name} in "
-                                          f"{secs:.1f} s, fp64 numpy oracle"}
+                                "sample": f"{heads} head evaluations of {w.name} (its {w.BH} (batch, head) "
+                                          f"units in turn) in {secs:.1f} s on {threads} host cores, fp64 "
+                                          f"numpy oracle; tokens/s extrapolated from the sample"}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:

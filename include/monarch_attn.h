@@ -67,7 +67,9 @@ typedef enum {
 /* T-step MonarchAttention forward (Eq. 7-10 then Eq. 4) with scale = 1/sqrt(d).
  * Q, K, V, Y: DEVICE pointers.  Uses a per-process, per-device workspace that the library grows
  * on demand (the only allocation it ever makes; call once outside any timed or captured region
- * to pre-size it).  Not safe to call concurrently from several host threads on one device. */
+ * to pre-size it).  One call in flight per device: not safe to call concurrently from several
+ * host threads on one device, nor on two streams whose work may overlap (use monarch_attn_fwd_ex
+ * with a workspace per stream for that; see there). */
 int monarch_attn_fwd(const void* Q, const void* K, const void* V, void* Y,
                      int batch, int heads, int N, int d, int b, int T,
                      int dtype, void* stream);
@@ -80,7 +82,18 @@ size_t monarch_attn_workspace_bytes(int batch, int heads, int N, int d, int b, i
 
 /* As monarch_attn_fwd, with an explicit softmax scale, an explicit path and caller-owned scratch.
  * workspace: DEVICE pointer, 256-byte aligned, at least monarch_attn_workspace_bytes() long; its
- * contents are overwritten.  Allocates nothing. */
+ * contents are overwritten.  Allocates nothing.
+ *
+ * Concurrency.  A workspace serves one call at a time: calls that may overlap on the GPU (different
+ * streams, no dependency) need a workspace each, and monarch_attn_fwd's library-owned workspace
+ * serves one call in flight per device.  The persistent kernels (MA_PATH_TENSOR,
+ * MA_PATH_TENSOR_TMEM; what AUTO picks for d = 64, m = b in {32, 64, 128}) deal their tiles out
+ * statically over one CTA per SM and the CTAs wait for each other's results, so such a launch only
+ * makes progress with every CTA resident: it needs the whole GPU.  The library chains these
+ * launches per device with an event, so two of them never share the SMs whatever streams they are
+ * on; a foreign kernel that holds SMs for longer than the bound of the device-side waits (about a
+ * second) while one of them runs makes the waits run out: the call then ends with undefined output
+ * and monarch_attn_device_status reports MA_ERR_TIMEOUT. */
 int monarch_attn_fwd_ex(const void* Q, const void* K, const void* V, void* Y,
                         int batch, int heads, int N, int d, int b, int T, int dtype,
                         float softmax_scale, int path,

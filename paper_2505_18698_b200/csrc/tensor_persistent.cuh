@@ -216,6 +216,29 @@ inline int sm_count() {   // of the current device
   return sms[dev];
 }
 
+struct PersistentChain {      // one event per device: the end of the last persistent launch
+  std::mutex mu;
+  cudaEvent_t ev[64] = {};
+  bool rec[64] = {};
+  int dev() const {
+    int d = 0;
+    return (cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < 64) ? d : -1;
+  }
+  cudaEvent_t event() {
+    const int d = dev();
+    if (d < 0) return nullptr;
+    if (ev[d] == nullptr && cudaEventCreateWithFlags(&ev[d], cudaEventDisableTiming) != cudaSuccess)
+      ev[d] = nullptr;
+    return ev[d];
+  }
+  bool recorded() const { const int d = dev(); return d >= 0 && rec[d]; }
+  void set_recorded() { const int d = dev(); if (d >= 0) rec[d] = true; }
+};
+inline PersistentChain& persistent_chain() {
+  static PersistentChain c;
+  return c;
+}
+
 template <typename T, int B, int SB>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int T_steps,
                     int dtype, float scale, void* ws, cudaStream_t st, int* launches, int mode,
@@ -276,6 +299,16 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   }
   const int num_sms = sm_count();
   if (num_sms <= 0) return 7;
+  // The grid only makes progress if every CTA is resident (tiles are dealt out statically and wait
+  // on each other's results), i.e. if it has the GPU to itself.  Two such launches on different
+  // streams could split the SMs between them and starve each other, so launches of this family are
+  // chained per device with an event: a later one starts when the earlier one has finished,
+  // whatever streams they are on.
+  PersistentChain& chain = persistent_chain();
+  std::lock_guard<std::mutex> chain_lock(chain.mu);
+  cudaEvent_t ev = chain.event();
+  if (ev == nullptr) return 7;
+  if (chain.recorded() && cudaStreamWaitEvent(st, ev, 0) != cudaSuccess) return 7;
   const int total = 2 * T_steps * P.tiles_per_phase;
   // one launch, dependencies tracked by counters
   P.g_begin = knobs().skip_first_half_step ? P.tiles_per_phase : 0; P.g_end = total; P.check_deps = 1;
@@ -287,6 +320,8 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
     e = launch_decoupled<T, B, SB>(P, grid, st);
   }
   if (e != cudaSuccess) return 7;
+  if (cudaEventRecord(ev, st) != cudaSuccess) return 7;
+  chain.set_recorded();
   *launches = 1;
   return 0;
 }

@@ -734,3 +734,64 @@ def test_varlen_entry_point_argument_errors():
     sl = torch.tensor([99, -5], dtype=torch.int32, device="cuda")
     Y = binding.monarch_attn_fwd_varlen(Q + 1.0, K, V + 2.0, 4, 1, sl)
     assert bool(torch.isfinite(Y).all())
+
+
+# ------------------------------------------------------------------ sharding helper on one GPU
+def test_sharded_forward_on_one_gpu_is_the_plain_call():
+    """monarch_attn_fwd_sharded with one rank (no process group): host tensors are moved to the
+    current device, device tensors are used in place, and the result is the plain call's."""
+    from paper_2505_18698_b200 import distributed as D
+    Q, K, V = wl.make_qkv(2, 3, 256, 64, "f16", 8, 2.0, seed=77)
+    Qd, Kd, Vd = (binding.to_device(x, "f16") for x in (Q, K, V))
+    ref = binding.monarch_attn_fwd(Qd, Kd, Vd, 16, 2)
+    a = D.monarch_attn_fwd_sharded(Qd, Kd, Vd, 16, 2)
+    b_ = D.monarch_attn_fwd_sharded(Qd.cpu(), Kd.cpu(), Vd.cpu(), 16, 2)
+    ys, (lo, hi) = D.monarch_attn_fwd_sharded(Qd, Kd, Vd, 16, 2, gather=False)
+    torch.cuda.synchronize()
+    assert (lo, hi) == (0, 6) and a.shape == ref.shape and b_.is_cuda
+    assert torch.equal(a, ref) and torch.equal(b_, ref) and torch.equal(ys.reshape(ref.shape), ref)
+
+
+# ------------------------------------------------------------------ concurrency and range
+def test_persistent_launches_on_two_streams_do_not_starve_each_other():
+    """The persistent kernels need every CTA resident; the library chains such launches per device,
+    so two calls on two streams (a workspace each) both finish with correct results."""
+    w = wl.WORKLOADS["C4"]
+    Q, K, V = wl.make_qkv(1, 8, w.N, w.d, w.dtype, w.rank, w.s, seed=61)
+    Qd, Kd, Vd = (binding.to_device(x, w.dtype) for x in (Q, K, V))
+    need = binding.monarch_attn_workspace_bytes(1, 8, w.N, w.d, w.b, w.T, Qd.dtype, binding.MA_PATH_TENSOR)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    ws = [torch.zeros(need, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    ys = [torch.empty_like(Qd) for _ in range(2)]
+    torch.cuda.synchronize()
+    for rep in range(4):
+        for i, (st, path) in enumerate(((s1, binding.MA_PATH_TENSOR), (s2, binding.MA_PATH_TENSOR_TMEM))):
+            binding.monarch_attn_fwd_ex(Qd, Kd, Vd, w.b, w.T, path=path, workspace=ws[i], Y=ys[i], stream=st)
+    torch.cuda.synchronize()
+    assert binding.monarch_attn_device_status(ws[0]) == 0 and binding.monarch_attn_device_status(ws[1]) == 0
+    ref = mo.monarch_attention(Q, K, V, w.b, w.T)
+    for y in ys:
+        assert rel_err(y.float().cpu().numpy().astype(np.float64), ref) <= 1e-2
+
+
+@pytest.mark.parametrize("factor", [2.0 ** -22, 2.0 ** 18])
+def test_bf16_values_outside_the_f16_range(factor):
+    """The fused per-head kernel and the tile kernels compute in f16 whatever the input type: bf16
+    inputs are converted on the way in, exact for magnitudes in [6.1e-5, 65504], clamped or flushed
+    beyond.  bf16 V scaled far outside that range therefore comes back finite but wrong from those
+    paths (documented in the header), while the generic kernels (fp32) hold the tolerance: that is
+    the path for such inputs."""
+    Q, K, V = wl.make_qkv(1, 4, 256, 64, "bf16", 8, 1.0, seed=5)
+    V = wl.round_to_dtype(V * np.float32(factor), "bf16")
+    ref = mo.monarch_attention(Q, K, V, 16, 2)
+    Yg = gpu_forward(Q, K, V, "bf16", 16, 2, binding.MA_PATH_GENERIC)
+    assert rel_err(Yg, ref) <= 1e-2
+    for path in (binding.MA_PATH_FUSED_SMALL, binding.MA_PATH_TILE_MMA):
+        Yf = gpu_forward(Q, K, V, "bf16", 16, 2, path)
+        assert np.isfinite(Yf).all()
+        assert rel_err(Yf, ref) > 1e-2          # out of range for f16 arithmetic: not silently "fine"
+    # inside the range the same paths are within tolerance
+    V_ok = wl.round_to_dtype(V / np.float32(factor), "bf16")
+    ref_ok = mo.monarch_attention(Q, K, V_ok, 16, 2)
+    for path in (binding.MA_PATH_FUSED_SMALL, binding.MA_PATH_TILE_MMA):
+        assert rel_err(gpu_forward(Q, K, V_ok, "bf16", 16, 2, path), ref_ok) <= 1e-2

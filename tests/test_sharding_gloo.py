@@ -1,6 +1,7 @@
-"""The N > 1 path on CPU: two gloo ranks partition the (batch, head) units, each computes its own
-shard (with the oracle standing in for the GPU call), and the pieces reassemble to the
-single-process result with no data-path collective."""
+"""The N > 1 path on CPU: gloo ranks partition the (batch, head) units through the same helper the
+GPU path uses (monarch_attn_fwd_sharded), each computes its own shard (a CPU stand-in takes the
+place of the library call: the partition and the gather are what is exercised here), and the pieces
+reassemble to the single-process result with no data-path collective."""
 import os
 import socket
 
@@ -20,39 +21,62 @@ def _free_port():
     return p
 
 
-def _worker(rank, world, port, q):
+def _stand_in(Qs, Ks, Vs, b, T):
+    """What the library call computes, on the host: [1, units, N, d] -> [1, units, N, d]."""
+    return torch.from_numpy(mo.monarch_attention(Qs.numpy(), Ks.numpy(), Vs.numpy(), b, T))
+
+
+def _worker(rank, world, port, q, shape):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
                       LOCAL_RANK=str(rank), WORLD_SIZE=str(world))
     r, _, w = D.init("gloo")
     assert (r, w) == (rank, world)
-    batch, heads, N, d, b, T = 3, 3, 24, 4, 6, 2
-    Q, K, V = wl.make_qkv(batch, heads, N, d, "f32", 2, 1.0, seed=9)
-    total = batch * heads
-    lo, hi = D.my_units(total)
-    flat = lambda x: x.reshape(total, N, d)
-    mine = mo.monarch_attention(flat(Q)[lo:hi], flat(K)[lo:hi], flat(V)[lo:hi], b, T)
+    batch, heads, N, d, b, T = shape
+    Q, K, V = (torch.from_numpy(x).double() for x in wl.make_qkv(batch, heads, N, d, "f32", 2, 1.0, seed=9))
+    mine, (lo, hi) = D.monarch_attn_fwd_sharded(Q, K, V, b, T, gather=False, fwd=_stand_in)
+    assert mine.shape == (hi - lo, N, d) and (lo, hi) == D.my_units(batch * heads)
     D.barrier()
     step_time = D.max_over_ranks(1.0 + rank)            # max over ranks, as the benchmark does
-    full = D.gather_units(torch.from_numpy(mine), total).numpy()
+    full = D.monarch_attn_fwd_sharded(Q, K, V, b, T, gather=True, fwd=_stand_in)
     if rank == 0:
-        q.put((lo, hi, step_time, full))
+        q.put((lo, hi, step_time, full.numpy()))
     D.barrier()
     torch.distributed.destroy_process_group()
 
 
-def test_two_gloo_ranks_partition_heads_and_reassemble():
-    world = 2
+def _run(world, shape):
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
     port = _free_port()
-    procs = [ctx.Process(target=_worker, args=(r, world, port, q)) for r in range(world)]
+    procs = [ctx.Process(target=_worker, args=(r, world, port, q, shape)) for r in range(world)]
     for p in procs:
         p.start()
-    lo, hi, step_time, full = q.get(timeout=120)
+    out = q.get(timeout=120)
     for p in procs:
         p.join(timeout=120)
         assert p.exitcode == 0
+    return out
+
+
+def test_two_gloo_ranks_partition_heads_and_reassemble():
+    shape = (3, 3, 24, 4, 6, 2)
+    lo, hi, step_time, full = _run(2, shape)
     assert (lo, hi) == (0, 5) and step_time == 2.0
     Q, K, V = wl.make_qkv(3, 3, 24, 4, "f32", 2, 1.0, seed=9)
-    ref = mo.monarch_attention(Q, K, V, 6, 2).reshape(9, 24, 4)
+    ref = mo.monarch_attention(Q.astype(np.float64), K.astype(np.float64), V.astype(np.float64), 6, 2)
     assert np.array_equal(full, ref)
+
+
+def test_more_ranks_than_units_leaves_some_ranks_idle():
+    shape = (1, 2, 12, 4, 4, 1)
+    lo, hi, step_time, full = _run(3, shape)
+    assert (lo, hi) == (0, 1) and step_time == 3.0
+    Q, K, V = wl.make_qkv(1, 2, 12, 4, "f32", 2, 1.0, seed=9)
+    ref = mo.monarch_attention(Q.astype(np.float64), K.astype(np.float64), V.astype(np.float64), 4, 1)
+    assert np.array_equal(full, ref)
+
+
+def test_without_a_process_group_it_is_the_single_process_call():
+    Q, K, V = (torch.from_numpy(x).double() for x in wl.make_qkv(2, 2, 12, 4, "f32", 2, 1.0, seed=3))
+    full = D.monarch_attn_fwd_sharded(Q, K, V, 4, 2, fwd=_stand_in)
+    assert np.array_equal(full.numpy(), mo.monarch_attention(Q.numpy(), K.numpy(), V.numpy(), 4, 2))
