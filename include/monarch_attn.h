@@ -55,6 +55,12 @@ typedef enum {
   MA_PATH_TENSOR_BASIC = 4,  /* one CTA per tile, one launch per half-step (no pipelining);
                                 m = b in {64, 128}; the plain statement the persistent kernels are
                                 tested against */
+  MA_PATH_FUSED_F32 = 5, /* fp32 arithmetic and fp32 states in shared memory, one launch for all T
+                            rounds: any dtype, any N = m*b whose K, V and one position's states fit
+                            shared memory (N <= ~430 at d = 64); a CTA owns a set of in-block
+                            positions of one head (the recursion is independent across them), so a
+                            single small head is spread over up to b CTAs.  What AUTO takes for
+                            fp32 inputs of that size */
   MA_PATH_FUSED_SMALL = 7, /* the same idea for any block shape: f16/bf16, m and b <= 32 (m need not
                              equal b), d <= 64 a multiple of 8, N <= 580 for T = 1 and <= 440 for
                              T > 1 (the states of a head must fit shared memory); f16 arithmetic */

@@ -20,6 +20,7 @@ HEADER_PATH = os.path.join(INCLUDE_DIR, "monarch_attn.h")
 
 MA_F32, MA_F16, MA_BF16 = 0, 1, 2
 MA_PATH_AUTO, MA_PATH_GENERIC, MA_PATH_TENSOR, MA_PATH_TENSOR_TMEM, MA_PATH_TENSOR_BASIC = 0, 1, 2, 3, 4
+MA_PATH_FUSED_F32 = 5
 MA_PATH_FUSED_SMALL = 7
 MA_PATH_TILE_MMA = 8
 MA_OK = 0
@@ -114,6 +115,25 @@ def _shape_of(Q, K, V):
     return tuple(int(x) for x in Q.shape)
 
 
+class _on_device_of:
+    """Runs the body with the tensor's device current; free when it already is."""
+    __slots__ = ("idx", "prev")
+
+    def __init__(self, t):
+        self.idx = t.device.index if t.is_cuda else None
+        self.prev = None
+
+    def __enter__(self):
+        if self.idx is not None and self.idx != torch.cuda.current_device():
+            self.prev = torch.cuda.current_device()
+            torch.cuda.set_device(self.idx)
+
+    def __exit__(self, *exc):
+        if self.prev is not None:
+            torch.cuda.set_device(self.prev)
+        return False
+
+
 def _out_like(Y, Q, what="Y"):
     """A caller-supplied output must match the input exactly: the kernels write Q.numel() elements
     of Q's dtype through its pointer, on Q's device."""
@@ -138,7 +158,7 @@ def _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code, paths):
     return torch.zeros(max(need, 256), dtype=torch.uint8, device=Q.device)
 
 
-_ANY_PATH = (MA_PATH_TENSOR, MA_PATH_GENERIC, MA_PATH_TILE_MMA, MA_PATH_FUSED_SMALL)
+_ANY_PATH = (MA_PATH_TENSOR, MA_PATH_GENERIC, MA_PATH_TILE_MMA, MA_PATH_FUSED_SMALL, MA_PATH_FUSED_F32)
 
 
 def monarch_attn_workspace_bytes(batch, heads, N, d, b, T, dtype, path=MA_PATH_AUTO) -> int:
@@ -154,7 +174,7 @@ def monarch_attn_fwd(Q, K, V, b, T, Y=None, stream=None):
         raise MonarchAttnError(-2, "monarch_attn_fwd needs CUDA tensors; there is no CPU path")
     batch, heads, N, d = _shape_of(Q, K, V)
     Y = _out_like(Y, Q)
-    with torch.cuda.device(Q.device):
+    with _on_device_of(Q):
         _check(lib.monarch_attn_fwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                     batch, heads, N, d, b, T, _TORCH_TO_CODE[Q.dtype],
                                     _stream_ptr(stream)))
@@ -174,7 +194,7 @@ def monarch_attn_fwd_ex(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, wo
         softmax_scale = 1.0 / math.sqrt(d)
     Y = _out_like(Y, Q)
     workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code, (path,))
-    with torch.cuda.device(Q.device):
+    with _on_device_of(Q):
         _check(lib.monarch_attn_fwd_ex(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                        batch, heads, N, d, b, T, code, float(softmax_scale), int(path),
                                        workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
@@ -195,7 +215,7 @@ def monarch_attn_fwd_objective(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_A
     Y = _out_like(Y, Q)
     lse = torch.empty((batch, heads, N), dtype=torch.float32, device=Q.device)
     workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code, _ANY_PATH)
-    with torch.cuda.device(Q.device):
+    with _on_device_of(Q):
         _check(lib.monarch_attn_fwd_objective(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                               batch, heads, N, d, b, T, code, float(softmax_scale),
                                               int(path), lse.data_ptr(), workspace.data_ptr(),
@@ -220,7 +240,7 @@ def monarch_attn_fwd_bshd(Q, K, V, b, T, softmax_scale=None, path=MA_PATH_AUTO, 
         softmax_scale = 1.0 / math.sqrt(d)
     Y = _out_like(Y, Q)
     workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code, _ANY_PATH)
-    with torch.cuda.device(Q.device):
+    with _on_device_of(Q):
         _check(lib.monarch_attn_fwd_bshd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                          batch, N, heads, d, b, T, code, float(softmax_scale), int(path),
                                          workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
@@ -241,7 +261,7 @@ def monarch_attn_fwd_padded(Q, K, V, b, T, n_valid, softmax_scale=None, workspac
         softmax_scale = 1.0 / math.sqrt(d)
     Y = _out_like(Y, Q)
     workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code, _ANY_PATH)
-    with torch.cuda.device(Q.device):
+    with _on_device_of(Q):
         _check(lib.monarch_attn_fwd_padded(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                            batch, heads, N, d, b, T, code, float(softmax_scale),
                                            int(n_valid), workspace.data_ptr(), workspace.numel(),
@@ -267,7 +287,7 @@ def monarch_attn_fwd_varlen(Q, K, V, b, T, seq_len, softmax_scale=None, workspac
     Y = _out_like(Y, Q)
     workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code,
                                (MA_PATH_GENERIC, MA_PATH_FUSED_SMALL))
-    with torch.cuda.device(Q.device):
+    with _on_device_of(Q):
         _check(lib.monarch_attn_fwd_varlen(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                            batch, heads, N, d, b, T, code, float(softmax_scale),
                                            seq_len.data_ptr(), workspace.data_ptr(), workspace.numel(),
@@ -304,7 +324,7 @@ def monarch_attn_fwd_noalloc(Q, K, V, b, T, Y, stream=None):
     if Y is None:
         raise ValueError("monarch_attn_fwd_noalloc allocates nothing: pass the output tensor Y")
     _out_like(Y, Q)
-    with torch.cuda.device(Q.device):
+    with _on_device_of(Q):
         _check(lib.monarch_attn_fwd_noalloc(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                             batch, heads, N, d, b, T, _TORCH_TO_CODE[Q.dtype],
                                             _stream_ptr(stream)))

@@ -14,6 +14,7 @@
 #include "tensor_persistent.cuh"
 #include "tensor_decoupled.cuh"
 #include "fused_small.cuh"
+#include "fused_f32.cuh"
 #include "tile_mma.cuh"
 
 namespace ma {
@@ -170,10 +171,13 @@ static int resolve_path(const Problem& p, int path) {
     if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TENSOR;
     if (fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
     if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
+    // fp32 inputs: short sequences in one launch with the states in shared memory
+    if (p.dtype == MA_F32 && p.BH <= 65535 && ffused::supported(p.N, p.d, p.b, p.m)) return MA_PATH_FUSED_F32;
     if (generic_supported(p)) return MA_PATH_GENERIC;
     return -1;
   }
   if (path == MA_PATH_GENERIC) return generic_supported(p) ? path : -1;
+  if (path == MA_PATH_FUSED_F32) return (p.BH <= 65535 && ffused::supported(p.N, p.d, p.b, p.m)) ? path : -1;
   if (path == MA_PATH_TILE_MMA) return tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
   if (path == MA_PATH_FUSED_SMALL)
     return fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T) ? path : -1;
@@ -199,14 +203,14 @@ static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused
     return generic_supported(p) ? MA_PATH_GENERIC : -1;
   }
   if (path == MA_PATH_TENSOR || path == MA_PATH_TILE_MMA || path == MA_PATH_GENERIC ||
-      (path == MA_PATH_FUSED_SMALL && with_fused_small))
+      path == MA_PATH_FUSED_F32 || (path == MA_PATH_FUSED_SMALL && with_fused_small))
     return resolve_path(p, path);
   return -1;
 }
 
 static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
-  if (resolved == MA_PATH_FUSED_SMALL) return kStatusBytes;   // no states leave the chip
+  if (resolved == MA_PATH_FUSED_SMALL || resolved == MA_PATH_FUSED_F32) return kStatusBytes;   // no states leave the chip
   if (resolved == MA_PATH_TILE_MMA) return tile::workspace_bytes(p.BH, p.N, p.d, p.T);
   if (resolved == MA_PATH_TENSOR_BASIC) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
   if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_TMEM)
@@ -260,6 +264,11 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   if (resolved == MA_PATH_FUSED_SMALL) {
     int rc = fsmall::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.m, p.T, p.dtype, scale, p.n_valid, p.H, p.lse, st,
                             p.seq_len, p.heads);
+    if (rc == MA_OK) g_last_launches = 1;
+    return rc;
+  }
+  if (resolved == MA_PATH_FUSED_F32) {
+    int rc = ffused::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.m, p.T, p.dtype, scale, p.n_valid, p.H, p.lse, st);
     if (rc == MA_OK) g_last_launches = 1;
     return rc;
   }
@@ -341,6 +350,7 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
   if (p.T <= 2 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) r = MA_PATH_FUSED_SMALL;
   else if (resolve_path(p, MA_PATH_AUTO) == MA_PATH_TENSOR && p.b != 32) r = MA_PATH_TENSOR;
   else if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) r = MA_PATH_TILE_MMA;
+  else if (p.dtype == MA_F32 && p.BH <= 65535 && ffused::supported(p.N, p.d, p.b, p.m)) r = MA_PATH_FUSED_F32;
   else if (generic_supported(p)) r = MA_PATH_GENERIC;
   if (r < 0) return MA_ERR_UNSUPPORTED;
   p.n_valid = n_valid;

@@ -795,3 +795,56 @@ def test_bf16_values_outside_the_f16_range(factor):
     ref_ok = mo.monarch_attention(Q, K, V_ok, 16, 2)
     for path in (binding.MA_PATH_FUSED_SMALL, binding.MA_PATH_TILE_MMA):
         assert rel_err(gpu_forward(Q, K, V_ok, "bf16", 16, 2, path), ref_ok) <= 1e-2
+
+
+# ------------------------------------------------------------------ fused fp32 kernel
+@pytest.mark.parametrize("N,b,d,T,dtype,batch,heads", [
+    (256, 16, 64, 1, "f32", 1, 1),          # configuration C1: one head over 16 CTAs
+    (256, 16, 64, 3, "f32", 2, 3),
+    (210, 14, 40, 2, "f32", 1, 5),          # m != b, d not a multiple of 4 floats per lane
+    (24, 2, 7, 2, "f32", 1, 2), (24, 12, 5, 3, "f32", 3, 1), (6, 6, 4, 2, "f32", 1, 1), (6, 1, 4, 2, "f32", 1, 1),
+    (384, 24, 64, 2, "f32", 40, 12),        # many heads: a CTA takes all positions of a head
+    (384, 96, 48, 1, "f32", 1, 3),          # blocks wider than a warp
+    (256, 16, 64, 3, "f16", 2, 2), (210, 15, 64, 2, "bf16", 1, 3),   # 16-bit inputs, fp32 arithmetic
+])
+def test_fused_f32_kernel_matches_oracle(N, b, d, T, dtype, batch, heads):
+    """One launch, fp32 states in shared memory, positions of a head spread over CTAs."""
+    err = check(batch, heads, N, d, b, T, dtype, rank=min(8, d), s=1.0, seed=N + T + heads,
+                path=binding.MA_PATH_FUSED_F32)
+    assert binding.monarch_attn_last_launch_count() == 1
+    if dtype == "f32":
+        assert err <= 1e-5
+
+
+def test_fused_f32_kernel_is_the_default_for_short_fp32_sequences_and_serves_the_other_entry_points():
+    Q, K, V = wl.make_qkv(2, 3, 210, 40, "f32", 8, 1.0, seed=3)
+    Qd, Kd, Vd = (binding.to_device(x, "f32") for x in (Q, K, V))
+    a = binding.monarch_attn_fwd(Qd, Kd, Vd, 14, 2)
+    assert binding.monarch_attn_last_launch_count() == 1
+    g = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 14, 2, path=binding.MA_PATH_GENERIC)
+    assert float((a - g).abs().max()) <= 1e-5 * float(g.abs().max())
+    # other layout
+    Qs, Ks, Vs = (x.transpose(1, 2).contiguous() for x in (Qd, Kd, Vd))
+    c = binding.monarch_attn_fwd_bshd(Qs, Ks, Vs, 14, 2)
+    assert binding.monarch_attn_last_launch_count() == 1 and torch.equal(c.transpose(1, 2), a)
+    # objective value, row by row
+    Y, lse = binding.monarch_attn_fwd_objective(Qd, Kd, Vd, 14, 2)
+    assert binding.monarch_attn_last_launch_count() == 1 and torch.equal(Y, a)
+    for h in range(3):
+        _, L, R = mo.monarch_attention_head(Q[0, h], K[0, h], V[0, h], 14, 2, return_factors=True)
+        rows = mo.final_row_lse(R, Q[0, h], K[0, h], 14, 1.0 / np.sqrt(40))
+        assert np.abs(lse[0, h].double().cpu().numpy() - rows).max() <= 1e-4
+    # padding mask
+    Kp, Vp = K.copy(), V.copy()
+    Kp[:, :, 197:] = 5.0
+    Vp[:, :, 197:] = -70.0
+    Yp = binding.monarch_attn_fwd_padded(Qd, binding.to_device(Kp, "f32"), binding.to_device(Vp, "f32"), 14, 2, 197)
+    assert binding.monarch_attn_last_launch_count() == 1
+    ref = mo.monarch_attention(Q, Kp, Vp, 14, 2, n_valid=197)
+    assert rel_err(Yp.double().cpu().numpy()[:, :, :197], ref[:, :, :197]) <= 1e-5
+    # too long for shared memory: the generic kernels take over
+    Q2, K2, V2 = (torch.randn(1, 1, 1024, 64, device="cuda") for _ in range(3))
+    binding.monarch_attn_fwd(Q2, K2, V2, 32, 1)
+    assert binding.monarch_attn_last_launch_count() == 2
+    with pytest.raises(binding.MonarchAttnError):
+        binding.monarch_attn_fwd_ex(Q2, K2, V2, 32, 1, path=binding.MA_PATH_FUSED_F32)
