@@ -452,9 +452,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             mbar_arrive(&bars->stage_free);
           }
           tma_store_wait_all();                 // rows (and c_L / c_R) are in global memory
+          // (a reduction with release semantics: nothing comes back, so the thread does not wait
+          // for the round trip to the counter's home in L2 as it would with a fence and an atomic)
           asm volatile("fence.proxy.async.global;" ::: "memory");
-          __threadfence();
-          atomicAdd(P.counters + t.p * P.BH + t.h, 1);
+          asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(P.counters + t.p * P.BH + t.h) : "memory");
           if (EXTRA) stamp(P, n, 7);
           round += nr;
         }

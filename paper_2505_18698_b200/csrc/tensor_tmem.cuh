@@ -544,6 +544,12 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
         TileIter it(P, first_g, stride_g, kBlocks);
         int round = 0, mine = 0;                 // staging rounds so far: all, and this thread's
         int* pending = nullptr;                  // counter of a store not yet known complete
+        // (a reduction with release semantics: nothing comes back, so the thread does not wait for
+        // the round trip to the counter's home in L2 as it would with a fence and an atomic)
+        auto signal = [&](int* ctr) {
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+          asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(ctr) : "memory");
+        };
         for (int n = 0; n < n_total; ++n, it.next()) {
           const Tile t = it.get();
           const int nr = rounds_of(t);
@@ -557,9 +563,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
             tma_store_commit();
             if (pending != nullptr) {
               tma_store_wait_all_but_one();
-              asm volatile("fence.proxy.async.global;" ::: "memory");
-              __threadfence();
-              atomicAdd(pending, 1);
+              signal(pending);
             }
             tma_store_wait_read();
             mbar_arrive(&bars->stage_free[w]);
@@ -567,18 +571,14 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
             ++mine;
             if (!mbar_poll_addr(smem_u32(&bars->stage_ready[w]), mine & 1)) {
               tma_store_wait_all();
-              asm volatile("fence.proxy.async.global;" ::: "memory");
-              __threadfence();
-              atomicAdd(pending, 1);
+              signal(pending);
               pending = nullptr;
             }
           }
         }
         if (pending != nullptr) {
           tma_store_wait_all();
-          asm volatile("fence.proxy.async.global;" ::: "memory");
-          __threadfence();
-          atomicAdd(pending, 1);
+          signal(pending);
         }
       }
     }
