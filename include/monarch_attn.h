@@ -61,6 +61,11 @@ typedef enum {
                             positions of one head (the recursion is independent across them), so a
                             single small head is spread over up to b CTAs.  What AUTO takes for
                             fp32 inputs of that size */
+  MA_PATH_FUSED_JSPLIT = 6, /* N = 1024 as m = b = 32 (d = 64, f16/bf16, standard layout, no mask, no
+                              row_lse): all T rounds in one launch; a head is split over four CTAs
+                              by in-block position (Eq. 7-10 never mix two positions j), each
+                              keeping K and its own rows of Q and of the states in shared memory.
+                              f16 arithmetic with plain f16 states: what AUTO takes for T <= 2 */
   MA_PATH_FUSED_SMALL = 7, /* the same idea for any block shape: f16/bf16, m and b <= 32 (m need not
                              equal b), d <= 64 a multiple of 8, N <= 580 for T = 1 and <= 440 for
                              T > 1 (the states of a head must fit shared memory); f16 arithmetic */

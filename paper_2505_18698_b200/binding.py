@@ -21,6 +21,7 @@ HEADER_PATH = os.path.join(INCLUDE_DIR, "monarch_attn.h")
 MA_F32, MA_F16, MA_BF16 = 0, 1, 2
 MA_PATH_AUTO, MA_PATH_GENERIC, MA_PATH_TENSOR, MA_PATH_TENSOR_TMEM, MA_PATH_TENSOR_BASIC = 0, 1, 2, 3, 4
 MA_PATH_FUSED_F32 = 5
+MA_PATH_FUSED_JSPLIT = 6
 MA_PATH_FUSED_SMALL = 7
 MA_PATH_TILE_MMA = 8
 MA_OK = 0

@@ -15,6 +15,7 @@
 #include "tensor_decoupled.cuh"
 #include "fused_small.cuh"
 #include "fused_f32.cuh"
+#include "fused_jsplit.cuh"
 #include "tile_mma.cuh"
 
 namespace ma {
@@ -158,13 +159,17 @@ static int launch_generic(const Problem& p, const void* Q, const void* K, const 
 }
 
 // ------------------------------------------------------------------ path selection
-static int resolve_path(const Problem& p, int path) {
+// `plain`: the call has the standard layout, no mask and no row_lse output (the kernel split by
+// in-block position serves nothing else).
+static int resolve_path(const Problem& p, int path, bool plain = true) {
   if (path == MA_PATH_AUTO) {
     // From the third round on, plain 16-bit states are too coarse on peaky logits (they are fed
     // back round after round: about one head in 300 of the N = 256 recipe exceeds 1e-2 at T = 3).
     // The fused per-head kernel and the tcgen05 kernels keep such states; the tile kernels switch to
     // hi + lo pairs from T = 3 on, so they take every 16-bit shape they support then.
     if (p.T >= 3 && tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
+    // N = 1024 as 32 x 32: one launch, a head split over four CTAs by in-block position
+    if (plain && p.T <= 2 && jsplit::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_FUSED_JSPLIT;
     // Short sequences with small blocks: one CTA per head, states in shared memory.
     if (p.b <= 16 && p.m <= 16 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T))
       return MA_PATH_FUSED_SMALL;
@@ -178,6 +183,8 @@ static int resolve_path(const Problem& p, int path) {
   }
   if (path == MA_PATH_GENERIC) return generic_supported(p) ? path : -1;
   if (path == MA_PATH_FUSED_F32) return (p.BH <= 65535 && ffused::supported(p.N, p.d, p.b, p.m)) ? path : -1;
+  if (path == MA_PATH_FUSED_JSPLIT)
+    return (plain && jsplit::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) ? path : -1;
   if (path == MA_PATH_TILE_MMA) return tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH) ? path : -1;
   if (path == MA_PATH_FUSED_SMALL)
     return fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T) ? path : -1;
@@ -197,20 +204,21 @@ static int resolve_path(const Problem& p, int path) {
 // AUTO, TENSOR, FUSED_SMALL, TILE_MMA or GENERIC; -1 if none applies.
 static int resolve_tensor_or_generic(const Problem& p, int path, bool with_fused_small = false) {
   if (path == MA_PATH_AUTO) {
-    const int r = resolve_path(p, MA_PATH_AUTO);
+    const int r = resolve_path(p, MA_PATH_AUTO, false);
     if (r != MA_PATH_FUSED_SMALL || with_fused_small) return r;
     if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
     return generic_supported(p) ? MA_PATH_GENERIC : -1;
   }
   if (path == MA_PATH_TENSOR || path == MA_PATH_TILE_MMA || path == MA_PATH_GENERIC ||
       path == MA_PATH_FUSED_F32 || (path == MA_PATH_FUSED_SMALL && with_fused_small))
-    return resolve_path(p, path);
+    return resolve_path(p, path, false);
   return -1;
 }
 
 static size_t workspace_bytes_for(const Problem& p, int resolved) {
   if (resolved == MA_PATH_GENERIC) return generic_layout(p, nullptr).bytes;
-  if (resolved == MA_PATH_FUSED_SMALL || resolved == MA_PATH_FUSED_F32) return kStatusBytes;   // no states leave the chip
+  if (resolved == MA_PATH_FUSED_SMALL || resolved == MA_PATH_FUSED_F32 || resolved == MA_PATH_FUSED_JSPLIT)
+    return kStatusBytes;   // no states leave the chip
   if (resolved == MA_PATH_TILE_MMA) return tile::workspace_bytes(p.BH, p.N, p.d, p.T);
   if (resolved == MA_PATH_TENSOR_BASIC) return tensor::workspace_bytes(p.BH, p.N, p.d, p.b, p.T);
   if (resolved == MA_PATH_TENSOR || resolved == MA_PATH_TENSOR_TMEM)
@@ -251,6 +259,8 @@ static int grow(void** ptr, size_t* have, size_t need) {
     *ptr = nullptr;
     return MA_ERR_CUDA;
   }
+  // the status word starts clear (kernels that never arm the workspace themselves only ever set it)
+  if (cudaMemset(*ptr, 0, sz < 256 ? sz : 256) != cudaSuccess) return MA_ERR_CUDA;
   *have = sz;
   return MA_OK;
 }
@@ -269,6 +279,11 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
   }
   if (resolved == MA_PATH_FUSED_F32) {
     int rc = ffused::launch(Q, K, V, Y, p.BH, p.N, p.d, p.b, p.m, p.T, p.dtype, scale, p.n_valid, p.H, p.lse, st);
+    if (rc == MA_OK) g_last_launches = 1;
+    return rc;
+  }
+  if (resolved == MA_PATH_FUSED_JSPLIT) {
+    int rc = jsplit::launch(Q, K, V, Y, p.BH, p.T, p.dtype, scale, (int*)ws, st);
     if (rc == MA_OK) g_last_launches = 1;
     return rc;
   }
@@ -348,7 +363,7 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
   // whole key block (b = 64, 128: the mask touches the last block's tiles only); else generic
   int r = -1;
   if (p.T <= 2 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) r = MA_PATH_FUSED_SMALL;
-  else if (resolve_path(p, MA_PATH_AUTO) == MA_PATH_TENSOR && p.b != 32) r = MA_PATH_TENSOR;
+  else if (resolve_path(p, MA_PATH_AUTO, false) == MA_PATH_TENSOR && p.b != 32) r = MA_PATH_TENSOR;
   else if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) r = MA_PATH_TILE_MMA;
   else if (p.dtype == MA_F32 && p.BH <= 65535 && ffused::supported(p.N, p.d, p.b, p.m)) r = MA_PATH_FUSED_F32;
   else if (generic_supported(p)) r = MA_PATH_GENERIC;

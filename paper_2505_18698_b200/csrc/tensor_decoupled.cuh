@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       if (deps && nE < n_total && itE.get().p > 0) ctrE = ld_acquire(counter_of(itE.get()));
       if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
       long long t0 = 0;
-      bool force = false, idle = false;
+      bool idle = false;
       RingPos<kRingE> rE;
       RingPos<kRingL> rL;
       RingPos<kRingV> rV;
@@ -251,10 +251,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         const uint32_t r_e = mbar_poll_addr(bEmptyE + rE.slot * 8, rE.par ^ 1);
         const uint32_t r_l = mbar_poll_addr(bEmptyL + rL.slot * 8, rL.par ^ 1);
         const uint32_t r_v = mbar_poll_addr(bEmptyV + rV.slot * 8, rV.par ^ 1);
-        if (nE < n_total && (force || (r_e & r_l))) {
+        if (nE < n_total && (r_e & r_l)) {
           // (the prefetched counter is looked at only once the slots are free: by then its load
           // has long landed and the thread does not stall on it)
-          bool ok = force || !deps || itE.p == 0 || ctrE >= P.tiles_per_head;
+          bool ok = !deps || itE.p == 0 || ctrE >= P.tiles_per_head;
           if (!ok) {
             ctrE = ld_acquire(counter_of(itE.get()));
             ok = ctrE >= P.tiles_per_head;
@@ -296,8 +296,8 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             did = true;
           }
         }
-        if (nVt < n_total && (force || r_v)) {
-          bool ok = force || !deps || itV.p == 0 || ctrV >= P.tiles_per_head;
+        if (nVt < n_total && r_v) {
+          bool ok = !deps || itV.p == 0 || ctrV >= P.tiles_per_head;
           if (!ok) {
             ctrV = ld_acquire(counter_of(itV.get()));
             ok = ctrV >= P.tiles_per_head;
@@ -319,16 +319,16 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         }
         if (did) {
           idle = false;
-        } else if (!force) {
+        } else {
           if (!idle) {
             idle = true;
             t0 = clock64();
           } else if (bars->abort_flag) {
-            force = true;
+            break;   // stop issuing: what is in flight drains before the CTA leaves
           } else if (clock64() - t0 > P.wait_cycles) {
             report_timeout(P.status, 10);
             bars->abort_flag = 1;
-            force = true;
+            break;   // stop issuing: what is in flight drains before the CTA leaves
           }
           __nanosleep(32);
         }
@@ -343,7 +343,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
       int i1 = 0, i2 = 0;
       TileIter it1(P, first_g, stride_g, kBlocks), it2(P, first_g, stride_g, kBlocks);
       long long t0 = 0;
-      bool force = false, idle = false;
+      bool idle = false;
       RingPos<kRingE> r1E;                        // score MMA: tile i1
       RingPos<kRingL> r1L, r2L;                   // apply MMA: tile i2
       RingPos<kStagesS> r1S;
@@ -361,10 +361,10 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         const uint32_t r_of = mbar_poll_addr(bOFree + r2O.slot * 8, r2O.par ^ 1);
         const uint32_t r_v = mbar_poll_addr(bFullV + rV.slot * 8, rV.par);
         const uint32_t r_l = mbar_poll_addr(bFullL + r1L.slot * 8, r1L.par);
-        if (i2 < i1 && (force || (r_ready & r_of))) {
+        if (i2 < i1 && (r_ready & r_of)) {
           const Tile t = it2.get();
           const bool needV = needs_v(t);
-          if (force || !needV || r_v) {
+          if (!needV || r_v) {
             const int eL2 = r2L.slot, eV = rV.slot, o2 = r2O.slot;
             const uint32_t sL = sL0 + eL2 * kSlot, sV = sV0 + eV * kSlot, sP = sP0 + c * kPBytes;
             const uint32_t tO = tmem_o + o2 * 128;
@@ -386,7 +386,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
             did = true;
           }
         }
-        if (i1 < n_total && i1 < i2 + kStagesS && (force || r_l)) {
+        if (i1 < n_total && i1 < i2 + kStagesS && r_l) {
           const Tile t = it1.get();
           const int eE = r1E.slot, eL1 = r1L.slot, s1 = r1S.slot;
           tc_fence_after();
@@ -406,16 +406,16 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_decoupled(const __grid_co
         }
         if (did) {
           idle = false;
-        } else if (!force) {
+        } else {
           if (!idle) {
             idle = true;
             t0 = clock64();
           } else if (bars->abort_flag) {
-            force = true;
+            break;   // stop issuing: what is in flight drains before the CTA leaves
           } else if (clock64() - t0 > P.wait_cycles) {
             report_timeout(P.status, 20);
             bars->abort_flag = 1;
-            force = true;
+            break;   // stop issuing: what is in flight drains before the CTA leaves
           }
           __nanosleep(20);
         }

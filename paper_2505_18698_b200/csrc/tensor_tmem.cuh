@@ -324,7 +324,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
         if (deps && nE < n_total && itE.get().p > 0) ctrE = ld_acquire(counter_of(itE.get()));
         if (deps && nVt < n_total && itV.get().p > 0) ctrV = ld_acquire(counter_of(itV.get()));
         long long t0 = 0;
-        bool force = false, idle = false;
+        bool idle = false;
         RingPos<kRingE> rE;
         RingPos<kRingL> rL;
         RingPos<kRingV> rV;
@@ -335,9 +335,9 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
           const uint32_t r_e = mbar_poll_addr(bEmptyE + rE.slot * 8, rE.par ^ 1);
           const uint32_t r_l = mbar_poll_addr(bEmptyL + rL.slot * 8, rL.par ^ 1);
           const uint32_t r_v = mbar_poll_addr(bEmptyV + rV.slot * 8, rV.par ^ 1);
-          if (nE < n_total && (force || (r_e & r_l))) {
+          if (nE < n_total && (r_e & r_l)) {
             const Tile t = itE.get();
-            bool ok = force || !deps || t.p == 0 || ctrE >= need_of(t);
+            bool ok = !deps || t.p == 0 || ctrE >= need_of(t);
             if (!ok) {
               ctrE = ld_acquire(counter_of(t));
               ok = ctrE >= need_of(t);
@@ -373,9 +373,9 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
               did = true;
             }
           }
-          if (nVt < n_total && (force || r_v)) {
+          if (nVt < n_total && r_v) {
             const Tile t = itV.get();
-            bool ok = force || !deps || t.p == 0 || ctrV >= need_of(t);
+            bool ok = !deps || t.p == 0 || ctrV >= need_of(t);
             if (!ok) {
               ctrV = ld_acquire(counter_of(t));
               ok = ctrV >= need_of(t);
@@ -400,16 +400,16 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
           }
           if (did) {
             idle = false;
-          } else if (!force) {
+          } else {
             if (!idle) {
               idle = true;
               t0 = clock64();
             } else if (bars->abort_flag) {
-              force = true;
+              break;   // stop issuing: what is in flight drains before the CTA leaves
             } else if (clock64() - t0 > P.wait_cycles) {
               report_timeout(P.status, 10);
               bars->abort_flag = 1;
-              force = true;
+              break;   // stop issuing: what is in flight drains before the CTA leaves
             }
             __nanosleep(32);
           }
@@ -429,7 +429,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
         int uc = 0;                                 // output units handed out so far
         TileIter it1(P, first_g, stride_g, kBlocks), it2(P, first_g, stride_g, kBlocks);
         long long t0 = 0;
-        bool force = false, idle = false;
+        bool idle = false;
         RingPos<kRingE> r1E, r2E;
         RingPos<kRingL> r1L, r2L;
         RingPos<kStagesS> r1S;
@@ -449,11 +449,11 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
           const uint32_t r_v = mbar_poll_addr(bFullV + rV.slot * 8, rV.par);
           const uint32_t r_l = mbar_poll_addr(bFullL + r1L.slot * 8, r1L.par);
           const uint32_t r_sf = mbar_poll_addr(bSFree + r1S.slot * 8, r1S.par ^ 1);
-          if (i2 < i1 && (force || (r_ready & r_ofA))) {
+          if (i2 < i1 && (r_ready & r_ofA)) {
             const Tile t = it2.get();
             const bool needV = needs_v(t);
             const int nu = units_of(t);
-            if (force || ((!needV || r_v) && (nu == 1 || r_ofB))) {
+            if ((!needV || r_v) && (nu == 1 || r_ofB)) {
               const int eL2 = r2L.slot, eV = rV.slot, eE2 = r2E.slot;
               const uint32_t sL = sL0 + eL2 * kSlot, sV = sV0 + eV * kSlot, sE = sE0 + eE2 * kSlot;
               const uint32_t tOA = tmem_o + 64 * uA, tOB = tmem_o + 64 * uB, tP = tmem_p + c * NP;
@@ -494,7 +494,7 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
               did = true;
             }
           }
-          if (i1 < n_total && (force || (r_l & r_sf))) {
+          if (i1 < n_total && (r_l & r_sf)) {
             const Tile t = it1.get();
             const int eE = r1E.slot, eL1 = r1L.slot, s1 = r1S.slot;
             tc_fence_after();
@@ -514,16 +514,16 @@ __global__ void __launch_bounds__(kThreads, 1) monarch_tmem(const __grid_constan
           }
           if (did) {
             idle = false;
-          } else if (!force) {
+          } else {
             if (!idle) {
               idle = true;
               t0 = clock64();
             } else if (bars->abort_flag) {
-              force = true;
+              break;   // stop issuing: what is in flight drains before the CTA leaves
             } else if (clock64() - t0 > P.wait_cycles) {
               report_timeout(P.status, 20);
               bars->abort_flag = 1;
-              force = true;
+              break;   // stop issuing: what is in flight drains before the CTA leaves
             }
             __nanosleep(20);
           }

@@ -103,9 +103,10 @@ __device__ __forceinline__ uint4 to_f16x8(uint4 v, const __nv_bfloat16*) {
   uint32_t* w = reinterpret_cast<uint32_t*>(&v);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const float lo = fminf(fmaxf(__uint_as_float(w[i] << 16), -65504.f), 65504.f);
-    const float hi = fminf(fmaxf(__uint_as_float(w[i] & 0xffff0000u), -65504.f), 65504.f);
-    w[i] = Mma<__half>::pack(lo, hi);
+    // a bf16 is the upper half of an fp32; the conversion saturates at +-65504
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;"
+        : "=r"(w[i])
+        : "f"(__uint_as_float(w[i] & 0xffff0000u)), "f"(__uint_as_float(w[i] << 16)));
   }
   return v;
 }

@@ -848,3 +848,44 @@ def test_fused_f32_kernel_is_the_default_for_short_fp32_sequences_and_serves_the
     assert binding.monarch_attn_last_launch_count() == 2
     with pytest.raises(binding.MonarchAttnError):
         binding.monarch_attn_fwd_ex(Q2, K2, V2, 32, 1, path=binding.MA_PATH_FUSED_F32)
+
+
+# ------------------------------------------------------------------ kernel split by in-block position
+@pytest.mark.parametrize("T,dtype,batch,heads,s", [
+    (1, "f16", 1, 1, 1.0), (2, "f16", 1, 3, 1.0), (2, "bf16", 2, 5, 1.5), (1, "bf16", 1, 7, 0.0),
+    (3, "f16", 1, 4, 0.5), (2, "bf16", 4, 37, 1.0),    # 148 heads: 592 CTAs, four waves
+])
+def test_position_split_kernel_matches_oracle(T, dtype, batch, heads, s):
+    """N = 1024 as 32 x 32 in one launch: four CTAs per head, eight in-block positions each."""
+    check(batch, heads, 1024, 64, 32, T, dtype, rank=16 if s else 0, s=s, seed=7 * T + heads,
+          path=binding.MA_PATH_FUSED_JSPLIT)
+    assert binding.monarch_attn_last_launch_count() == 1
+
+
+def test_position_split_kernel_is_the_default_for_its_shape_and_nothing_else():
+    Q, K, V = wl.make_qkv(1, 6, 1024, 64, "bf16", 16, 1.0, seed=11)
+    Qd, Kd, Vd = (binding.to_device(x, "bf16") for x in (Q, K, V))
+    a = binding.monarch_attn_fwd(Qd, Kd, Vd, 32, 2)
+    assert binding.monarch_attn_last_launch_count() == 1
+    e = binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 32, 2, path=binding.MA_PATH_FUSED_JSPLIT)
+    assert torch.equal(a, e)
+    ref = mo.monarch_attention(Q, K, V, 32, 2)
+    assert rel_err(a.float().cpu().numpy().astype(np.float64), ref) <= 1e-2
+    # every position's rows are written, by exactly the CTA that owns the position
+    Y0 = torch.full_like(Qd, float("nan"))
+    binding.monarch_attn_fwd_ex(Qd, Kd, Vd, 32, 2, path=binding.MA_PATH_FUSED_JSPLIT, Y=Y0)
+    assert torch.equal(Y0, a)
+    # three rounds go to the kernels with hi + lo states; fp32 and other shapes never come here
+    binding.monarch_attn_fwd(Qd, Kd, Vd, 32, 3)
+    assert binding.monarch_attn_last_launch_count() > 1
+    for bad in [dict(b=16), dict(b=64)]:
+        with pytest.raises(binding.MonarchAttnError):
+            binding.monarch_attn_fwd_ex(Qd, Kd, Vd, bad["b"], 2, path=binding.MA_PATH_FUSED_JSPLIT)
+    with pytest.raises(binding.MonarchAttnError):
+        binding.monarch_attn_fwd_ex(Qd.float(), Kd.float(), Vd.float(), 32, 2, path=binding.MA_PATH_FUSED_JSPLIT)
+    # the entry points with a mask, another layout or the row_lse output keep their own kernels
+    Y, lse = binding.monarch_attn_fwd_objective(Qd, Kd, Vd, 32, 2)
+    assert binding.monarch_attn_last_launch_count() >= 1 and bool(torch.isfinite(lse).all())
+    assert rel_err(Y.float().cpu().numpy().astype(np.float64), ref) <= 1e-2
+    with pytest.raises(binding.MonarchAttnError):
+        binding.monarch_attn_fwd_objective(Qd, Kd, Vd, 32, 2, path=binding.MA_PATH_FUSED_JSPLIT)
