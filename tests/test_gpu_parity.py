@@ -241,7 +241,8 @@ def test_extra_workloads_at_full_size(name):
 
 def test_general_fused_kernel_is_the_default_where_it_applies():
     """AUTO: 16-bit inputs with small blocks take the one-launch kernel, with or without padding
-    and in either layout; fp32 inputs and sequences too long for shared memory do not."""
+    and in either layout; fp32 inputs (which have a one-launch kernel of their own) and sequences too
+    long for shared memory do not."""
     Q, K, V = wl.make_qkv(2, 2, 384, 64, "f16", 8, 1.0, seed=3)
     Qd, Kd, Vd = (binding.to_device(x, "f16") for x in (Q, K, V))
     a = binding.monarch_attn_fwd(Qd, Kd, Vd, 24, 1)
@@ -258,7 +259,7 @@ def test_general_fused_kernel_is_the_default_where_it_applies():
     Q, K, V = wl.make_qkv(1, 2, 384, 64, "f32", 8, 1.0, seed=3)
     x = [binding.to_device(t_, "f32") for t_ in (Q, K, V)]
     binding.monarch_attn_fwd(*x, 24, 1)
-    assert binding.monarch_attn_last_launch_count() == 2           # generic: one launch per half-step
+    assert binding.monarch_attn_last_launch_count() == 1           # the one-launch kernel with fp32 states
     with pytest.raises(binding.MonarchAttnError) as e:
         binding.monarch_attn_fwd_ex(*x, 24, 1, path=binding.MA_PATH_FUSED_SMALL)
     assert e.value.code == 4
