@@ -66,8 +66,8 @@ typedef enum {
                               by in-block position (Eq. 7-10 never mix two positions j), each
                               keeping K and its own rows of Q and of the states in shared memory.
                               f16 arithmetic with plain f16 states: what AUTO takes for T <= 2 */
-  MA_PATH_FUSED_SMALL = 7, /* the same idea for any block shape: f16/bf16, m and b <= 32 (m need not
-                             equal b), d <= 64 a multiple of 8, N <= 580 for T = 1 and <= 440 for
+  MA_PATH_FUSED_SMALL = 7, /* the same idea for any block shape: f16/bf16, m <= 32 and b <= 64 (m need
+                             not equal b), d <= 64 a multiple of 8, N <= 580 for T = 1 and <= 440 for
                              T > 1 (the states of a head must fit shared memory); f16 arithmetic */
   MA_PATH_TILE_MMA = 8    /* warp-MMA kernels, one launch per half-step, f16 states in the workspace
                              (hi + lo pairs of f16 from T = 3 on): f16/bf16, m and b <= 128 (m need
@@ -188,7 +188,7 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
  *   - rows seq_len[e] .. ceil(seq_len[e] / b) * b - 1 of Y carry no meaning, later rows are zero;
  *     rows of Q, K, V in absent blocks are never read.
  * Q, K, V, Y: DEVICE pointers, [batch][heads][N][d], rules as monarch_attn_fwd_ex.  Runs on the
- * general fused kernel (f16/bf16, m and b <= 32, d <= 64, short N: one launch) where that
+ * general fused kernel (f16/bf16, m <= 32, b <= 64, d <= 64, short N: one launch) where that
  * applies, else on the generic kernels (any dtype, any N = m b); workspace: the larger of
  * monarch_attn_workspace_bytes() for MA_PATH_FUSED_SMALL and MA_PATH_GENERIC that is not 0.
  * Asynchronous on `stream`. */

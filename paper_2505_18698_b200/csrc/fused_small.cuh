@@ -1,4 +1,4 @@
-// Fused per-head kernel for short sequences of any block shape: N = m*b with m, b <= 32,
+// Fused per-head kernel for short sequences of any block shape: N = m*b with m <= 32, b <= 64,
 // d <= 64 (a multiple of 8), f16/bf16, optional key padding mask (App. C.3) and either layout.
 //
 // One CTA (8 warps) per (batch, head), one launch for all T rounds.  Q, K, V are read from HBM
@@ -75,9 +75,9 @@ inline size_t smem_bytes(int N, int T, int threads = kThreads) {
   return (size_t)(T == 1 ? 3 : 4) * N * kRowBytes + (((size_t)N * 4 + 15) & ~(size_t)15) + dump_bytes(threads) + 1024;
 }
 
-// BP, MP: b and m rounded up to 16 or 32.
+// BP: b rounded up to 16, 32, 48 or 64; MP: m rounded up to 16 or 32.
 template <typename TIn, int BP, int MP>
-__global__ void __launch_bounds__((BP == 16 || MP == 16) ? 2 * kThreads : kThreads, 1)
+__global__ void __launch_bounds__((BP <= 32 && (BP == 16 || MP == 16)) ? 2 * kThreads : kThreads, 1)
 monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
                     TIn* __restrict__ Y, int N, int d, int b, int m, int T_steps, float scale,
                     int n_valid, int H, float* __restrict__ lse, const int* __restrict__ seq_len,
@@ -529,7 +529,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
 }
 
 inline bool supported(int N, int d, int b, int m, int dtype, int T) {
-  return (dtype == 1 || dtype == 2) && d % 8 == 0 && d <= 64 && b <= 32 && m <= 32 &&
+  return (dtype == 1 || dtype == 2) && d % 8 == 0 && d <= 64 && b <= 64 && m <= 32 &&
          smem_bytes(N, T) <= (size_t)kMaxSmem;
 }
 
@@ -546,7 +546,7 @@ inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH
   // The 16 x 16 kernel is compiled for 128 registers: two CTAs of 8 warps per SM where shared memory
   // lets two fit, else one CTA of 16 warps (each warp then owns at most one tile per half-step).
   int threads = kThreads;
-  if ((BP == 16 || MP == 16) && 2 * (smem_bytes(N, T) + 1024) > (size_t)228 * 1024 && (m > 8 || b > 8) &&
+  if (BP <= 32 && (BP == 16 || MP == 16) && 2 * (smem_bytes(N, T) + 1024) > (size_t)228 * 1024 && (m > 8 || b > 8) &&
       smem_bytes(N, T, 2 * kThreads) <= (size_t)kMaxSmem)
     threads = 2 * kThreads;
   const size_t smem = smem_bytes(N, T, threads);
@@ -577,6 +577,8 @@ inline int launch_d(const void* Q, const void* K, const void* V, void* Y, int BH
                     int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st,
                     const int* seq_len, int heads) {
 #define MA_FS_ARGS Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st, seq_len, heads
+  if (b > 48) return m <= 16 ? launch_t<TIn, 64, 16>(MA_FS_ARGS) : launch_t<TIn, 64, 32>(MA_FS_ARGS);
+  if (b > 32) return m <= 16 ? launch_t<TIn, 48, 16>(MA_FS_ARGS) : launch_t<TIn, 48, 32>(MA_FS_ARGS);
   if (b <= 16 && m <= 16) return launch_t<TIn, 16, 16>(MA_FS_ARGS);
   if (b <= 16) return launch_t<TIn, 16, 32>(MA_FS_ARGS);
   if (m <= 16) return launch_t<TIn, 32, 16>(MA_FS_ARGS);

@@ -99,6 +99,10 @@ EXTRA_WORKLOADS = {
                    "BART sequence 8192 as 128 blocks of 64 (m != b), one round"),
     "S4": Workload("S4", 1, 8, 7680, 48, 128, 2, "f16", 8, 1.0, 8,
                    "graph transformer: 7600 nodes padded to 60 blocks of 128, d = 48, two rounds"),
+    "S5": Workload("S5", 8, 16, 256, 72, 16, 3, "f16", 8, 1.0, 9,
+                   "DiT: 256 image tokens as 16 blocks of 16, d = 72, three rounds"),
+    "S6": Workload("S6", 32, 12, 384, 64, 48, 1, "f16", 8, 1.0, 10,
+                   "RoBERTa sequence 384 as 8 blocks of 48, one round"),
 }
 
 

@@ -213,9 +213,12 @@ def test_a_fused_kernel_is_the_default_for_short_sequences_and_launches_once():
     (416, 13, 64, 2, "bf16"), (330, 11, 48, 2, "f16"),      # m = 32 / 30 with a short block, d = 48
     (320, 32, 64, 3, "f16"), (100, 10, 40, 3, "f16"),       # d = 40: a half 16-column step
     (60, 6, 8, 2, "f16"), (27, 3, 24, 4, "bf16"), (31, 31, 16, 2, "f16"), (29, 1, 32, 2, "f16"),
+    (384, 48, 64, 1, "f16"), (384, 48, 64, 2, "bf16"),      # blocks of 33 .. 64 rows: three or four
+    (384, 64, 64, 2, "f16"), (200, 40, 64, 2, "bf16"),      # 16-row tiles per block
+    (432, 36, 56, 2, "f16"), (128, 64, 64, 3, "bf16"), (441, 63, 64, 1, "f16"),
 ])
 def test_general_fused_kernel_matches_oracle(N, b, d, T, dtype):
-    """Any m, b <= 32 and d <= 64 in one launch per call, states in shared memory (Sec. 3)."""
+    """Any m <= 32, b <= 64 and d <= 64 in one launch per call, states in shared memory (Sec. 3)."""
     check(2, 3, N, d, b, T, dtype, rank=min(8, d), s=1.0, seed=N + 3 * T, path=binding.MA_PATH_FUSED_SMALL)
     assert binding.monarch_attn_last_launch_count() == 1
 
@@ -224,15 +227,15 @@ def test_general_fused_kernel_many_heads():
     check(151, 3, 210, 64, 14, 2, "f16", rank=8, s=1.0, seed=5, path=binding.MA_PATH_FUSED_SMALL)
 
 
-@pytest.mark.parametrize("name", ["S1", "S2", "S3", "S4"])
+@pytest.mark.parametrize("name", ["S1", "S2", "S3", "S4", "S5", "S6"])
 def test_extra_workloads_at_full_size(name):
-    """The extra workloads bench.py can time (fused kernel: S1, S2; tile kernels: S3, S4), at full
-    size, every head against the oracle."""
+    """The extra workloads bench.py can time (fused kernel: S1, S2, S6; tile kernels: S3, S4, S5), at
+    full size, every head against the oracle."""
     w = wl.EXTRA_WORKLOADS[name]
     Q, K, V = wl.make_workload_inputs(w)
     Qd, Kd, Vd = (binding.to_device(x, w.dtype) for x in (Q, K, V))
     Y = binding.monarch_attn_fwd(Qd, Kd, Vd, w.b, w.T).float().cpu().numpy().astype(np.float64)
-    assert binding.monarch_attn_last_launch_count() == (1 if name in ("S1", "S2") else 2 * w.T)
+    assert binding.monarch_attn_last_launch_count() == (1 if name in ("S1", "S2", "S6") else 2 * w.T)
     ref = mo.monarch_attention(Q, K, V, w.b, w.T)
     err = (np.linalg.norm((Y - ref).reshape(w.BH, -1), axis=1)
            / np.linalg.norm(ref.reshape(w.BH, -1), axis=1))
