@@ -186,9 +186,11 @@ def workload_config(w, world, strong=False):
 
 
 # ----------------------------------------------------------------------------- ours
-def time_config(w, steps, warmup, torch, binding, n_sets=3, dist=None, units=None):
+def time_config(w, steps, warmup, torch, binding, n_sets=3, dist=None, units=None, path=None):
     """Device-timed steps of workload w (or, with `units` = (lo, hi), of that slice of its
-    (batch, head) units: strong scaling).  Returns dict with ms_per_step etc."""
+    (batch, head) units: strong scaling).  `path`: None = the library's own choice through
+    monarch_attn_fwd; a path constant = that kernel through monarch_attn_fwd_ex with a workspace
+    allocated once.  Returns dict with ms_per_step etc."""
     sets = []
     for r in range(n_sets):
         seed = w.seed + 1000 * r + 17 * int(os.environ.get("RANK", "0"))
@@ -198,12 +200,25 @@ def time_config(w, steps, warmup, torch, binding, n_sets=3, dist=None, units=Non
             Q, K, V = wl.make_qkv(1, units[1] - units[0], w.N, w.d, w.dtype, w.rank, w.s, seed)
         Qd, Kd, Vd = (binding.to_device(x, w.dtype) for x in (Q, K, V))
         sets.append((Qd, Kd, Vd, torch.empty_like(Qd)))
-    binding.monarch_attn_fwd(sets[0][0], sets[0][1], sets[0][2], w.b, w.T, Y=sets[0][3])  # sizes ws
+    if path is None:
+        def call(s):
+            binding.monarch_attn_fwd(s[0], s[1], s[2], w.b, w.T, Y=s[3])
+        status_of = None
+    else:
+        q0 = sets[0][0]
+        need = binding.monarch_attn_workspace_bytes(q0.shape[0], q0.shape[1], w.N, w.d, w.b, w.T, q0.dtype, path)
+        if need == 0:
+            raise SystemExit(f"--path: that kernel does not take workload {w.name}")
+        ws = torch.zeros(need, dtype=torch.uint8, device=q0.device)
+        status_of = ws
+
+        def call(s):
+            binding.monarch_attn_fwd_ex(s[0], s[1], s[2], w.b, w.T, path=path, workspace=ws, Y=s[3])
+    call(sets[0])                                   # sizes the library's workspace
     torch.cuda.synchronize()
     launches = binding.monarch_attn_last_launch_count()
     for i in range(warmup):
-        s = sets[i % n_sets]
-        binding.monarch_attn_fwd(s[0], s[1], s[2], w.b, w.T, Y=s[3])
+        call(sets[i % n_sets])
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
@@ -211,15 +226,14 @@ def time_config(w, steps, warmup, torch, binding, n_sets=3, dist=None, units=Non
     evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
     evs[0].record()
     for i in range(steps):
-        s = sets[(warmup + i) % n_sets]
-        binding.monarch_attn_fwd(s[0], s[1], s[2], w.b, w.T, Y=s[3])
+        call(sets[(warmup + i) % n_sets])
         evs[i + 1].record()
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     total_ms = evs[0].elapsed_time(evs[-1])
     per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
-    assert binding.monarch_attn_device_status() == 0
+    assert binding.monarch_attn_device_status(status_of) == 0
     # Launch-bound sizes (a call shorter than the Python call loop can issue them): the same calls
     # captured in a CUDA graph and replayed, so that the number is the device's, not the host's.
     loop_ms = total_ms / steps
@@ -232,8 +246,7 @@ def time_config(w, steps, warmup, torch, binding, n_sets=3, dist=None, units=Non
                 graph = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(graph, stream=side):
                     for i in range(steps):
-                        s = sets[i % n_sets]
-                        binding.monarch_attn_fwd(s[0], s[1], s[2], w.b, w.T, Y=s[3])
+                        call(sets[i % n_sets])
             torch.cuda.synchronize()
             graph.replay()
             torch.cuda.synchronize()
@@ -253,10 +266,9 @@ def time_config(w, steps, warmup, torch, binding, n_sets=3, dist=None, units=Non
     # host time of one call with an idle stream (argument checks, cached tensor maps, launch)
     host = []
     for i in range(20):
-        s = sets[i % n_sets]
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        binding.monarch_attn_fwd(s[0], s[1], s[2], w.b, w.T, Y=s[3])
+        call(sets[i % n_sets])
         host.append((time.perf_counter() - t0) * 1e6)
     torch.cuda.synchronize()
     return {"total_ms": total_ms, "ms_per_step": total_ms / steps, "min_ms": min(per),
@@ -343,6 +355,11 @@ def main():
     ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
                     help="weak: every rank runs the whole configuration on its own batch; strong: the "
                          "configuration's (batch, head) units are split over the ranks")
+    ap.add_argument("--path", default="auto",
+                    choices=["auto", "generic", "tensor", "tensor_tmem", "tensor_basic", "fused_f32",
+                             "fused_jsplit", "fused_small", "tile_mma"],
+                    help="auto: the kernel the library picks (monarch_attn_fwd); else that kernel by name "
+                         "through monarch_attn_fwd_ex (for profiling one kernel against another)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the other configurations, SDPA context and the CPU baseline")
     args = ap.parse_args()
@@ -375,7 +392,8 @@ def main():
         raise SystemExit(f"--scaling strong: {w.name} has only {w.BH} units for {world} ranks")
     sampler = ClockSampler(local)
     sampler.start()
-    res = time_config(w, steps, warmup, torch, binding, dist=dist, units=units)
+    path = None if args.path == "auto" else getattr(binding, "MA_PATH_" + args.path.upper())
+    res = time_config(w, steps, warmup, torch, binding, dist=dist, units=units, path=path)
     clocks = sampler.stop()
     ms = D.max_over_ranks(res["total_ms"] / steps, device="cuda")
     e2e_ms, h2d, d2h = time_e2e(w, max(3, min(steps, 20)), 3, torch, binding, dist)
@@ -397,6 +415,8 @@ def main():
         "min_ms": res["min_ms"], "median_ms": res["median_ms"],
         "host_us_per_call": res["host_us_per_call"], "timing": res["timing"],
     }
+    if path is not None:
+        line["config"]["path"] = args.path
 
     if rank == 0 and not args.no_extras and world == 1:
         line["context"] = {"sdpa_dense_attention_ms": sdpa_ms(w, torch, res["sets"]),
