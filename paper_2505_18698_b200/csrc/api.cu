@@ -174,8 +174,9 @@ static int resolve_path(const Problem& p, int path, bool plain = true) {
     if (p.b <= 16 && p.m <= 16 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T))
       return MA_PATH_FUSED_SMALL;
     if (tp::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TENSOR;
-    // (blocks of more than 48 rows: the tile kernels' two launches are as fast or faster, measured)
-    if (p.b <= 48 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
+    // (blocks of more than 32 rows: the tile kernels' two launches are as fast or faster with inputs
+    // in HBM, measured; the fused kernel takes them when asked for by name, and for the mask entries)
+    if (p.b <= 32 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
     if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
     // fp32 inputs: short sequences in one launch with the states in shared memory
     if (p.dtype == MA_F32 && p.BH <= 65535 && ffused::supported(p.N, p.d, p.b, p.m)) return MA_PATH_FUSED_F32;
