@@ -75,8 +75,10 @@ inline size_t smem_bytes(int N, int T, int threads = kThreads) {
   return (size_t)(T == 1 ? 3 : 4) * N * kRowBytes + (((size_t)N * 4 + 15) & ~(size_t)15) + dump_bytes(threads) + 1024;
 }
 
-// BP: b rounded up to 16, 32, 48 or 64; MP: m rounded up to 16 or 32.
-template <typename TIn, int BP, int MP>
+// BP: b rounded up to 16, 32, 48 or 64; MP: m rounded up to 16 or 32.  EXACT: b = BP, m = MP, d = 64
+// and no mask, known at compile time: every clamp, mask and bounds predicate below folds away and
+// the index products become shifts (the instruction stream, not a pipe, bounds this kernel).
+template <typename TIn, int BP, int MP, bool EXACT = false>
 __global__ void __launch_bounds__((BP <= 32 && (BP == 16 || MP == 16)) ? 2 * kThreads : kThreads, 1)
 monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
                     TIn* __restrict__ Y, int N, int d, int b, int m, int T_steps, float scale,
@@ -91,8 +93,15 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   // m = ceil(length / b) blocks and the appendix's mask in the last of them.  Rows are addressed
   // by (block, position) with the block size b only, so running the smaller problem is a matter
   // of the block count; the rows of Y past it are zeroed, the rows of Q, K, V past it never read.
+  if (EXACT) {
+    b = BP;
+    m = MP;
+    N = BP * MP;
+    d = 64;
+    n_valid = 0x7fffffff;
+  }
   const int m_alloc = m;
-  if (seq_len != nullptr) {
+  if (!EXACT && seq_len != nullptr) {
     n_valid = min(max(seq_len[blockIdx.x / heads], 1), N);
     m = (n_valid + b - 1) / b;
   }
@@ -230,7 +239,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
 #pragma unroll
               for (int e = 0; e < 2; ++e) {
                 const int i = 8 * nt + 2 * t + e;
-                const bool valid = i < b && k * b + i < n_valid;
+                const bool valid = EXACT || (i < b && k * b + i < n_valid);
                 const float z = valid ? s[nt][2 * hh + e] * fl : -INFINITY;
                 s[nt][2 * hh + e] = z;
                 mx = fmaxf(mx, z);
@@ -538,11 +547,11 @@ int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, 
            const int* seq_len = nullptr, int heads = 1);
 
 #ifdef MA_TU_FUSED_SMALL
-template <typename TIn, int BP, int MP>
+template <typename TIn, int BP, int MP, bool EXACT = false>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
                     int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st,
                     const int* seq_len, int heads) {
-  auto kern = monarch_fused_small<TIn, BP, MP>;
+  auto kern = monarch_fused_small<TIn, BP, MP, EXACT>;
   // The 16 x 16 kernel is compiled for 128 registers: two CTAs of 8 warps per SM where shared memory
   // lets two fit, else one CTA of 16 warps (each warp then owns at most one tile per half-step).
   int threads = kThreads;
@@ -577,6 +586,12 @@ inline int launch_d(const void* Q, const void* K, const void* V, void* Y, int BH
                     int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st,
                     const int* seq_len, int heads) {
 #define MA_FS_ARGS Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st, seq_len, heads
+  if (d == 64 && n_valid >= N && seq_len == nullptr) {   // exact fits, no mask
+    if (b == 16 && m == 16) return launch_t<TIn, 16, 16, true>(MA_FS_ARGS);
+    if (b == 32 && m == 32) return launch_t<TIn, 32, 32, true>(MA_FS_ARGS);
+    if (b == 16 && m == 32) return launch_t<TIn, 16, 32, true>(MA_FS_ARGS);
+    if (b == 32 && m == 16) return launch_t<TIn, 32, 16, true>(MA_FS_ARGS);
+  }
   if (b > 48) return m <= 16 ? launch_t<TIn, 64, 16>(MA_FS_ARGS) : launch_t<TIn, 64, 32>(MA_FS_ARGS);
   if (b > 32) return m <= 16 ? launch_t<TIn, 48, 16>(MA_FS_ARGS) : launch_t<TIn, 48, 32>(MA_FS_ARGS);
   if (b <= 16 && m <= 16) return launch_t<TIn, 16, 16>(MA_FS_ARGS);
