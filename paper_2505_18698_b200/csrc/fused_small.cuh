@@ -58,28 +58,49 @@ __device__ __forceinline__ void stsm_x4(uint32_t saddr, uint32_t r0, uint32_t r1
                : "memory");
 }
 
+// Tile layouts.  KS = number of 16-column steps a row holds (4: d <= 64, 5: d <= 80, 8: d <= 128).
+// KS = 4: 128-byte rows, row k*b + i, 16-byte chunks XOR-swizzled with (i & 7) ^ (k & 7).
+// KS > 4: rows of 32 KS + 16 bytes and 16 more bytes after every block, no swizzle: eight rows of
+// a block are 16 bytes (mod 128) apart, and so are the rows (l, j) of eight consecutive blocks, so
+// fragment loads are conflict-free in both directions here too.
+template <int KS> __device__ __forceinline__ constexpr int row_bytes() { return KS == 4 ? 128 : 32 * KS + 16; }
+template <int KS> __host__ __device__ __forceinline__ int block_bytes(int b) {
+  return KS == 4 ? b * 128 : b * (32 * KS + 16) + 16;
+}
 // Byte offset of element (block k, position i, column col) in a tile.
-__device__ __forceinline__ uint32_t at(int k, int i, int b, int col) {
-  const int chunk = (col >> 3) ^ (i & 7) ^ (k & 7);
-  return (uint32_t)((k * b + i) * kRowBytes + (chunk << 4) + ((col & 7) << 1));
+template <int KS> __device__ __forceinline__ uint32_t at(int k, int i, int b, int col) {
+  if (KS == 4) {
+    const int chunk = (col >> 3) ^ (i & 7) ^ (k & 7);
+    return (uint32_t)((k * b + i) * kRowBytes + (chunk << 4) + ((col & 7) << 1));
+  }
+  return (uint32_t)(k * block_bytes<KS>(b) + i * row_bytes<KS>() + (col << 1));
 }
 
 // The same for the 16-column step `step` when the lane's chunk within the step is c (0 or 1):
-// rowx(k, i, b, c) ^ (step << 5), valid on top of any 128-byte aligned tile address -- one XOR per
-// fragment load instead of the whole index computation.
-__device__ __forceinline__ uint32_t rowx(int k, int i, int b, int c) {
-  return (uint32_t)((k * b + i) * kRowBytes + ((c ^ (i & 7) ^ (k & 7)) << 4));
+// stp(rowx(k, i, b, c), step), valid on top of any 128-byte aligned tile address -- one XOR (or
+// add) per fragment load instead of the whole index computation.
+template <int KS> __device__ __forceinline__ uint32_t rowx(int k, int i, int b, int c) {
+  if (KS == 4) return (uint32_t)((k * b + i) * kRowBytes + ((c ^ (i & 7) ^ (k & 7)) << 4));
+  return (uint32_t)(k * block_bytes<KS>(b) + i * row_bytes<KS>() + (c << 4));
+}
+template <int KS> __device__ __forceinline__ uint32_t stp(uint32_t addr, int step) {
+  return KS == 4 ? addr ^ (uint32_t)(step << 5) : addr + (uint32_t)(step << 5);
 }
 
-inline size_t smem_bytes(int N, int T, int threads = kThreads) {
-  return (size_t)(T == 1 ? 3 : 4) * N * kRowBytes + (((size_t)N * 4 + 15) & ~(size_t)15) + dump_bytes(threads) + 1024;
+inline size_t tile_bytes(int N, int b, int ks) {
+  const int m = (N + b - 1) / b;
+  return ks == 4 ? (size_t)N * kRowBytes : (size_t)m * ((size_t)b * (32 * ks + 16) + 16);
+}
+inline int ksteps_for(int d) { return d <= 64 ? 4 : (d <= 80 ? 5 : 8); }
+inline size_t smem_bytes(int N, int T, int threads = kThreads, int b = 16, int ks = 4) {
+  return (size_t)(T == 1 ? 3 : 4) * tile_bytes(N, b, ks) + (((size_t)N * 4 + 15) & ~(size_t)15) + dump_bytes(threads) + 1024;
 }
 
 // BP: b rounded up to 16, 32, 48 or 64; MP: m rounded up to 16 or 32.  EXACT: b = BP, m = MP, d = 64
 // and no mask, known at compile time: every clamp, mask and bounds predicate below folds away and
 // the index products become shifts (the instruction stream, not a pipe, bounds this kernel).
-template <typename TIn, int BP, int MP, bool EXACT = false>
-__global__ void __launch_bounds__((BP <= 32 && (BP == 16 || MP == 16)) ? 2 * kThreads : kThreads, 1)
+template <typename TIn, int BP, int MP, bool EXACT = false, int KS = 4>
+__global__ void __launch_bounds__((KS == 4 && BP <= 32 && (BP == 16 || MP == 16)) ? 2 * kThreads : kThreads, 1)
 monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
                     TIn* __restrict__ Y, int N, int d, int b, int m, int T_steps, float scale,
                     int n_valid, int H, float* __restrict__ lse, const int* __restrict__ seq_len,
@@ -106,7 +127,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
     m = (n_valid + b - 1) / b;
   }
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  const int tile = N * kRowBytes;
+  const int tile = KS == 4 ? N * kRowBytes : (N / b) * block_bytes<KS>(b);
   uint8_t* sQ = smem;
   // then K, then V (loaded when the last round starts) ...
   //                                                  ... alpha_L of the earlier rounds until then;
@@ -125,9 +146,11 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   const int nw = blockDim.x >> 5;    // 8 warps, or 16 where only one CTA fits an SM (16 x 16 blocks)
   const int g = lane >> 2, t = lane & 3;
   const int h_idx = blockIdx.x;
-  // Contractions over d always run over the 64 padded columns (zeros beyond d: the inputs are
+  // Contractions over d always run over the 16 KS padded columns (zeros beyond d: the inputs are
   // zero-filled on the way in and the states are products with them), so every loop unrolls.
-  constexpr int ksteps = 4;
+  constexpr int ksteps = KS;
+  constexpr int LPR = KS == 4 ? 8 : 16;      // lanes that share a row in the copy loops
+  constexpr int RPI = 32 / LPR;              // rows per iteration of a warp
 
   // Rows of this head in global memory.
   const size_t head_base = H == 0 ? (size_t)h_idx * N * d : ((size_t)(h_idx / H) * N * H + (h_idx % H)) * d;
@@ -138,23 +161,24 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   // starts on a block as soon as that group has landed: no CTA-wide wait before the first tile.
   // The raw 16-bit values are copied; bf16 is converted to f16 in place by the lane that copied it.
   auto load_block = [&](const TIn* __restrict__ src, int a, int k) {
-    const int ch = lane & 7;
-    for (int i = lane >> 3; i < b; i += 4) {
-      const uint32_t off = (uint32_t)(a * tile) + at(k, i, b, ch * 8);
+    const int ch = lane & (LPR - 1);
+    if (ch >= 2 * KS) return;
+    for (int i = lane / LPR; i < b; i += RPI) {
+      const uint32_t off = (uint32_t)(a * tile) + at<KS>(k, i, b, ch * 8);
       if (ch * 8 < d) {
         const TIn* gp = src + head_base + (size_t)(k * b + i) * row_stride + ch * 8;
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sQ_u + off), "l"(gp) : "memory");
       } else {
-        *reinterpret_cast<uint4*>(smem + off) = make_uint4(0u, 0u, 0u, 0u);   // columns d..63
+        *reinterpret_cast<uint4*>(smem + off) = make_uint4(0u, 0u, 0u, 0u);   // columns d .. 16 KS - 1
       }
     }
   };
   auto convert_block = [&](int a, int k) {
     if (!Mma<TIn>::is_f16) {
-      const int ch = lane & 7;
-      for (int i = lane >> 3; i < b; i += 4) {
+      const int ch = lane & (LPR - 1);
+      for (int i = lane / LPR; i < b; i += RPI) {
         if (ch * 8 >= d) continue;
-        uint4* p = reinterpret_cast<uint4*>(smem + (size_t)a * tile + at(k, i, b, ch * 8));
+        uint4* p = reinterpret_cast<uint4*>(smem + (size_t)a * tile + at<KS>(k, i, b, ch * 8));
         *p = warpmma::to_f16x8(*p, (const TIn*)nullptr);
       }
     }
@@ -212,19 +236,19 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
 #pragma unroll
             for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
           const uint32_t a_u =
-              sA_u + rowx(k, min(j0 + (lane & 7) + ((lane >> 3) & 1) * 8, b - 1), b, lane >> 4);
+              sA_u + rowx<KS>(k, min(j0 + (lane & 7) + ((lane >> 3) & 1) * 8, b - 1), b, lane >> 4);
           uint32_t b_u[BP / 16];
 #pragma unroll
           for (int cp = 0; cp < BP / 16; ++cp)
-            b_u[cp] = sK_u + rowx(k, min(16 * cp + (lane & 7) + (lane >> 4) * 8, b - 1), b, (lane >> 3) & 1);
+            b_u[cp] = sK_u + rowx<KS>(k, min(16 * cp + (lane & 7) + (lane >> 4) * 8, b - 1), b, (lane >> 3) & 1);
 #pragma unroll
           for (int ks = 0; ks < ksteps; ++ks) {
             uint32_t a[4];
-            ldsm_x4(a, a_u ^ (ks << 5));
+            ldsm_x4(a, stp<KS>(a_u, ks));
 #pragma unroll
             for (int cp = 0; cp < BP / 16; ++cp) {
               uint32_t bf[4];
-              ldsm_x4(bf, b_u[cp] ^ (ks << 5));
+              ldsm_x4(bf, stp<KS>(b_u[cp], ks));
               Mma<T>::run(s[2 * cp], a, bf);
               Mma<T>::run(s[2 * cp + 1], a, bf + 2);
             }
@@ -276,14 +300,14 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
         const uint32_t dstL_u = last ? sK_u : sV_u;     // alpha_L of earlier rounds shares V's buffer
         uint32_t v_off[BP / 16];    // rows (k, i) of K and V as the second product's B operand
 #pragma unroll
-        for (int kk = 0; kk < BP / 16; ++kk) v_off[kk] = rowx(k, min(16 * kk + (lane & 15), b - 1), b, lane >> 4);
+        for (int kk = 0; kk < BP / 16; ++kk) v_off[kk] = rowx<KS>(k, min(16 * kk + (lane & 15), b - 1), b, lane >> 4);
 #pragma unroll
         for (int np = 0; np < ksteps; ++np) {   // two 8-column tiles of v per transposing ldmatrix
           uint32_t bk[BP / 16][4], bv[BP / 16][4];
 #pragma unroll
           for (int kk = 0; kk < BP / 16; ++kk) {
-            ldsm_x4_trans(bk[kk], (sK_u + v_off[kk]) ^ (np << 5));
-            if (last) ldsm_x4_trans(bv[kk], (sV_u + v_off[kk]) ^ (np << 5));
+            ldsm_x4_trans(bk[kk], stp<KS>(sK_u + v_off[kk], np));
+            if (last) ldsm_x4_trans(bv[kk], stp<KS>(sV_u + v_off[kk], np));
           }
           __syncwarp();
 #pragma unroll
@@ -301,7 +325,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
               }
             }
             const int j = 16 * rt + st_row;
-            const uint32_t off = rowx(k, j, b, st_nt) ^ (np << 5);
+            const uint32_t off = stp<KS>(rowx<KS>(k, j, b, st_nt), np);
             const float i0 = inv_s[rt][0], i1 = inv_s[rt][1];
             stsm_x4(j < b ? dstL_u + off : dump_u, Mma<T>::pack(o[0][0] * i0, o[0][1] * i0),
                     Mma<T>::pack(o[0][2] * i1, o[0][3] * i1), Mma<T>::pack(o[1][0] * i0, o[1][1] * i0),
@@ -345,19 +369,19 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
 #pragma unroll
             for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
           const uint32_t a_u =
-              sQ_u + rowx(min(l0 + (lane & 7) + ((lane >> 3) & 1) * 8, m - 1), j, b, lane >> 4);
+              sQ_u + rowx<KS>(min(l0 + (lane & 7) + ((lane >> 3) & 1) * 8, m - 1), j, b, lane >> 4);
           uint32_t b_u[MP / 16];
 #pragma unroll
           for (int cp = 0; cp < MP / 16; ++cp)
-            b_u[cp] = sAL_u + rowx(min(16 * cp + (lane & 7) + (lane >> 4) * 8, m - 1), j, b, (lane >> 3) & 1);
+            b_u[cp] = sAL_u + rowx<KS>(min(16 * cp + (lane & 7) + (lane >> 4) * 8, m - 1), j, b, (lane >> 3) & 1);
 #pragma unroll
           for (int ks = 0; ks < ksteps; ++ks) {
             uint32_t a[4];
-            ldsm_x4(a, a_u ^ (ks << 5));
+            ldsm_x4(a, stp<KS>(a_u, ks));
 #pragma unroll
             for (int cp = 0; cp < MP / 16; ++cp) {
               uint32_t bf[4];
-              ldsm_x4(bf, b_u[cp] ^ (ks << 5));
+              ldsm_x4(bf, stp<KS>(b_u[cp], ks));
               Mma<T>::run(s[2 * cp], a, bf);
               Mma<T>::run(s[2 * cp + 1], a, bf + 2);
             }
@@ -405,11 +429,11 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             uint32_t y_u[MP / 16];
 #pragma unroll
             for (int kk = 0; kk < MP / 16; ++kk)
-              y_u[kk] = sV_u + rowx(min(16 * kk + (lane & 15), m - 1), j, b, lane >> 4);
+              y_u[kk] = sV_u + rowx<KS>(min(16 * kk + (lane & 15), m - 1), j, b, lane >> 4);
             // only this warp reads the rows (l, j) of Q, and for this row tile it has (they were the
             // A operand of the scores): Y takes their place, slab by slab
             const int l = l0 + st_row;
-            const uint32_t row_u = sQ_u + rowx(l, j, b, st_nt);
+            const uint32_t row_u = sQ_u + rowx<KS>(l, j, b, st_nt);
             __syncwarp();
 #pragma unroll
             for (int np = 0; np < ksteps; ++np) {
@@ -417,11 +441,11 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
 #pragma unroll
               for (int kk = 0; kk < MP / 16; ++kk) {
                 uint32_t bf[4];
-                ldsm_x4_trans(bf, y_u[kk] ^ (np << 5));
+                ldsm_x4_trans(bf, stp<KS>(y_u[kk], np));
                 Mma<T>::run(o[0], pa[kk], bf);
                 Mma<T>::run(o[1], pa[kk], bf + 2);
               }
-              stsm_x4(l < m ? row_u ^ (np << 5) : dump_u, Mma<T>::pack(o[0][0] * inv_s[0], o[0][1] * inv_s[0]),
+              stsm_x4(l < m ? stp<KS>(row_u, np) : dump_u, Mma<T>::pack(o[0][0] * inv_s[0], o[0][1] * inv_s[0]),
                       Mma<T>::pack(o[0][2] * inv_s[1], o[0][3] * inv_s[1]),
                       Mma<T>::pack(o[1][0] * inv_s[0], o[1][1] * inv_s[0]),
                       Mma<T>::pack(o[1][2] * inv_s[1], o[1][3] * inv_s[1]));
@@ -442,10 +466,10 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
         if (last) {
           // the m rows (l, j) of Y are complete: this warp copies them out, 16 bytes per lane
           // (rows of blocks that are absent from a shorter sequence's problem: zeros)
-          const int ch = lane & 7;
-          for (int l = lane >> 3; l < m_alloc; l += 4) {
+          const int ch = lane & (LPR - 1);
+          for (int l = lane / LPR; l < m_alloc; l += RPI) {
             if (ch * 8 >= d) continue;
-            const uint4 v = l < m ? *reinterpret_cast<const uint4*>(sQ + at(l, j, b, ch * 8))
+            const uint4 v = l < m ? *reinterpret_cast<const uint4*>(sQ + at<KS>(l, j, b, ch * 8))
                                   : make_uint4(0u, 0u, 0u, 0u);
             TIn* gp = Y + head_base + (size_t)(l * b + j) * row_stride + ch * 8;
             *reinterpret_cast<uint4*>(gp) = warpmma::from_f16x8(v, gp);
@@ -511,20 +535,20 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             uint32_t q_u[MP / 16];
 #pragma unroll
             for (int ls = 0; ls < MP / 16; ++ls)
-              q_u[ls] = sQ_u + rowx(min(16 * ls + (lane & 15), m - 1), j, b, lane >> 4);
+              q_u[ls] = sQ_u + rowx<KS>(min(16 * ls + (lane & 15), m - 1), j, b, lane >> 4);
             const int kr = 16 * kt + st_row;                   // alpha_R row (kr, j) this lane addresses
-            const uint32_t row_u = sAR_u + rowx(kr, j, b, st_nt);
+            const uint32_t row_u = sAR_u + rowx<KS>(kr, j, b, st_nt);
 #pragma unroll
             for (int np = 0; np < ksteps; ++np) {
               float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
               for (int ls = 0; ls < MP / 16; ++ls) {
                 uint32_t bf[4];   // B[kk = l][n = v] = Q(l,j)[v], read transposed; two 8-column tiles
-                ldsm_x4_trans(bf, q_u[ls] ^ (np << 5));
+                ldsm_x4_trans(bf, stp<KS>(q_u[ls], np));
                 Mma<T>::run(o[0], pa[ls], bf);
                 Mma<T>::run(o[1], pa[ls], bf + 2);
               }
-              stsm_x4(kr < m ? row_u ^ (np << 5) : dump_u,
+              stsm_x4(kr < m ? stp<KS>(row_u, np) : dump_u,
                       Mma<T>::pack(o[0][0] * ic[0], o[0][1] * ic[0]), Mma<T>::pack(o[0][2] * ic[1], o[0][3] * ic[1]),
                       Mma<T>::pack(o[1][0] * ic[0], o[1][1] * ic[0]), Mma<T>::pack(o[1][2] * ic[1], o[1][3] * ic[1]));
             }
@@ -538,8 +562,8 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
 }
 
 inline bool supported(int N, int d, int b, int m, int dtype, int T) {
-  return (dtype == 1 || dtype == 2) && d % 8 == 0 && d <= 64 && b <= 64 && m <= 32 &&
-         smem_bytes(N, T) <= (size_t)kMaxSmem;
+  return (dtype == 1 || dtype == 2) && d % 8 == 0 && d <= 128 && b <= (d <= 64 ? 64 : 32) && m <= 32 &&
+         smem_bytes(N, T, kThreads, b, ksteps_for(d)) <= (size_t)kMaxSmem;
 }
 
 int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
@@ -547,18 +571,18 @@ int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, 
            const int* seq_len = nullptr, int heads = 1);
 
 #ifdef MA_TU_FUSED_SMALL
-template <typename TIn, int BP, int MP, bool EXACT = false>
+template <typename TIn, int BP, int MP, bool EXACT = false, int KS = 4>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
                     int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st,
                     const int* seq_len, int heads) {
-  auto kern = monarch_fused_small<TIn, BP, MP, EXACT>;
+  auto kern = monarch_fused_small<TIn, BP, MP, EXACT, KS>;
   // The 16 x 16 kernel is compiled for 128 registers: two CTAs of 8 warps per SM where shared memory
   // lets two fit, else one CTA of 16 warps (each warp then owns at most one tile per half-step).
   int threads = kThreads;
-  if (BP <= 32 && (BP == 16 || MP == 16) && 2 * (smem_bytes(N, T) + 1024) > (size_t)228 * 1024 && (m > 8 || b > 8) &&
-      smem_bytes(N, T, 2 * kThreads) <= (size_t)kMaxSmem)
+  if (KS == 4 && BP <= 32 && (BP == 16 || MP == 16) && 2 * (smem_bytes(N, T) + 1024) > (size_t)228 * 1024 &&
+      (m > 8 || b > 8) && smem_bytes(N, T, 2 * kThreads) <= (size_t)kMaxSmem)
     threads = 2 * kThreads;
-  const size_t smem = smem_bytes(N, T, threads);
+  const size_t smem = smem_bytes(N, T, threads, b, KS);
   if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
     return 7;
@@ -591,6 +615,14 @@ inline int launch_d(const void* Q, const void* K, const void* V, void* Y, int BH
     if (b == 32 && m == 32) return launch_t<TIn, 32, 32, true>(MA_FS_ARGS);
     if (b == 16 && m == 32) return launch_t<TIn, 16, 32, true>(MA_FS_ARGS);
     if (b == 32 && m == 16) return launch_t<TIn, 32, 16, true>(MA_FS_ARGS);
+  }
+  if (d > 80) {          // rows of up to 128 columns
+    if (b <= 16) return m <= 16 ? launch_t<TIn, 16, 16, false, 8>(MA_FS_ARGS) : launch_t<TIn, 16, 32, false, 8>(MA_FS_ARGS);
+    return m <= 16 ? launch_t<TIn, 32, 16, false, 8>(MA_FS_ARGS) : launch_t<TIn, 32, 32, false, 8>(MA_FS_ARGS);
+  }
+  if (d > 64) {          // rows of up to 80 columns (d = 72)
+    if (b <= 16) return m <= 16 ? launch_t<TIn, 16, 16, false, 5>(MA_FS_ARGS) : launch_t<TIn, 16, 32, false, 5>(MA_FS_ARGS);
+    return m <= 16 ? launch_t<TIn, 32, 16, false, 5>(MA_FS_ARGS) : launch_t<TIn, 32, 32, false, 5>(MA_FS_ARGS);
   }
   if (b > 48) return m <= 16 ? launch_t<TIn, 64, 16>(MA_FS_ARGS) : launch_t<TIn, 64, 32>(MA_FS_ARGS);
   if (b > 32) return m <= 16 ? launch_t<TIn, 48, 16>(MA_FS_ARGS) : launch_t<TIn, 48, 32>(MA_FS_ARGS);

@@ -216,9 +216,13 @@ def test_a_fused_kernel_is_the_default_for_short_sequences_and_launches_once():
     (384, 48, 64, 1, "f16"), (384, 48, 64, 2, "bf16"),      # blocks of 33 .. 64 rows: three or four
     (384, 64, 64, 2, "f16"), (200, 40, 64, 2, "bf16"),      # 16-row tiles per block
     (432, 36, 56, 2, "f16"), (128, 64, 64, 3, "bf16"), (441, 63, 64, 1, "f16"),
+    (256, 16, 72, 3, "f16"), (256, 16, 72, 1, "bf16"),      # rows wider than 64 columns: d = 72 (80
+    (210, 14, 80, 2, "f16"), (240, 30, 72, 2, "bf16"),      # padded), then up to 128
+    (256, 16, 128, 1, "f16"), (192, 12, 96, 2, "bf16"), (128, 32, 104, 2, "f16"),
 ])
 def test_general_fused_kernel_matches_oracle(N, b, d, T, dtype):
-    """Any m <= 32, b <= 64 and d <= 64 in one launch per call, states in shared memory (Sec. 3)."""
+    """Any m <= 32, b <= 64 with d <= 64 or b <= 32 with d <= 128, in one launch per call, states
+    in shared memory (Sec. 3)."""
     check(2, 3, N, d, b, T, dtype, rank=min(8, d), s=1.0, seed=N + 3 * T, path=binding.MA_PATH_FUSED_SMALL)
     assert binding.monarch_attn_last_launch_count() == 1
 
