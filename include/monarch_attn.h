@@ -188,10 +188,10 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
  *   - rows seq_len[e] .. ceil(seq_len[e] / b) * b - 1 of Y carry no meaning, later rows are zero;
  *     rows of Q, K, V in absent blocks are never read.
  * Q, K, V, Y: DEVICE pointers, [batch][heads][N][d], rules as monarch_attn_fwd_ex.  Runs on the
- * general fused kernel (f16/bf16, m <= 32, b <= 64, d <= 64, short N: one launch) where that
- * applies, else on the generic kernels (any dtype, any N = m b); workspace: the larger of
- * monarch_attn_workspace_bytes() for MA_PATH_FUSED_SMALL and MA_PATH_GENERIC that is not 0.
- * Asynchronous on `stream`. */
+ * general fused kernel (f16/bf16, short N, up to two rounds: one launch) where that applies, else
+ * on the warp-MMA tile kernels (f16/bf16, m, b, d <= 128), else on the generic kernels (any dtype,
+ * any N = m b); workspace: the largest of monarch_attn_workspace_bytes() for MA_PATH_FUSED_SMALL,
+ * MA_PATH_TILE_MMA and MA_PATH_GENERIC.  Asynchronous on `stream`. */
 int monarch_attn_fwd_varlen(const void* Q, const void* K, const void* V, void* Y, int batch,
                             int heads, int N, int d, int b, int T, int dtype, float softmax_scale,
                             const int* seq_len, void* workspace, size_t workspace_bytes,

@@ -287,7 +287,7 @@ def monarch_attn_fwd_varlen(Q, K, V, b, T, seq_len, softmax_scale=None, workspac
         softmax_scale = 1.0 / math.sqrt(d)
     Y = _out_like(Y, Q)
     workspace = _workspace_for(lib, workspace, Q, batch, heads, N, d, b, T, code,
-                               (MA_PATH_GENERIC, MA_PATH_FUSED_SMALL))
+                               (MA_PATH_GENERIC, MA_PATH_FUSED_SMALL, MA_PATH_TILE_MMA))
     with _on_device_of(Q):
         _check(lib.monarch_attn_fwd_varlen(Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(),
                                            batch, heads, N, d, b, T, code, float(softmax_scale),

@@ -290,7 +290,7 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
     return rc;
   }
   if (resolved == MA_PATH_TILE_MMA) {
-    tile::Args a{Q, K, V, Y, p.lse, p.BH, p.N, p.d, p.b, p.m, p.T, p.n_valid, p.H, scale};
+    tile::Args a{Q, K, V, Y, p.lse, p.BH, p.N, p.d, p.b, p.m, p.T, p.n_valid, p.H, scale, p.seq_len, p.heads};
     int n = 0;
     int rc = tile::launch(a, p.dtype, ws, st, &n);
     if (rc == MA_OK) g_last_launches = n;
@@ -386,10 +386,12 @@ int monarch_attn_fwd_varlen(const void* Q, const void* K, const void* V, void* Y
   if (!seq_len) return MA_ERR_NULL;
   if (((uintptr_t)seq_len & 3) != 0) return MA_ERR_ALIGN;
   if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
-  // short 16-bit sequences with up to two rounds: the fused per-head kernel (one launch); else the
-  // generic kernels (fp32 states: also what three or more rounds on peaky logits need)
+  // short 16-bit sequences with up to two rounds: the fused per-head kernel (one launch); other
+  // 16-bit shapes: the warp-MMA tile kernels (hi + lo states from the third round on); else the
+  // generic kernels
   int r = -1;
   if (p.T <= 2 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) r = MA_PATH_FUSED_SMALL;
+  else if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) r = MA_PATH_TILE_MMA;
   else if (generic_supported(p)) r = MA_PATH_GENERIC;
   if (r < 0) return MA_ERR_UNSUPPORTED;
   p.seq_len = seq_len;

@@ -153,11 +153,18 @@ r_tile_kernel(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* _
               const __half* __restrict__ aR, __half* __restrict__ aL, __half* __restrict__ y,
               const __half* __restrict__ aR_lo, __half* __restrict__ aL_lo,
               float* __restrict__ cL, int N, int d, int b, float scale, int n_valid, int H, int first,
-              int last) {
+              int last, const int* __restrict__ seq_len, int heads) {
   extern __shared__ __align__(128) uint8_t smem[];
   constexpr int kPitch = pitch_of(DT);
   grid_dependency_sync();
   const int k = blockIdx.x, h = blockIdx.y;
+  // Batched sequences of different lengths (App. C.3): a key block that lies wholly in this
+  // sequence's padding is absent from its problem (the L half-step never reads its rows of the
+  // states); the last block that is present gets the appendix's mask.
+  if (seq_len != nullptr) {
+    n_valid = min(max(seq_len[h / heads], 1), N);
+    if (k * b >= n_valid) return;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int rb = round16(b);
   uint8_t* sA = smem;
@@ -347,11 +354,15 @@ __global__ void __launch_bounds__(256)
 l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const float* __restrict__ cL,
               const __half* __restrict__ y, __half* __restrict__ aR, const __half* __restrict__ aL_lo,
               __half* __restrict__ aR_lo, TIn* __restrict__ Y, float* __restrict__ lse, int N, int d, int b,
-              int m, float scale, int H, int last) {
+              int m, float scale, int H, int last, const int* __restrict__ seq_len, int heads) {
   extern __shared__ __align__(128) uint8_t smem[];
   constexpr int kPitch = pitch_of(DT), kPPitch = CM * 2 + 16;
   grid_dependency_sync();
   const int j = blockIdx.x, h = blockIdx.y;
+  // Batched sequences of different lengths (App. C.3): this sequence's problem has the blocks
+  // 0 .. ceil(length / b) - 1 only; rows of Y in blocks past them are written as zeros.
+  const int m_alloc = m;
+  if (seq_len != nullptr) m = (min(max(seq_len[h / heads], 1), N) + b - 1) / b;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int rm = round16(m);
   uint8_t* sQ = smem;
@@ -445,6 +456,14 @@ l_tile_kernel(const TIn* __restrict__ Q, const __half* __restrict__ aL, const fl
   }
 
   if (last) {
+    if (m < m_alloc) {
+      const HeadRows hz = head_rows(h, N, d, H);
+      const int cpr = d / 8;                       // 16-byte chunks per row
+      for (int idx = threadIdx.x; idx < (m_alloc - m) * cpr; idx += blockDim.x) {
+        const int l = m + idx / cpr, ch = idx - (idx / cpr) * cpr;
+        *reinterpret_cast<uint4*>(Y + hz.base + ((size_t)l * b + j) * hz.stride + ch * 8) = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
     if (!active) return;
     // Y(l,j) = sum_k L[l,k] y(k,j): A = weights rows l, B = y rows (k,j) read transposed
     uint32_t pa[CM / 16][4];
@@ -651,6 +670,8 @@ struct Args {
   float* lse;
   int BH, N, d, b, m, T, n_valid, H;
   float scale;
+  const int* seq_len = nullptr;   // optional DEVICE array [BH / heads]: valid length of every sequence
+  int heads = 1;
 };
 
 int launch(const Args& a, int dtype, void* ws, cudaStream_t st, int* launches);
@@ -665,7 +686,7 @@ inline int launch_r(const Args& a, const Ws& w, bool first, bool last, cudaStrea
   cudaLaunchConfig_t cfg = serialised_config(dim3(a.m, a.BH), 32 * ((a.b + 15) / 16), smem, st);
   return cudaLaunchKernelEx(&cfg, kern, (const TIn*)a.Q, (const TIn*)a.K, (const TIn*)a.V, (const __half*)w.aR,
                             w.aL, w.y, (const __half*)w.aR_lo, w.aL_lo, w.cL, a.N, a.d, a.b, a.scale, a.n_valid,
-                            a.H, first ? 1 : 0, last ? 1 : 0) == cudaSuccess
+                            a.H, first ? 1 : 0, last ? 1 : 0, a.seq_len, a.heads) == cudaSuccess
              ? 0
              : 7;
 }
@@ -678,8 +699,8 @@ inline int launch_l(const Args& a, const Ws& w, bool last, cudaStream_t st) {
   cudaLaunchConfig_t cfg = serialised_config(dim3(a.b, a.BH), 32 * ((a.m + 15) / 16), smem, st);
   return cudaLaunchKernelEx(&cfg, kern, (const TIn*)a.Q, (const __half*)w.aL, (const float*)w.cL,
                             (const __half*)w.y, w.aR, (const __half*)w.aL_lo, w.aR_lo, (TIn*)a.Y,
-                            last ? a.lse : (float*)nullptr, a.N, a.d, a.b, a.m, a.scale, a.H, last ? 1 : 0) ==
-                 cudaSuccess
+                            last ? a.lse : (float*)nullptr, a.N, a.d, a.b, a.m, a.scale, a.H, last ? 1 : 0, a.seq_len,
+                            a.heads) == cudaSuccess
              ? 0
              : 7;
 }

@@ -683,14 +683,18 @@ def test_results_are_bit_identical_from_call_to_call(name):
 
 
 # ------------------------------------------------------------------ sequences of different lengths
-@pytest.mark.parametrize("N,b,d,T,dtype,lens,launches", [
-    (24, 4, 8, 2, "f32", [24, 17, 9, 3, 12], 4),            # generic kernels, tiny
-    (210, 14, 64, 2, "f16", [197, 210, 120, 29, 14, 1], 1),  # fused per-head kernel: ViT-like batch
-    (384, 24, 64, 1, "bf16", [384, 300, 100, 23], 1),       # fused kernel, m != b
-    (256, 16, 64, 3, "f16", [256, 250, 130, 40], 6),        # three rounds: generic kernels
-    (1024, 32, 64, 2, "bf16", [1024, 700, 333, 64, 31], 4),  # longer than the fused kernel takes
+@pytest.mark.parametrize("N,b,d,T,dtype,lens,launches,kernel", [
+    (24, 4, 8, 2, "f32", [24, 17, 9, 3, 12], 4, "GENERIC"),              # generic kernels, tiny
+    (210, 14, 64, 2, "f16", [197, 210, 120, 29, 14, 1], 1, "FUSED_SMALL"),  # ViT-like batch
+    (384, 24, 64, 1, "bf16", [384, 300, 100, 23], 1, "FUSED_SMALL"),     # fused kernel, m != b
+    (256, 16, 72, 2, "f16", [256, 131, 16], 1, "FUSED_SMALL"),           # fused kernel, wide rows
+    (256, 16, 64, 3, "f16", [256, 250, 130, 40], 6, "TILE_MMA"),         # three rounds: hi + lo states
+    (1024, 32, 64, 2, "bf16", [1024, 700, 333, 64, 31], 4, "TILE_MMA"),  # longer than the fused kernel takes
+    (768, 96, 48, 1, "f16", [768, 500, 97, 96, 700], 2, "TILE_MMA"),     # wide blocks, m != b, d = 48
+    (2048, 32, 64, 2, "f16", [2048, 1030, 33], 4, "TILE_MMA"),           # m = 64 blocks, most of them absent
+    (640, 160, 32, 1, "bf16", [640, 161, 480], 2, "GENERIC"),            # blocks wider than any tensor-core path
 ])
-def test_batched_sequences_of_different_lengths_match_the_oracle(N, b, d, T, dtype, lens, launches):
+def test_batched_sequences_of_different_lengths_match_the_oracle(N, b, d, T, dtype, lens, launches, kernel):
     """App. C.3, batches padded to a maximum length: one length per batch entry, including lengths
     more than a block short of N (key blocks lying wholly in the padding).  Valid rows must match
     the oracle's reading (each sequence's own problem); rows past a sequence's own padded length
@@ -724,7 +728,7 @@ def test_batched_sequences_of_different_lengths_match_the_oracle(N, b, d, T, dty
     full = torch.full((batch,), N, dtype=torch.int32, device="cuda")
     Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))
     a = binding.monarch_attn_fwd_varlen(Qd, Kd, Vd, b, T, full)
-    same_path = binding.MA_PATH_FUSED_SMALL if launches == 1 else binding.MA_PATH_GENERIC
+    same_path = getattr(binding, "MA_PATH_" + kernel)
     assert torch.equal(a, binding.monarch_attn_fwd_ex(Qd, Kd, Vd, b, T, path=same_path))
 
 
