@@ -61,7 +61,7 @@ typedef enum {
                             positions of one head (the recursion is independent across them), so a
                             single small head is spread over up to b CTAs.  What AUTO takes for
                             fp32 inputs of that size */
-  MA_PATH_FUSED_JSPLIT = 6, /* N = 1024 as m = b = 32 (d = 64, f16/bf16, standard layout, no mask, no
+  MA_PATH_FUSED_JSPLIT = 6, /* N = 1024 as m = b = 32 (d = 64, f16/bf16, either layout, no mask, no
                               row_lse): all T rounds in one launch; a head is split over four CTAs
                               by in-block position (Eq. 7-10 never mix two positions j), each
                               keeping K and its own rows of Q and of the states in shared memory.

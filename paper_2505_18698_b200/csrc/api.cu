@@ -159,8 +159,8 @@ static int launch_generic(const Problem& p, const void* Q, const void* K, const 
 }
 
 // ------------------------------------------------------------------ path selection
-// `plain`: the call has the standard layout, no mask and no row_lse output (the kernel split by
-// in-block position serves nothing else).
+// `plain`: the call has no mask and no row_lse output (the kernel split by in-block position
+// serves nothing else; the entry point for the other layout selects it itself).
 static int resolve_path(const Problem& p, int path, bool plain = true) {
   if (path == MA_PATH_AUTO) {
     // From the third round on, plain 16-bit states are too coarse on peaky logits (they are fed
@@ -285,7 +285,7 @@ static int fwd_ex(const void* Q, const void* K, const void* V, void* Y, const Pr
     return rc;
   }
   if (resolved == MA_PATH_FUSED_JSPLIT) {
-    int rc = jsplit::launch(Q, K, V, Y, p.BH, p.T, p.dtype, scale, (int*)ws, st);
+    int rc = jsplit::launch(Q, K, V, Y, p.BH, p.T, p.dtype, scale, (int*)ws, st, p.H);
     if (rc == MA_OK) g_last_launches = 1;
     return rc;
   }
@@ -425,7 +425,14 @@ int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, 
   rc = check_ptrs(Q, K, V, Y, p);
   if (rc != MA_OK) return rc;
   if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return MA_ERR_SHAPE;
-  const int r = resolve_tensor_or_generic(p, path, true);
+  // (the kernel split by in-block position takes this layout too: a head is a column offset of
+  // its tensor maps)
+  int r;
+  if (((path == MA_PATH_AUTO && p.T <= 2) || path == MA_PATH_FUSED_JSPLIT) &&
+      jsplit::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH))
+    r = MA_PATH_FUSED_JSPLIT;
+  else
+    r = resolve_tensor_or_generic(p, path, true);
   if (r < 0) return MA_ERR_UNSUPPORTED;
   p.H = heads;
   return fwd_ex(Q, K, V, Y, p, softmax_scale, r, workspace, workspace_bytes, (cudaStream_t)stream);

@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 monarch_jsplit32(const __grid_constant__ CUtensorMap tmQ,    // Q as [BH*N rows][64], box of 8 rows
                  const __grid_constant__ CUtensorMap tmK,    // K, box of 32 rows
                  const __grid_constant__ CUtensorMap tmV,    // V, box of 32 rows
-                 TIn* __restrict__ Y, int T_steps, float scale, int* status) {
+                 TIn* __restrict__ Y, int T_steps, float scale, int* status, int H) {
   typedef __half T;
   extern __shared__ uint8_t smem_raw[];
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -114,7 +114,12 @@ monarch_jsplit32(const __grid_constant__ CUtensorMap tmQ,    // Q as [BH*N rows]
   uint64_t* vbar = kbar + kM;                                     // block k: V(k, .) has landed
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int c4 = blockIdx.x;                    // which 8 of the 32 positions
-  const int row0 = blockIdx.y * kN;             // the head's first row
+  // H = 0: tensors [batch][heads][N][64], the maps see [BH * N rows][64 columns]; H = heads: tensors
+  // [batch][N][heads][64], the maps see [batch * N rows][heads * 64 columns] and a head is a column
+  // offset
+  const int hb = H ? (int)blockIdx.y / H : (int)blockIdx.y;   // which sequence of rows
+  const int x0 = H ? ((int)blockIdx.y - hb * H) * kD : 0;     // first column of the head
+  const int row0 = hb * kN;                                   // the head's first row
   const float fl = scale * kLog2e;
   const int kk[2] = {warp, warp + kWarps};      // the key blocks this warp owns in the R half-steps
 #ifdef MA_JSPLIT_TRACE
@@ -136,8 +141,8 @@ monarch_jsplit32(const __grid_constant__ CUtensorMap tmQ,    // Q as [BH*N rows]
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       mbar_expect_tx(&kbar[kk[u]], kBlkK + kPJ * 128);
-      tma_load_2d(smem + rk(kk[u], 0), &tmK, &kbar[kk[u]], 0, row0 + kk[u] * kB);
-      tma_load_2d(smem + rq(kk[u], 0), &tmQ, &kbar[kk[u]], 0, row0 + kk[u] * kB + c4 * kPJ);
+      tma_load_2d(smem + rk(kk[u], 0), &tmK, &kbar[kk[u]], x0, row0 + kk[u] * kB);
+      tma_load_2d(smem + rq(kk[u], 0), &tmQ, &kbar[kk[u]], x0, row0 + kk[u] * kB + c4 * kPJ);
     }
   }
   // bf16 -> f16 of a fragment in registers (a no-op for f16 inputs)
@@ -266,7 +271,7 @@ monarch_jsplit32(const __grid_constant__ CUtensorMap tmQ,    // Q as [BH*N rows]
 #pragma unroll
             for (int u = U0; u < U1; ++u) {
               mbar_expect_tx(&vbar[kk[u]], kBlkK);
-              tma_load_2d(smem + rk(kk[u], 0), &tmV, &vbar[kk[u]], 0, row0 + kk[u] * kB);
+              tma_load_2d(smem + rk(kk[u], 0), &tmV, &vbar[kk[u]], x0, row0 + kk[u] * kB);
             }
           }
         }
@@ -401,7 +406,7 @@ monarch_jsplit32(const __grid_constant__ CUtensorMap tmQ,    // Q as [BH*N rows]
         for (int r = 0; r < 4; ++r) {
           const int l = 16 * lt + (lane >> 3) + 4 * r;
           const uint4 v = *reinterpret_cast<const uint4*>(smem + swz(rq(l, jj), lane & 7));
-          TIn* gp = Y + ((size_t)row0 + l * kB + c4 * kPJ + jj) * kD + (lane & 7) * 8;
+          TIn* gp = Y + ((size_t)row0 + l * kB + c4 * kPJ + jj) * (size_t)(H ? H * kD : kD) + x0 + (lane & 7) * 8;
           *reinterpret_cast<uint4*>(gp) = warpmma::from_f16x8(v, gp);
         }
       } else {
@@ -488,19 +493,21 @@ inline bool supported(int N, int d, int b, int m, int dtype, int BH) {
 
 // `status`: device word that a bounded wait which ran out sets (never cleared by the kernel).
 int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int T, int dtype, float scale,
-           int* status, cudaStream_t st);
+           int* status, cudaStream_t st, int H = 0);
 
 #ifdef MA_TU_FUSED_JSPLIT
 struct Maps {
   const void *q = nullptr, *k = nullptr, *v = nullptr;
-  int BH = 0, dtype = 0, dev = -1;
+  int BH = 0, dtype = 0, dev = -1, H = 0;
   CUtensorMap tmQ, tmK, tmV;
 };
-inline bool make_map(CUtensorMap* tm, int dtype, const void* base, uint64_t rows, uint32_t box_rows) {
+inline bool make_map(CUtensorMap* tm, int dtype, const void* base, uint64_t rows, uint32_t box_rows, int H) {
   tensor::EncodeTiledFn fn = tensor::encode_fn();
   if (!fn) return false;
-  cuuint64_t dims[2] = {kD, rows};
-  cuuint64_t strides[1] = {kD * 2};
+  const uint64_t cols = H ? (uint64_t)H * kD : kD;
+  if (H) rows /= H;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
   cuuint32_t box[2] = {kD, box_rows};
   cuuint32_t es[2] = {1, 1};
   return fn(tm, dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
@@ -511,7 +518,7 @@ inline bool make_map(CUtensorMap* tm, int dtype, const void* base, uint64_t rows
 
 template <typename TIn>
 inline int launch_t(const Maps& mp, void* Y, int BH, int T, float scale, int* status, cudaStream_t st,
-                    int dev) {
+                    int dev, int H) {
   auto kern = monarch_jsplit32<TIn>;
   static bool prepared[64] = {};
   if (!prepared[dev]) {
@@ -529,11 +536,11 @@ inline int launch_t(const Maps& mp, void* Y, int BH, int T, float scale, int* st
   cfg.stream = st;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, mp.tmQ, mp.tmK, mp.tmV, (TIn*)Y, T, scale, status) == cudaSuccess ? 0 : 7;
+  return cudaLaunchKernelEx(&cfg, kern, mp.tmQ, mp.tmK, mp.tmV, (TIn*)Y, T, scale, status, H) == cudaSuccess ? 0 : 7;
 }
 
 int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int T, int dtype, float scale,
-           int* status, cudaStream_t st) {
+           int* status, cudaStream_t st, int H) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 7;
   // the tensor maps of the last few (Q, K, V) triples are kept: encoding three maps costs more host
@@ -543,21 +550,21 @@ int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int T, 
   const Maps* mp = nullptr;
   for (int i = 0; i < 4; ++i)
     if (cache[i].q == Q && cache[i].k == K && cache[i].v == V && cache[i].BH == BH && cache[i].dtype == dtype &&
-        cache[i].dev == dev)
+        cache[i].dev == dev && cache[i].H == H)
       mp = &cache[i];
   if (!mp) {
     Maps& m = cache[next];
     next = (next + 1) % 4;
     m.dev = -1;
     const uint64_t rows = (uint64_t)BH * kN;
-    if (!make_map(&m.tmQ, dtype, Q, rows, kPJ) || !make_map(&m.tmK, dtype, K, rows, kB) ||
-        !make_map(&m.tmV, dtype, V, rows, kB))
+    if (!make_map(&m.tmQ, dtype, Q, rows, kPJ, H) || !make_map(&m.tmK, dtype, K, rows, kB, H) ||
+        !make_map(&m.tmV, dtype, V, rows, kB, H))
       return 7;
-    m.q = Q; m.k = K; m.v = V; m.BH = BH; m.dtype = dtype; m.dev = dev;
+    m.q = Q; m.k = K; m.v = V; m.BH = BH; m.dtype = dtype; m.dev = dev; m.H = H;
     mp = &m;
   }
-  if (dtype == 1) return launch_t<__half>(*mp, Y, BH, T, scale, status, st, dev);
-  return launch_t<__nv_bfloat16>(*mp, Y, BH, T, scale, status, st, dev);
+  if (dtype == 1) return launch_t<__half>(*mp, Y, BH, T, scale, status, st, dev, H);
+  return launch_t<__nv_bfloat16>(*mp, Y, BH, T, scale, status, st, dev, H);
 }
 #endif  // MA_TU_FUSED_JSPLIT
 

@@ -895,7 +895,13 @@ def test_position_split_kernel_is_the_default_for_its_shape_and_nothing_else():
             binding.monarch_attn_fwd_ex(Qd, Kd, Vd, bad["b"], 2, path=binding.MA_PATH_FUSED_JSPLIT)
     with pytest.raises(binding.MonarchAttnError):
         binding.monarch_attn_fwd_ex(Qd.float(), Kd.float(), Vd.float(), 32, 2, path=binding.MA_PATH_FUSED_JSPLIT)
-    # the entry points with a mask, another layout or the row_lse output keep their own kernels
+    # the other layout: a head is a column offset of the tensor maps
+    Qs, Ks, Vs = (x.transpose(1, 2).contiguous() for x in (Qd, Kd, Vd))
+    c = binding.monarch_attn_fwd_bshd(Qs, Ks, Vs, 32, 2)
+    assert binding.monarch_attn_last_launch_count() == 1 and torch.equal(c.transpose(1, 2), a)
+    c1 = binding.monarch_attn_fwd_bshd(Qs, Ks, Vs, 32, 1, path=binding.MA_PATH_FUSED_JSPLIT)
+    assert torch.equal(c1.transpose(1, 2), binding.monarch_attn_fwd(Qd, Kd, Vd, 32, 1))
+    # the entry points with a mask or the row_lse output keep their own kernels
     Y, lse = binding.monarch_attn_fwd_objective(Qd, Kd, Vd, 32, 2)
     assert binding.monarch_attn_last_launch_count() >= 1 and bool(torch.isfinite(lse).all())
     assert rel_err(Y.float().cpu().numpy().astype(np.float64), ref) <= 1e-2
