@@ -144,7 +144,8 @@ int monarch_attn_fwd_objective(const void* Q, const void* K, const void* V, void
  * addressing changes.  Q, K, V, Y: DEVICE pointers to contiguous [batch][N][heads][d] arrays of
  * `dtype`, 16-byte aligned, Y not overlapping an input.  `path`: MA_PATH_AUTO, MA_PATH_TENSOR (the
  * second-generation kernel: the head becomes a column offset in the TMA tensor maps),
- * MA_PATH_FUSED_SMALL, MA_PATH_TILE_MMA or MA_PATH_GENERIC; other paths give MA_ERR_UNSUPPORTED.  Workspace as for monarch_attn_fwd_ex with
+ * MA_PATH_FUSED_JSPLIT (likewise), MA_PATH_FUSED_SMALL, MA_PATH_FUSED_F32, MA_PATH_TILE_MMA or
+ * MA_PATH_GENERIC; other paths give MA_ERR_UNSUPPORTED.  Workspace as for monarch_attn_fwd_ex with
  * the same path (monarch_attn_workspace_bytes does not depend on the layout).  Everything else as
  * monarch_attn_fwd_ex.  Asynchronous on `stream`. */
 int monarch_attn_fwd_bshd(const void* Q, const void* K, const void* V, void* Y, int batch, int N,
