@@ -108,3 +108,17 @@ def test_binding_refuses_cpu_tensors(lib):
     x = torch.zeros(1, 1, 16, 4)
     with pytest.raises(binding.MonarchAttnError):
         binding.monarch_attn_fwd(x, x, x, b=4, T=1)
+
+
+def test_binding_rejects_an_output_tensor_that_does_not_match_the_input():
+    """The kernels write Q.numel() elements of Q's dtype through Y's pointer: a smaller, differently
+    typed or strided Y must be refused on the host (no GPU needed to check the rule)."""
+    import torch
+    Q = torch.zeros(2, 3, 16, 8)
+    assert binding._out_like(None, Q).shape == Q.shape
+    ok = torch.empty_like(Q)
+    assert binding._out_like(ok, Q) is ok
+    for bad in (torch.zeros(2, 3, 16, 4), torch.zeros(2, 3, 16, 8, dtype=torch.float16),
+                torch.zeros(2, 3, 8, 16).transpose(2, 3), "not a tensor"):
+        with pytest.raises(ValueError):
+            binding._out_like(bad, Q)
