@@ -907,3 +907,63 @@ def test_position_split_kernel_is_the_default_for_its_shape_and_nothing_else():
     assert rel_err(Y.float().cpu().numpy().astype(np.float64), ref) <= 1e-2
     with pytest.raises(binding.MonarchAttnError):
         binding.monarch_attn_fwd_objective(Qd, Kd, Vd, 32, 2, path=binding.MA_PATH_FUSED_JSPLIT)
+
+
+# ------------------------------------------------------------------ seeded sweep over shapes and entry points
+@pytest.mark.parametrize("seed", [1, 2])
+def test_seeded_sweep_of_shapes_through_every_entry_point(seed):
+    """About a hundred shapes per seed drawn from the block sizes, block counts, head sizes, round
+    counts and dtypes the library claims, each through one of the entry points (plain, other layout,
+    objective, padded, different lengths) with the kernel the library picks itself, every head
+    against the oracle.  (fp32 is kept to the milder recipe: at T = 4 on the peaky one fp32
+    arithmetic itself is at 2e-5.)"""
+    import random
+    rng = random.Random(seed)
+    done = 0
+    for it in range(130):
+        dtype = rng.choice(["f16", "bf16", "f16", "bf16", "f32"])
+        b = rng.choice([1, 2, 3, 5, 7, 8, 12, 14, 16, 17, 24, 31, 32, 33, 40, 48, 63, 64, 65, 96, 128])
+        m = rng.choice([1, 2, 3, 4, 6, 8, 12, 15, 16, 17, 24, 32, 33, 48, 64])
+        N = b * m
+        if N > 2048 or N < 2:
+            continue
+        d = rng.choice([8, 16, 24, 40, 48, 64, 64, 64, 72, 80, 96, 128]) if dtype != "f32" else rng.choice([4, 5, 7, 16, 40, 64, 72])
+        T = rng.choice([1, 1, 2, 2, 3, 4])
+        batch, heads = rng.choice([(1, 1), (1, 3), (2, 2), (3, 5)])
+        s = rng.choice([0.0, 1.0, 1.0, 2.0]) if dtype != "f32" else rng.choice([0.0, 1.0])
+        mode = rng.choice(["fwd", "fwd", "bshd", "objective", "padded", "varlen"])
+        Q, K, V = wl.make_qkv(batch, heads, N, d, dtype, min(8, d) if s else 0, s, seed=5000 * seed + it)
+        Qd, Kd, Vd = (binding.to_device(x, dtype) for x in (Q, K, V))
+        what = (mode, dtype, N, b, d, T, batch, heads, s)
+        lens = None
+        try:
+            if mode == "fwd":
+                Y, nv = binding.monarch_attn_fwd(Qd, Kd, Vd, b, T), None
+            elif mode == "bshd":
+                Y, nv = binding.monarch_attn_fwd_bshd(*(x.transpose(1, 2).contiguous() for x in (Qd, Kd, Vd)),
+                                                      b, T).transpose(1, 2), None
+            elif mode == "objective":
+                (Y, lse), nv = binding.monarch_attn_fwd_objective(Qd, Kd, Vd, b, T), None
+                assert bool(torch.isfinite(lse).all()), what
+            elif mode == "padded":
+                nv = rng.randint(N - b + 1, N)
+                Y = binding.monarch_attn_fwd_padded(Qd, Kd, Vd, b, T, nv)
+            else:
+                lens = [rng.randint(1, N) for _ in range(batch)]
+                nv = np.array(lens)
+                Y = binding.monarch_attn_fwd_varlen(Qd, Kd, Vd, b, T, torch.tensor(lens, dtype=torch.int32, device="cuda"))
+        except binding.MonarchAttnError as e:        # a shape no kernel takes (a tile too large for shared memory)
+            assert e.code == 4, what
+            continue
+        torch.cuda.synchronize()
+        Yn = Y.float().cpu().numpy().astype(np.float64)
+        ref = mo.monarch_attention(Q, K, V, b, T, n_valid=nv)
+        if lens is not None:
+            err = max(rel_err(Yn[e:e + 1, :, :lens[e]], ref[e:e + 1, :, :lens[e]]) for e in range(batch))
+        else:
+            rows = slice(0, nv) if mode == "padded" else slice(None)
+            assert np.isfinite(Yn[:, :, rows]).all(), what
+            err = rel_err(Yn[:, :, rows], ref[:, :, rows])
+        assert err <= TOL[dtype], (what, err)
+        done += 1
+    assert done >= 80
