@@ -223,16 +223,28 @@ def time_config(w, steps, warmup, torch, binding, n_sets=3, dist=None, units=Non
     if dist is not None:
         dist.barrier()
         torch.cuda.synchronize()
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
-    evs[0].record()
+    # the K timed steps: one event before the first, one after the last (an event record between
+    # steps costs 2.5 - 4.5 us of device time per step and keeps consecutive launches from
+    # overlapping their tails; measured)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
     for i in range(steps):
         call(sets[(warmup + i) % n_sets])
-        evs[i + 1].record()
+    e1.record()
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
-    total_ms = evs[0].elapsed_time(evs[-1])
-    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+    total_ms = e0.elapsed_time(e1)
+    # per-step statistics from a second, shorter loop with an event after every step (each step of
+    # this loop carries that event's overhead)
+    n_stat = min(steps, 50)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_stat + 1)]
+    evs[0].record()
+    for i in range(n_stat):
+        call(sets[i % n_sets])
+        evs[i + 1].record()
+    torch.cuda.synchronize()
+    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(n_stat)]
     assert binding.monarch_attn_device_status(status_of) == 0
     # host time of one call with an idle stream (argument checks, cached tensor maps, launch)
     host = []
