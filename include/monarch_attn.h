@@ -68,7 +68,9 @@ typedef enum {
                               f16 arithmetic with plain f16 states: what AUTO takes for T <= 2 */
   MA_PATH_FUSED_SMALL = 7, /* the same idea for any block shape: f16/bf16, m <= 32 and b <= 64 (m need
                              not equal b), d <= 64 a multiple of 8 (or b <= 32 and d <= 128), N <= 580 for T = 1 and <= 440 for
-                             T > 1 (the states of a head must fit shared memory); f16 arithmetic */
+                             T > 1 (the states of a head must fit shared memory); f16 arithmetic.
+                             For T >= 3 with m, b <= 16 and N <= ~290 the states and the weights that
+                             form them are hi + lo pairs of f16 (what AUTO takes there) */
   MA_PATH_TILE_MMA = 8    /* warp-MMA kernels, one launch per half-step, f16 states in the workspace
                              (hi + lo pairs of f16 from T = 3 on): f16/bf16, m and b <= 128 (m need
                              not equal b), d <= 128 a multiple of 8; the 16-bit path of the shapes no

@@ -167,6 +167,8 @@ static int resolve_path(const Problem& p, int path, bool plain = true) {
     // back round after round: about one head in 300 of the N = 256 recipe exceeds 1e-2 at T = 3).
     // The fused per-head kernel and the tcgen05 kernels keep such states; the tile kernels switch to
     // hi + lo pairs from T = 3 on, so they take every 16-bit shape they support then.
+    // (short sequences with small blocks: the fused per-head kernel with hi + lo states, one launch)
+    if (p.T >= 3 && fsmall::supported_hilo(p.N, p.d, p.b, p.m, p.dtype, p.T)) return MA_PATH_FUSED_SMALL;
     if (p.T >= 3 && tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_TILE_MMA;
     // N = 1024 as 32 x 32: one launch, a head split over four CTAs by in-block position
     if (plain && p.T <= 2 && jsplit::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) return MA_PATH_FUSED_JSPLIT;
@@ -364,7 +366,9 @@ int monarch_attn_fwd_padded(const void* Q, const void* K, const void* V, void* Y
   // fused kernel for short sequences; the second-generation tensor kernel where a tile row owns a
   // whole key block (b = 64, 128: the mask touches the last block's tiles only); else generic
   int r = -1;
-  if (p.T <= 2 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) r = MA_PATH_FUSED_SMALL;
+  if ((p.T <= 2 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) ||
+      fsmall::supported_hilo(p.N, p.d, p.b, p.m, p.dtype, p.T))
+    r = MA_PATH_FUSED_SMALL;
   else if (resolve_path(p, MA_PATH_AUTO, false) == MA_PATH_TENSOR && p.b != 32) r = MA_PATH_TENSOR;
   else if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) r = MA_PATH_TILE_MMA;
   else if (p.dtype == MA_F32 && p.BH <= 65535 && ffused::supported(p.N, p.d, p.b, p.m)) r = MA_PATH_FUSED_F32;
@@ -390,7 +394,9 @@ int monarch_attn_fwd_varlen(const void* Q, const void* K, const void* V, void* Y
   // 16-bit shapes: the warp-MMA tile kernels (hi + lo states from the third round on); else the
   // generic kernels
   int r = -1;
-  if (p.T <= 2 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) r = MA_PATH_FUSED_SMALL;
+  if ((p.T <= 2 && fsmall::supported(p.N, p.d, p.b, p.m, p.dtype, p.T)) ||
+      fsmall::supported_hilo(p.N, p.d, p.b, p.m, p.dtype, p.T))
+    r = MA_PATH_FUSED_SMALL;
   else if (tile::supported(p.N, p.d, p.b, p.m, p.dtype, p.BH)) r = MA_PATH_TILE_MMA;
   else if (generic_supported(p)) r = MA_PATH_GENERIC;
   if (r < 0) return MA_ERR_UNSUPPORTED;

@@ -58,6 +58,17 @@ __device__ __forceinline__ void stsm_x4(uint32_t saddr, uint32_t r0, uint32_t r1
                : "memory");
 }
 
+// x rounded to f16 (hi) and the f16 rounding of what is left (lo): hi + lo carries 22 bits of x.
+template <bool HILO>
+__device__ __forceinline__ void split_hilo(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  hi = Mma<__half>::pack(x0, x1);
+  lo = 0u;
+  if (HILO) {
+    const float2 h = Mma<__half>::unpack(hi);
+    lo = Mma<__half>::pack(x0 - h.x, x1 - h.y);
+  }
+}
+
 // Tile layouts.  KS = number of 16-column steps a row holds (4: d <= 64, 5: d <= 80, 8: d <= 128).
 // KS = 4: 128-byte rows, row k*b + i, 16-byte chunks XOR-swizzled with (i & 7) ^ (k & 7).
 // KS > 4: rows of 32 KS + 16 bytes and 16 more bytes after every block, no swizzle: eight rows of
@@ -92,15 +103,18 @@ inline size_t tile_bytes(int N, int b, int ks) {
   return ks == 4 ? (size_t)N * kRowBytes : (size_t)m * ((size_t)b * (32 * ks + 16) + 16);
 }
 inline int ksteps_for(int d) { return d <= 64 ? 4 : (d <= 80 ? 5 : 8); }
-inline size_t smem_bytes(int N, int T, int threads = kThreads, int b = 16, int ks = 4) {
-  return (size_t)(T == 1 ? 3 : 4) * tile_bytes(N, b, ks) + (((size_t)N * 4 + 15) & ~(size_t)15) + dump_bytes(threads) + 1024;
+inline size_t smem_bytes(int N, int T, int threads = kThreads, int b = 16, int ks = 4, bool hilo = false) {
+  return (size_t)(T == 1 ? 3 : (hilo ? 6 : 4)) * tile_bytes(N, b, ks) + (((size_t)N * 4 + 15) & ~(size_t)15) + dump_bytes(threads) + 1024;
 }
 
 // BP: b rounded up to 16, 32, 48 or 64; MP: m rounded up to 16 or 32.  EXACT: b = BP, m = MP, d = 64
 // and no mask, known at compile time: every clamp, mask and bounds predicate below folds away and
 // the index products become shifts (the instruction stream, not a pipe, bounds this kernel).
-template <typename TIn, int BP, int MP, bool EXACT = false, int KS = 4>
-__global__ void __launch_bounds__((KS == 4 && BP <= 32 && (BP == 16 || MP == 16)) ? 2 * kThreads : kThreads, 1)
+// HILO: alpha_L, alpha_R and the weights that feed them are hi + lo pairs of f16 (two more tiles): what
+// three or more rounds on peaky logits need (plain 16-bit states, fed back round after round, lose
+// 1e-2 on about one head in 300 at T = 3).
+template <typename TIn, int BP, int MP, bool EXACT = false, int KS = 4, bool HILO = false>
+__global__ void __launch_bounds__((KS == 4 && !HILO && BP <= 32 && (BP == 16 || MP == 16)) ? 2 * kThreads : kThreads, 1)
 monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const TIn* __restrict__ V,
                     TIn* __restrict__ Y, int N, int d, int b, int m, int T_steps, float scale,
                     int n_valid, int H, float* __restrict__ lse, const int* __restrict__ seq_len,
@@ -132,7 +146,8 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   // then K, then V (loaded when the last round starts) ...
   //                                                  ... alpha_L of the earlier rounds until then;
   // alpha_R (T > 1 only) follows it
-  float* sCL = reinterpret_cast<float*>(smem + (T_steps == 1 ? 3 : 4) * (size_t)tile);   // [k*b + j]
+  // (hi + lo states: the low halves of alpha_L and alpha_R follow alpha_R)
+  float* sCL = reinterpret_cast<float*>(smem + (T_steps == 1 ? 3 : (HILO ? 6 : 4)) * (size_t)tile);   // [k*b + j]
   const uint32_t sQ_u = (uint32_t)__cvta_generic_to_shared(sQ);
   // stmatrix writes whole 8-row matrices: rows past a block's end land in a per-lane dump slot
   const uint32_t dump_u =
@@ -141,6 +156,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   const int st_row = (threadIdx.x & 7) + ((threadIdx.x >> 3) & 1) * 8;   // row within a 16-row tile
   const int st_nt = (threadIdx.x >> 4) & 1;                              // which of a pair of 8-column tiles
   const uint32_t sK_u = sQ_u + tile, sV_u = sK_u + tile;
+  const uint32_t sALlo_u = sQ_u + 4 * tile, sARlo_u = sQ_u + 5 * tile;   // HILO only
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nw = blockDim.x >> 5;    // 8 warps, or 16 where only one CTA fits an SM (16 x 16 blocks)
@@ -224,7 +240,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
         }
         // phase 1: scores and softmax of every 16-row tile of the block; the weights stay in
         // registers as A fragments
-        uint32_t pa[BP / 16][BP / 16][4];
+        uint32_t pa[BP / 16][BP / 16][4], pal[HILO ? BP / 16 : 1][HILO ? BP / 16 : 1][4];
         float inv_s[BP / 16][2];
 #pragma unroll
         for (int rt = 0; rt < BP / 16; ++rt) {
@@ -243,14 +259,19 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             b_u[cp] = sK_u + rowx<KS>(k, min(16 * cp + (lane & 7) + (lane >> 4) * 8, b - 1), b, (lane >> 3) & 1);
 #pragma unroll
           for (int ks = 0; ks < ksteps; ++ks) {
-            uint32_t a[4];
+            uint32_t a[4], al[4];
             ldsm_x4(a, stp<KS>(a_u, ks));
+            if (HILO && !first) ldsm_x4(al, stp<KS>(a_u - sA_u + sARlo_u, ks));
 #pragma unroll
             for (int cp = 0; cp < BP / 16; ++cp) {
               uint32_t bf[4];
               ldsm_x4(bf, stp<KS>(b_u[cp], ks));
               Mma<T>::run(s[2 * cp], a, bf);
               Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+              if (HILO && !first) {      // + <alpha_R lo, K>
+                Mma<T>::run(s[2 * cp], al, bf);
+                Mma<T>::run(s[2 * cp + 1], al, bf + 2);
+              }
             }
           }
           // rows j = j0 + g (c0, c1) and j0 + g + 8 (c2, c3); columns i = 8 nt + 2t, +1
@@ -292,6 +313,14 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             pa[rt][kk][1] = Mma<T>::pack(s[2 * kk][2], s[2 * kk][3]);
             pa[rt][kk][2] = Mma<T>::pack(s[2 * kk + 1][0], s[2 * kk + 1][1]);
             pa[rt][kk][3] = Mma<T>::pack(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+            if (HILO) {                // what the f16 rounding of the weights left out
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float2 hi = Mma<T>::unpack(pa[rt][kk][q]);
+                const int nt = 2 * kk + (q >> 1), e0 = 2 * (q & 1);
+                pal[rt][kk][q] = Mma<T>::pack(s[nt][e0] - hi.x, s[nt][e0 + 1] - hi.y);
+              }
+            }
           }
         }
         // phase 2: second products, one 16-column slab of v at a time for all row tiles.  This warp
@@ -319,6 +348,10 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             for (int kk = 0; kk < BP / 16; ++kk) {
               Mma<T>::run(o[0], pa[rt][kk], bk[kk]);
               Mma<T>::run(o[1], pa[rt][kk], bk[kk] + 2);
+              if (HILO) {
+                Mma<T>::run(o[0], pal[rt][kk], bk[kk]);
+                Mma<T>::run(o[1], pal[rt][kk], bk[kk] + 2);
+              }
               if (last) {
                 Mma<T>::run(y[0], pa[rt][kk], bv[kk]);
                 Mma<T>::run(y[1], pa[rt][kk], bv[kk] + 2);
@@ -327,9 +360,13 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
             const int j = 16 * rt + st_row;
             const uint32_t off = stp<KS>(rowx<KS>(k, j, b, st_nt), np);
             const float i0 = inv_s[rt][0], i1 = inv_s[rt][1];
-            stsm_x4(j < b ? dstL_u + off : dump_u, Mma<T>::pack(o[0][0] * i0, o[0][1] * i0),
-                    Mma<T>::pack(o[0][2] * i1, o[0][3] * i1), Mma<T>::pack(o[1][0] * i0, o[1][1] * i0),
-                    Mma<T>::pack(o[1][2] * i1, o[1][3] * i1));
+            uint32_t hi[4], lo[4];
+            split_hilo<HILO>(o[0][0] * i0, o[0][1] * i0, hi[0], lo[0]);
+            split_hilo<HILO>(o[0][2] * i1, o[0][3] * i1, hi[1], lo[1]);
+            split_hilo<HILO>(o[1][0] * i0, o[1][1] * i0, hi[2], lo[2]);
+            split_hilo<HILO>(o[1][2] * i1, o[1][3] * i1, hi[3], lo[3]);
+            stsm_x4(j < b ? dstL_u + off : dump_u, hi[0], hi[1], hi[2], hi[3]);
+            if (HILO) stsm_x4(j < b ? sALlo_u + off : dump_u, lo[0], lo[1], lo[2], lo[3]);
             if (last)
               stsm_x4(j < b ? sV_u + off : dump_u, Mma<T>::pack(y[0][0] * i0, y[0][1] * i0),
                       Mma<T>::pack(y[0][2] * i1, y[0][3] * i1), Mma<T>::pack(y[1][0] * i0, y[1][1] * i0),
@@ -384,6 +421,11 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
               ldsm_x4(bf, stp<KS>(b_u[cp], ks));
               Mma<T>::run(s[2 * cp], a, bf);
               Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+              if (HILO) {      // + <Q, alpha_L lo>
+                ldsm_x4(bf, stp<KS>(b_u[cp] - sAL_u + sALlo_u, ks));
+                Mma<T>::run(s[2 * cp], a, bf);
+                Mma<T>::run(s[2 * cp + 1], a, bf + 2);
+              }
             }
           }
           float inv_s[2];
@@ -481,7 +523,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
           // The result does not change when column k is multiplied by any g_k > 0: g_k = 2^-(exponent
           // of the column's largest weight) keeps every column's significant weights in the normal
           // f16 range however small c_R is.
-          uint32_t tp[MP / 16][2][MP / 8];
+          uint32_t tp[MP / 16][2][MP / 8], tpl[HILO ? MP / 16 : 1][2][HILO ? MP / 8 : 1];
           float cs[MP / 8][2];
 #pragma unroll
           for (int nt = 0; nt < MP / 8; ++nt) {
@@ -505,7 +547,14 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
               for (int hh = 0; hh < 2; ++hh) {
                 const uint32_t u = Mma<T>::pack(pn[rt][hh][nt][0] * gk[0], pn[rt][hh][nt][1] * gk[1]);
                 tp[rt][hh][nt] = u;
-                const float2 f = Mma<T>::unpack(u);
+                float2 f = Mma<T>::unpack(u);
+                if (HILO) {      // the pair carries the weight to 22 bits; c_R sums what the MMAs will see
+                  const uint32_t ul = Mma<T>::pack(pn[rt][hh][nt][0] * gk[0] - f.x, pn[rt][hh][nt][1] * gk[1] - f.y);
+                  tpl[rt][hh][nt] = ul;
+                  const float2 fl2 = Mma<T>::unpack(ul);
+                  f.x += fl2.x;
+                  f.y += fl2.y;
+                }
                 c0 += f.x;
                 c1 += f.y;
               }
@@ -524,13 +573,19 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
               const float cr = (g & 1) ? v1 : v0;
               ic[hh] = cr > 1e-30f ? 1.f / cr : 0.f;
             }
-            uint32_t pa[MP / 16][4];
+            uint32_t pa[MP / 16][4], pal[HILO ? MP / 16 : 1][4];
 #pragma unroll
             for (int ls = 0; ls < MP / 16; ++ls) {
               pa[ls][0] = movm_trans(tp[ls][0][2 * kt]);       // rows k 0-7,  cols l 0-7
               pa[ls][1] = movm_trans(tp[ls][0][2 * kt + 1]);   // rows k 8-15, cols l 0-7
               pa[ls][2] = movm_trans(tp[ls][1][2 * kt]);       // rows k 0-7,  cols l 8-15
               pa[ls][3] = movm_trans(tp[ls][1][2 * kt + 1]);   // rows k 8-15, cols l 8-15
+              if (HILO) {
+                pal[ls][0] = movm_trans(tpl[ls][0][2 * kt]);
+                pal[ls][1] = movm_trans(tpl[ls][0][2 * kt + 1]);
+                pal[ls][2] = movm_trans(tpl[ls][1][2 * kt]);
+                pal[ls][3] = movm_trans(tpl[ls][1][2 * kt + 1]);
+              }
             }
             uint32_t q_u[MP / 16];
 #pragma unroll
@@ -547,10 +602,18 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
                 ldsm_x4_trans(bf, stp<KS>(q_u[ls], np));
                 Mma<T>::run(o[0], pa[ls], bf);
                 Mma<T>::run(o[1], pa[ls], bf + 2);
+                if (HILO) {
+                  Mma<T>::run(o[0], pal[ls], bf);
+                  Mma<T>::run(o[1], pal[ls], bf + 2);
+                }
               }
-              stsm_x4(kr < m ? stp<KS>(row_u, np) : dump_u,
-                      Mma<T>::pack(o[0][0] * ic[0], o[0][1] * ic[0]), Mma<T>::pack(o[0][2] * ic[1], o[0][3] * ic[1]),
-                      Mma<T>::pack(o[1][0] * ic[0], o[1][1] * ic[0]), Mma<T>::pack(o[1][2] * ic[1], o[1][3] * ic[1]));
+              uint32_t hi[4], lo[4];
+              split_hilo<HILO>(o[0][0] * ic[0], o[0][1] * ic[0], hi[0], lo[0]);
+              split_hilo<HILO>(o[0][2] * ic[1], o[0][3] * ic[1], hi[1], lo[1]);
+              split_hilo<HILO>(o[1][0] * ic[0], o[1][1] * ic[0], hi[2], lo[2]);
+              split_hilo<HILO>(o[1][2] * ic[1], o[1][3] * ic[1], hi[3], lo[3]);
+              stsm_x4(kr < m ? stp<KS>(row_u, np) : dump_u, hi[0], hi[1], hi[2], hi[3]);
+              if (HILO) stsm_x4(kr < m ? stp<KS>(row_u - sAR_u + sARlo_u, np) : dump_u, lo[0], lo[1], lo[2], lo[3]);
             }
           }
         }
@@ -566,23 +629,29 @@ inline bool supported(int N, int d, int b, int m, int dtype, int T) {
          smem_bytes(N, T, kThreads, b, ksteps_for(d)) <= (size_t)kMaxSmem;
 }
 
+// Three or more rounds with hi + lo states: blocks and block counts up to 16, six tiles in shared memory.
+inline bool supported_hilo(int N, int d, int b, int m, int dtype, int T) {
+  return (dtype == 1 || dtype == 2) && T >= 3 && d % 8 == 0 && d <= 64 && b <= 16 && m <= 16 &&
+         smem_bytes(N, T, kThreads, b, 4, true) <= (size_t)kMaxSmem;
+}
+
 int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
            int m, int T, int dtype, float scale, int n_valid, int H, float* lse, cudaStream_t st,
            const int* seq_len = nullptr, int heads = 1);
 
 #ifdef MA_TU_FUSED_SMALL
-template <typename TIn, int BP, int MP, bool EXACT = false, int KS = 4>
+template <typename TIn, int BP, int MP, bool EXACT = false, int KS = 4, bool HILO = false>
 inline int launch_t(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
                     int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st,
                     const int* seq_len, int heads) {
-  auto kern = monarch_fused_small<TIn, BP, MP, EXACT, KS>;
+  auto kern = monarch_fused_small<TIn, BP, MP, EXACT, KS, HILO>;
   // The 16 x 16 kernel is compiled for 128 registers: two CTAs of 8 warps per SM where shared memory
   // lets two fit, else one CTA of 16 warps (each warp then owns at most one tile per half-step).
   int threads = kThreads;
-  if (KS == 4 && BP <= 32 && (BP == 16 || MP == 16) && 2 * (smem_bytes(N, T) + 1024) > (size_t)228 * 1024 &&
+  if (KS == 4 && !HILO && BP <= 32 && (BP == 16 || MP == 16) && 2 * (smem_bytes(N, T) + 1024) > (size_t)228 * 1024 &&
       (m > 8 || b > 8) && smem_bytes(N, T, 2 * kThreads) <= (size_t)kMaxSmem)
     threads = 2 * kThreads;
-  const size_t smem = smem_bytes(N, T, threads, b, KS);
+  const size_t smem = smem_bytes(N, T, threads, b, KS, HILO);
   if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
     return 7;
@@ -610,6 +679,8 @@ inline int launch_d(const void* Q, const void* K, const void* V, void* Y, int BH
                     int m, int T, float scale, int n_valid, int H, float* lse, cudaStream_t st,
                     const int* seq_len, int heads) {
 #define MA_FS_ARGS Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st, seq_len, heads
+  if (supported_hilo(N, d, b, m, 1, T))   // three or more rounds: hi + lo states
+    return launch_t<TIn, 16, 16, false, 4, true>(MA_FS_ARGS);
   if (d == 64 && n_valid >= N && seq_len == nullptr) {   // exact fits, no mask
     if (b == 16 && m == 16) return launch_t<TIn, 16, 16, true>(MA_FS_ARGS);
     if (b == 32 && m == 32) return launch_t<TIn, 32, 32, true>(MA_FS_ARGS);

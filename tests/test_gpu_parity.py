@@ -152,11 +152,15 @@ def test_three_rounds_on_peaky_logits_hold_the_tolerance_on_every_head(N, b):
     w = wl.WORKLOADS["C2"]
     Q, K, V = wl.make_qkv(26, 12, N, 64, "f16", w.rank, w.s, seed=900 + N)
     Y = gpu_forward(Q, K, V, "f16", b, 3, use_ex=False)
+    assert binding.monarch_attn_last_launch_count() == 1       # the fused kernel with hi + lo states
     ref = mo.monarch_attention(Q, K, V, b, 3)
     errs = np.array([np.linalg.norm(Y[e, h] - ref[e, h]) / np.linalg.norm(ref[e, h])
                      for e in range(26) for h in range(12)])
     print(f"N={N} b={b} T=3: worst {errs.max():.3e}, mean {errs.mean():.3e}, over 5e-3: {(errs > 5e-3).sum()}")
     assert errs.max() <= 1e-2, errs.max()
+    # the same through the tile kernels (what shapes too long for six tiles of shared memory get)
+    Yt = gpu_forward(Q[:4], K[:4], V[:4], "f16", b, 3, binding.MA_PATH_TILE_MMA)
+    assert rel_err(Yt, ref[:4]) <= 1e-2
 
 
 def test_persistent_tensor_kernels_agree_with_the_one_tile_per_cta_kernels():
@@ -688,7 +692,8 @@ def test_results_are_bit_identical_from_call_to_call(name):
     (210, 14, 64, 2, "f16", [197, 210, 120, 29, 14, 1], 1, "FUSED_SMALL"),  # ViT-like batch
     (384, 24, 64, 1, "bf16", [384, 300, 100, 23], 1, "FUSED_SMALL"),     # fused kernel, m != b
     (256, 16, 72, 2, "f16", [256, 131, 16], 1, "FUSED_SMALL"),           # fused kernel, wide rows
-    (256, 16, 64, 3, "f16", [256, 250, 130, 40], 6, "TILE_MMA"),         # three rounds: hi + lo states
+    (256, 16, 64, 3, "f16", [256, 250, 130, 40], 1, "FUSED_SMALL"),      # three rounds: fused kernel, hi + lo states
+    (384, 24, 64, 3, "f16", [384, 250, 130, 40], 6, "TILE_MMA"),         # three rounds, blocks wider than 16: tile kernels
     (1024, 32, 64, 2, "bf16", [1024, 700, 333, 64, 31], 4, "TILE_MMA"),  # longer than the fused kernel takes
     (768, 96, 48, 1, "f16", [768, 500, 97, 96, 700], 2, "TILE_MMA"),     # wide blocks, m != b, d = 48
     (2048, 32, 64, 2, "f16", [2048, 1030, 33], 4, "TILE_MMA"),           # m = 64 blocks, most of them absent
