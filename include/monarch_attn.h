@@ -69,7 +69,7 @@ typedef enum {
   MA_PATH_FUSED_SMALL = 7, /* the same idea for any block shape: f16/bf16, m <= 32 and b <= 64 (m need
                              not equal b), d <= 64 a multiple of 8 (or b <= 32 and d <= 128), N <= 580 for T = 1 and <= 440 for
                              T > 1 (the states of a head must fit shared memory); f16 arithmetic.
-                             For T >= 3 with m, b <= 16 and N <= ~290 the states and the weights that
+                             For T >= 3 with m, b <= 16 and d <= 80 the states and the weights that
                              form them are hi + lo pairs of f16 (what AUTO takes there) */
   MA_PATH_TILE_MMA = 8    /* warp-MMA kernels, one launch per half-step, f16 states in the workspace
                              (hi + lo pairs of f16 from T = 3 on): f16/bf16, m and b <= 128 (m need

@@ -104,7 +104,9 @@ inline size_t tile_bytes(int N, int b, int ks) {
 }
 inline int ksteps_for(int d) { return d <= 64 ? 4 : (d <= 80 ? 5 : 8); }
 inline size_t smem_bytes(int N, int T, int threads = kThreads, int b = 16, int ks = 4, bool hilo = false) {
-  return (size_t)(T == 1 ? 3 : (hilo ? 6 : 4)) * tile_bytes(N, b, ks) + (((size_t)N * 4 + 15) & ~(size_t)15) + dump_bytes(threads) + 1024;
+  // (alignment slack: the XOR-swizzled layout needs a 1024-byte aligned base, the padded one 128)
+  return (size_t)(T == 1 ? 3 : (hilo ? 5 : 4)) * tile_bytes(N, b, ks) + (((size_t)N * 4 + 15) & ~(size_t)15) + dump_bytes(threads) +
+         (ks == 4 ? 1024 : 128);
 }
 
 // BP: b rounded up to 16, 32, 48 or 64; MP: m rounded up to 16 or 32.  EXACT: b = BP, m = MP, d = 64
@@ -140,14 +142,17 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
     n_valid = min(max(seq_len[blockIdx.x / heads], 1), N);
     m = (n_valid + b - 1) / b;
   }
-  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  constexpr uintptr_t kAlign = KS == 4 ? 1024 : 128;
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + kAlign - 1) & ~(kAlign - 1));
   const int tile = KS == 4 ? N * kRowBytes : (N / b) * block_bytes<KS>(b);
   uint8_t* sQ = smem;
   // then K, then V (loaded when the last round starts) ...
   //                                                  ... alpha_L of the earlier rounds until then;
   // alpha_R (T > 1 only) follows it
-  // (hi + lo states: the low halves of alpha_L and alpha_R follow alpha_R)
-  float* sCL = reinterpret_cast<float*>(smem + (T_steps == 1 ? 3 : (HILO ? 6 : 4)) * (size_t)tile);   // [k*b + j]
+  // hi + lo states (HILO): Q, K, V, then ONE state tile and its low halves -- alpha_R and alpha_L
+  // replace each other in place there (an R tile reads the rows (k, .) it then overwrites, an L tile
+  // the rows (., j)), and V has a tile of its own from the start
+  float* sCL = reinterpret_cast<float*>(smem + (T_steps == 1 ? 3 : (HILO ? 5 : 4)) * (size_t)tile);   // [k*b + j]
   const uint32_t sQ_u = (uint32_t)__cvta_generic_to_shared(sQ);
   // stmatrix writes whole 8-row matrices: rows past a block's end land in a per-lane dump slot
   const uint32_t dump_u =
@@ -156,7 +161,8 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   const int st_row = (threadIdx.x & 7) + ((threadIdx.x >> 3) & 1) * 8;   // row within a 16-row tile
   const int st_nt = (threadIdx.x >> 4) & 1;                              // which of a pair of 8-column tiles
   const uint32_t sK_u = sQ_u + tile, sV_u = sK_u + tile;
-  const uint32_t sALlo_u = sQ_u + 4 * tile, sARlo_u = sQ_u + 5 * tile;   // HILO only
+  const uint32_t sS_u = sQ_u + 3 * tile, sALlo_u = sQ_u + 4 * tile, sARlo_u = sALlo_u;   // HILO only
+  const bool v_early = HILO || T_steps == 1;      // V comes in with the first round's loads
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nw = blockDim.x >> 5;    // 8 warps, or 16 where only one CTA fits an SM (16 x 16 blocks)
@@ -209,7 +215,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   for (int k = warp; k < m; k += nw) {
     load_block(Q, 0, k);
     load_block(K, 1, k);
-    if (T_steps == 1) load_block(V, 2, k);
+    if (v_early) load_block(V, 2, k);
     asm volatile("cp.async.commit_group;" ::: "memory");
     ++my_tiles;
   }
@@ -217,7 +223,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
   const float fl = scale * kLog2e;
   for (int step = 1; step <= T_steps; ++step) {
     const bool first = step == 1, last = step == T_steps;
-    if (last && !first) {   // alpha_L of the round before is dead: V takes its buffer
+    if (last && !first && !v_early) {   // alpha_L of the round before is dead: V takes its buffer
       for (int k = warp; k < m; k += nw) {
         load_block(V, 2, k);
         asm volatile("cp.async.commit_group;" ::: "memory");
@@ -226,16 +232,16 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
     // ================================================================ R half-step (Eq. 7, 9, 10)
     // tile k: Z_R[j,i] = fl * <alpha_R(k,j), K(k,i)>, softmax over i, alpha_L(k,j) = sum_i R K(k,i)
     {
-      const uint32_t sA_u = first ? sQ_u : sV_u + tile;   // alpha_R (= Q rows while L is the identity)
+      const uint32_t sA_u = first ? sQ_u : (HILO ? sS_u : sV_u + tile);   // alpha_R (= Q rows while L is the identity)
       int it = 0;
       for (int k = warp; k < m; k += nw, ++it) {
-        if (first || last) {          // block k may still be on its way
+        if (first || (last && !v_early)) {          // block k may still be on its way
           wait_pending(my_tiles - 1 - it);
           if (first) {
             convert_block(0, k);
             convert_block(1, k);
           }
-          if (last) convert_block(2, k);
+          if (first ? v_early : true) convert_block(2, k);
           __syncwarp();
         }
         // phase 1: scores and softmax of every 16-row tile of the block; the weights stay in
@@ -326,7 +332,7 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
         // phase 2: second products, one 16-column slab of v at a time for all row tiles.  This warp
         // alone reads block k of K and V, and every score is formed: on the last round the slab of
         // alpha_L / y goes straight over the slab of K / V it was computed from.
-        const uint32_t dstL_u = last ? sK_u : sV_u;     // alpha_L of earlier rounds shares V's buffer
+        const uint32_t dstL_u = last ? sK_u : (HILO ? sS_u : sV_u);     // alpha_L of earlier rounds shares V's buffer
         uint32_t v_off[BP / 16];    // rows (k, i) of K and V as the second product's B operand
 #pragma unroll
         for (int kk = 0; kk < BP / 16; ++kk) v_off[kk] = rowx<KS>(k, min(16 * kk + (lane & 15), b - 1), b, lane >> 4);
@@ -380,8 +386,8 @@ monarch_fused_small(const TIn* __restrict__ Q, const TIn* __restrict__ K, const 
     // ================================================================ L half-step (Eq. 8, 9 / Eq. 4)
     // tile j: Z_L[l,k] = fl * <Q(l,j), alpha_L(k,j)> - c_L(k,j), softmax over k
     {
-      const uint32_t sAL_u = last ? sK_u : sV_u;      // alpha_L of earlier rounds shares V's buffer
-      const uint32_t sAR_u = sV_u + tile;
+      const uint32_t sAL_u = last ? sK_u : (HILO ? sS_u : sV_u);      // alpha_L of earlier rounds shares V's buffer
+      const uint32_t sAR_u = HILO ? sS_u : sV_u + tile;
       for (int j = warp; j < b; j += nw) {
         float c[MP / 8][2];
 #pragma unroll
@@ -629,10 +635,11 @@ inline bool supported(int N, int d, int b, int m, int dtype, int T) {
          smem_bytes(N, T, kThreads, b, ksteps_for(d)) <= (size_t)kMaxSmem;
 }
 
-// Three or more rounds with hi + lo states: blocks and block counts up to 16, six tiles in shared memory.
+// Three or more rounds with hi + lo states: blocks and block counts up to 16, d <= 80, five tiles in
+// shared memory.
 inline bool supported_hilo(int N, int d, int b, int m, int dtype, int T) {
-  return (dtype == 1 || dtype == 2) && T >= 3 && d % 8 == 0 && d <= 64 && b <= 16 && m <= 16 &&
-         smem_bytes(N, T, kThreads, b, 4, true) <= (size_t)kMaxSmem;
+  return (dtype == 1 || dtype == 2) && T >= 3 && d % 8 == 0 && d <= 80 && b <= 16 && m <= 16 &&
+         smem_bytes(N, T, kThreads, b, ksteps_for(d), true) <= (size_t)kMaxSmem;
 }
 
 int launch(const void* Q, const void* K, const void* V, void* Y, int BH, int N, int d, int b,
@@ -680,7 +687,7 @@ inline int launch_d(const void* Q, const void* K, const void* V, void* Y, int BH
                     const int* seq_len, int heads) {
 #define MA_FS_ARGS Q, K, V, Y, BH, N, d, b, m, T, scale, n_valid, H, lse, st, seq_len, heads
   if (supported_hilo(N, d, b, m, 1, T))   // three or more rounds: hi + lo states
-    return launch_t<TIn, 16, 16, false, 4, true>(MA_FS_ARGS);
+    return d <= 64 ? launch_t<TIn, 16, 16, false, 4, true>(MA_FS_ARGS) : launch_t<TIn, 16, 16, false, 5, true>(MA_FS_ARGS);
   if (d == 64 && n_valid >= N && seq_len == nullptr) {   // exact fits, no mask
     if (b == 16 && m == 16) return launch_t<TIn, 16, 16, true>(MA_FS_ARGS);
     if (b == 32 && m == 32) return launch_t<TIn, 32, 32, true>(MA_FS_ARGS);
